@@ -1,0 +1,195 @@
+/*
+ * team.h -- C ABI of the TEAM MoE-layer library for NVIDIA B200 (sm_100a).
+ *
+ * One call of team_moe_forward() is the MoE feed-forward layer of one
+ * denoising step of a block-diffusion MoE language model, with the expert
+ * activation rule of TEAM (arXiv 2602.08404):
+ *
+ *   - Sec. 4.1 (delayed caching, DCD): tokens decoded two or more steps ago
+ *     are not recomputed; only masked tokens and tokens accepted in the
+ *     previous step enter the layer.
+ *   - Sec. 4.2, Eq. 4: a masked token is "hot" if its last confidence exceeds
+ *     tau_hot or it lies within L_hot positions of a decoded token, else "cold".
+ *   - Sec. 4.3, Algorithm 1 (limited activation, LAC): newly accepted and hot
+ *     tokens are routed over all experts; the union of their top-k sets is the
+ *     necessary set E_A; cold tokens are routed inside E_A only.
+ *   - Sec. 4.2 (speculative exploration, SEH): the caller lays the branches of
+ *     a sequence out as extra rows with a branch id; rows of one group share
+ *     E_A and one pass over the expert weights.
+ *   - The layer itself: fp32 router, softmax, top-k, renormalised routing
+ *     weights, expert dispatch, SwiGLU experts, weighted combine (Sec. 1 and
+ *     Algorithm 1 "Router"; the paper leaves the arithmetic to the base model).
+ *
+ * Conventions
+ *   - Every pointer inside team_weights, team_step_state, team_routing and the
+ *     x / y arguments is DEVICE memory owned by the caller.  The library
+ *     borrows weight pointers from team_set_weights() until they are replaced
+ *     or the context is destroyed, and never frees caller memory.
+ *   - team_config, team_weights, team_step_state and team_routing structs
+ *     themselves live in HOST memory and are read during the call only.
+ *   - Calls are asynchronous on `stream` (a cudaStream_t passed as void*,
+ *     NULL = default stream).  The return value reports argument and launch
+ *     errors only; conditions detected on the device (an index out of range,
+ *     a bounded wait that gave up, a layout contract broken) set a status word
+ *     read back with team_read_status(); kernels always terminate.
+ *   - No global state; a context may be used from one thread at a time.  Calls
+ *     on one context must be stream-ordered with respect to each other because
+ *     they share the context's workspace.
+ *   - There is no CPU fallback: without a usable CUDA device every compute
+ *     entry point returns TEAM_ERR_CUDA.
+ *
+ * Row layout.  A call presents T = n_rows rows.  Rows that share (group,
+ * branch) must be contiguous and form one decoding block (at most
+ * TEAM_MAX_BLOCK rows); `pos` is the position inside that block.  `group` is
+ * the scope of E_A (normally the sequence), 0 <= group < max_groups.
+ *
+ * Slot ids.  Row t's j-th routed choice is slot t*top_k + j.  Shared expert s
+ * (expert id n_experts + s) applied to row t is slot T*top_k + s*T + t and has
+ * combine weight 1.
+ */
+#ifndef TEAM_H_
+#define TEAM_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct team_ctx team_ctx;
+
+enum {
+  TEAM_OK = 0,
+  TEAM_ERR_ARG = -1,     /* NULL pointer, n_rows out of range, missing weights         */
+  TEAM_ERR_SHAPE = -2,   /* configuration the kernels do not support                   */
+  TEAM_ERR_CUDA = -3,    /* CUDA runtime / driver error (see team_last_cuda_error)     */
+  TEAM_ERR_TIMEOUT = -4, /* device status: a bounded wait expired                      */
+  TEAM_ERR_STATE = -5    /* device status: row layout contract broken / index range    */
+};
+
+enum { TEAM_TOK_MASKED = 0, TEAM_TOK_NEW = 1, TEAM_TOK_CACHED = 2 };   /* team_step_state.tok_state */
+enum { TEAM_CLS_SKIP = 0, TEAM_CLS_FIRST = 1, TEAM_CLS_COLD = 2 };     /* team_routing.tok_class    */
+enum { TEAM_F_DCD = 1, TEAM_F_LAC = 2 };                               /* team_config.flags; 0 = vanilla top-k */
+enum { TEAM_DTYPE_F32 = 0, TEAM_DTYPE_BF16 = 1 };
+
+#define TEAM_MAX_EXPERTS 256   /* routed experts                       */
+#define TEAM_MAX_TOPK 16
+#define TEAM_MAX_SHARED 4
+#define TEAM_MAX_ROWS 4096     /* rows per call                        */
+#define TEAM_MAX_BLOCK 64      /* rows of one (group, branch)          */
+
+typedef struct {
+  int32_t hidden;      /* H; multiple of 64 for bf16, of 4 for fp32                      */
+  int32_t n_experts;   /* E routed experts, multiple of 32, <= TEAM_MAX_EXPERTS (fp32 path: any E >= top_k) */
+  int32_t top_k;       /* k <= min(E, TEAM_MAX_TOPK)                                    */
+  int32_t inter;       /* I; multiple of 64 for bf16, of 4 for fp32                      */
+  int32_t n_shared;    /* always-on experts appended after the routed ones              */
+  int32_t max_rows;    /* largest n_rows of any call on this context                    */
+  int32_t max_groups;  /* group ids are in [0, max_groups)                              */
+  int32_t dtype;       /* TEAM_DTYPE_F32: x and expert weights fp32 (plain FMA kernels);
+                          TEAM_DTYPE_BF16: x and expert weights bf16, fp32 accumulation
+                          on tensor cores.  Router weights and y are fp32 in both.      */
+  int32_t flags;       /* TEAM_F_* bits                                                 */
+  float tau_hot;       /* Eq. 4 confidence threshold (paper default 0.7)                */
+  int32_t L_hot;       /* Eq. 4 distance bound (paper default 3)                        */
+  int32_t hot_dist_inclusive; /* 1: |k-j| <= L_hot (Sec. 5.1 wording), 0: < (Eq. 4 as printed) */
+  int32_t prefix_decoded;     /* 1: position -1 (previous block) counts as decoded      */
+  int32_t norm_topk;          /* 1: routing weights renormalised over the k chosen      */
+} team_config;
+
+typedef struct {
+  const void *w_router; /* fp32 [E, H] row-major                                          */
+  const void *w_gate;   /* [E + n_shared, I, H] row-major, dtype per config               */
+  const void *w_up;     /* [E + n_shared, I, H]                                           */
+  const void *w_down;   /* [E + n_shared, H, I]                                           */
+} team_weights;
+
+/* State carried from the previous denoising step (Algorithm 1 inputs D, M; Eq. 4). */
+typedef struct {
+  int32_t n_rows;           /* T, 1 <= T <= max_rows                                      */
+  const uint8_t *tok_state; /* [T] TEAM_TOK_*                                             */
+  const float *conf;        /* [T] confidence c_k of the previous step's prediction       */
+  const int32_t *pos;       /* [T] position in the block                                  */
+  const int32_t *group;     /* [T] scope of E_A                                           */
+  const int32_t *branch;    /* [T] speculative branch id (scope of "decoded" in Eq. 4)    */
+} team_step_state;
+
+/* Optional outputs; any pointer may be NULL.  team_route fills probs, topk_idx,
+ * topk_w, margin with the plain (unrestricted) top-k of every computed row;
+ * team_select_experts / team_moe_forward fill everything with TEAM's choice. */
+typedef struct {
+  float *probs;           /* [T, E] softmax over all experts (computed rows; others 0)     */
+  int32_t *topk_idx;      /* [T, k] descending score, ties to the lower id; -1 if skipped  */
+  float *topk_w;          /* [T, k] routing weights                                        */
+  float *margin;          /* [T] logit gap between the last expert taken and the best one
+                             left out of the candidate set (+inf if none, or skipped)     */
+  uint8_t *tok_class;     /* [T] TEAM_CLS_*                                                */
+  uint64_t *group_mask;   /* [max_groups, ceil(E/64)] necessary set E_A per group          */
+  int32_t *expert_count;  /* [E + n_shared] slots per expert                               */
+  int32_t *expert_offset; /* [E + n_shared + 1] exclusive prefix sum of expert_count       */
+  int32_t *perm;          /* [T*(k+n_shared)] slot ids grouped by expert (ascending expert,
+                             ascending slot id inside); unused tail -1                    */
+  int32_t *active;        /* [E + n_shared] ascending ids of experts with count > 0        */
+  int32_t *n_active;      /* [1] size of the activated set (the layer's APF, Table 1)      */
+  int32_t *n_rows_active; /* [1] rows computed this step                                   */
+} team_routing;
+
+/* Create / destroy a context.  team_create allocates the context's device
+ * workspace (a few MB at max_rows = 1024) on the current device.
+ * Errors: TEAM_ERR_ARG, TEAM_ERR_SHAPE, TEAM_ERR_CUDA. */
+int team_create(const team_config *cfg, team_ctx **out);
+int team_destroy(team_ctx *ctx);
+
+/* Borrow the layer's weights (device pointers, 16-byte aligned; bf16 expert
+ * weights 128-byte aligned).  Builds the TMA descriptors for the bf16 path.
+ * May be called again to switch layers; a switch is stream-ordered by the
+ * caller (descriptors are passed by value at launch). */
+int team_set_weights(team_ctx *ctx, const team_weights *w);
+
+/* Change flags / tau_hot / L_hot / hot_dist_inclusive / prefix_decoded /
+ * norm_topk of an existing context (shapes and dtype must be unchanged). */
+int team_set_policy(team_ctx *ctx, const team_config *cfg);
+
+/* Router (Algorithm 1 "Router", Sec. 4.1 row selection): logits = x W_r^T in
+ * fp32 for every computed row, softmax over all experts, plain top-k with
+ * renormalised weights and the decision margin.  x: [T, H] row-major, dtype per
+ * config.  Logits stay in the context for team_select_experts. */
+int team_route(team_ctx *ctx, const void *x, const team_step_state *st, team_routing *out, void *stream);
+
+/* TEAM selection (Eq. 4, Algorithm 1 steps 1-3) and dispatch tables, from the
+ * logits left by the preceding team_route on the same context, stream and rows. */
+int team_select_experts(team_ctx *ctx, const team_step_state *st, team_routing *out, void *stream);
+
+/* The whole layer step: route, select, dispatch, SwiGLU experts, weighted
+ * combine.  y: fp32 [T, H]; rows with class TEAM_CLS_SKIP are left untouched
+ * (they keep the previous step's output), all other rows are overwritten.
+ * `out` may be NULL. */
+int team_moe_forward(team_ctx *ctx, const void *x, const team_step_state *st, team_routing *out,
+                     float *y, void *stream);
+
+/* Stack glue for a MoE-only multi-layer model: x[t,:] <- x[t,:] + y[t,:] for
+ * every row computed by the preceding team_moe_forward (fp32 add, stored in
+ * x's dtype, round to nearest even). */
+int team_residual_add(team_ctx *ctx, void *x, const float *y, int32_t n_rows, void *stream);
+
+/* Synchronise `stream` and return the device status word (TEAM_OK or the first
+ * TEAM_ERR_TIMEOUT / TEAM_ERR_STATE recorded since the last read; reading
+ * clears it).  detail_out (optional, host) receives a kernel-specific code. */
+int team_read_status(team_ctx *ctx, void *stream, int32_t *detail_out);
+
+/* Number of kernels the last compute call on this context launched. */
+int team_last_launch_count(const team_ctx *ctx);
+
+/* Average device time (ms) of the expert kernel over the launches made since
+ * the counters were last reset, measured with CUDA events on the launching
+ * stream when timing is enabled.  Synchronises the stream. */
+int team_expert_timing(team_ctx *ctx, int32_t enable, void *stream, float *avg_ms_out, int32_t *launches_out);
+
+const char *team_strerror(int code);
+const char *team_last_cuda_error(const team_ctx *ctx);
+int team_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TEAM_H_ */
