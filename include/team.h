@@ -75,17 +75,18 @@ enum { TEAM_DTYPE_F32 = 0, TEAM_DTYPE_BF16 = 1 };
 #define TEAM_MAX_EXPERTS 256   /* routed experts                       */
 #define TEAM_MAX_TOPK 16
 #define TEAM_MAX_SHARED 4
-#define TEAM_MAX_ROWS 4096     /* rows per call                        */
+#define TEAM_MAX_ROWS 2048     /* rows per call                        */
+#define TEAM_MAX_GROUPS 1024
 #define TEAM_MAX_BLOCK 64      /* rows of one (group, branch)          */
 
 typedef struct {
-  int32_t hidden;      /* H; multiple of 64 for bf16, of 4 for fp32                      */
-  int32_t n_experts;   /* E routed experts, multiple of 32, <= TEAM_MAX_EXPERTS (fp32 path: any E >= top_k) */
+  int32_t hidden;      /* H; multiple of 128 for bf16, of 4 for fp32                     */
+  int32_t n_experts;   /* E routed experts, top_k <= E <= TEAM_MAX_EXPERTS               */
   int32_t top_k;       /* k <= min(E, TEAM_MAX_TOPK)                                    */
   int32_t inter;       /* I; multiple of 64 for bf16, of 4 for fp32                      */
   int32_t n_shared;    /* always-on experts appended after the routed ones              */
   int32_t max_rows;    /* largest n_rows of any call on this context                    */
-  int32_t max_groups;  /* group ids are in [0, max_groups)                              */
+  int32_t max_groups;  /* group ids are in [0, max_groups), <= TEAM_MAX_GROUPS; branch ids in [0, 256) */
   int32_t dtype;       /* TEAM_DTYPE_F32: x and expert weights fp32 (plain FMA kernels);
                           TEAM_DTYPE_BF16: x and expert weights bf16, fp32 accumulation
                           on tensor cores.  Router weights and y are fp32 in both.      */
@@ -184,6 +185,11 @@ int team_last_launch_count(const team_ctx *ctx);
  * the counters were last reset, measured with CUDA events on the launching
  * stream when timing is enabled.  Synchronises the stream. */
 int team_expert_timing(team_ctx *ctx, int32_t enable, void *stream, float *avg_ms_out, int32_t *launches_out);
+
+/* Diagnostic: run the expert FFNs of a bf16 context through the plain-FMA
+ * kernels instead of the tensor-core kernel (allocates scratch on first use).
+ * Meant for triage of a parity failure, not for production. */
+int team_debug_force_simt(team_ctx *ctx, int on);
 
 const char *team_strerror(int code);
 const char *team_last_cuda_error(const team_ctx *ctx);

@@ -1,0 +1,382 @@
+// C ABI of the TEAM MoE-layer library: context, argument checks, kernel launch sequences.
+#include <cuda.h>
+
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "team_common.cuh"
+
+namespace team {
+int make_weight_map(void* out_map, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows);
+cudaError_t launch_experts_tc(const void* maps, int item_tile, const void* x, Workspace ws, float* y, Dims d,
+                              int grid, cudaStream_t s);
+}  // namespace team
+
+struct team_ctx {
+  team_config cfg;
+  team::Workspace ws;
+  void* ws_base;
+  size_t ws_bytes;
+  team_weights w;
+  bool has_weights;
+  alignas(64) CUtensorMap maps[3];
+  int device;
+  int n_sms;
+  int item_tile;
+  int last_launches;
+  int force_simt;
+  void* simt_act;   // diagnostic fp32-FMA path on bf16 weights: activation scratch
+  char cuda_err[256];
+  // expert-kernel timing
+  bool timing;
+  std::vector<cudaEvent_t> ev;   // pairs
+  size_t ev_used;
+};
+
+namespace {
+
+int fail_cuda(team_ctx* ctx, cudaError_t e, const char* what) {
+  if (ctx) snprintf(ctx->cuda_err, sizeof(ctx->cuda_err), "%s: %s", what, cudaGetErrorString(e));
+  return TEAM_ERR_CUDA;
+}
+
+team::Dims dims_of(const team_config& c, int T) {
+  team::Dims d;
+  d.T = T; d.H = c.hidden; d.E = c.n_experts; d.k = c.top_k; d.I = c.inter; d.ns = c.n_shared; d.G = c.max_groups;
+  return d;
+}
+
+team::Policy policy_of(const team_config& c) {
+  team::Policy p;
+  p.flags = c.flags; p.tau_hot = c.tau_hot; p.L_hot = c.L_hot; p.inclusive = c.hot_dist_inclusive;
+  p.prefix_decoded = c.prefix_decoded; p.norm_topk = c.norm_topk;
+  return p;
+}
+
+int check_config(const team_config* c) {
+  if (c == nullptr) return TEAM_ERR_ARG;
+  if (c->hidden <= 0 || c->n_experts <= 0 || c->top_k <= 0 || c->inter <= 0 || c->n_shared < 0) return TEAM_ERR_SHAPE;
+  if (c->n_experts > TEAM_MAX_EXPERTS || c->top_k > TEAM_MAX_TOPK || c->top_k > c->n_experts) return TEAM_ERR_SHAPE;
+  if (c->n_shared > TEAM_MAX_SHARED) return TEAM_ERR_SHAPE;
+  if (c->max_rows <= 0 || c->max_rows > TEAM_MAX_ROWS) return TEAM_ERR_SHAPE;
+  if (c->max_groups <= 0 || c->max_groups > TEAM_MAX_GROUPS) return TEAM_ERR_SHAPE;
+  if (c->dtype == TEAM_DTYPE_F32) {
+    if (c->hidden % 4 || c->inter % 4) return TEAM_ERR_SHAPE;
+  } else if (c->dtype == TEAM_DTYPE_BF16) {
+    if (c->hidden % 128 || c->inter % 64) return TEAM_ERR_SHAPE;
+  } else {
+    return TEAM_ERR_SHAPE;
+  }
+  if (c->L_hot < 0) return TEAM_ERR_ARG;
+  return TEAM_OK;
+}
+
+int check_state(const team_ctx* ctx, const team_step_state* st) {
+  if (ctx == nullptr || st == nullptr) return TEAM_ERR_ARG;
+  if (st->n_rows < 1 || st->n_rows > ctx->cfg.max_rows) return TEAM_ERR_ARG;
+  if (!st->tok_state || !st->conf || !st->pos || !st->group || !st->branch) return TEAM_ERR_ARG;
+  return TEAM_OK;
+}
+
+team::StepPtrs step_ptrs(const team_step_state* st) {
+  team::StepPtrs s;
+  s.tok_state = st->tok_state; s.conf = st->conf; s.pos = st->pos; s.group = st->group; s.branch = st->branch;
+  return s;
+}
+
+team::RoutePtrs export_ptrs(const team_routing* r) {
+  team::RoutePtrs e;
+  memset(&e, 0, sizeof(e));
+  if (r == nullptr) return e;
+  e.probs = r->probs; e.topk_idx = r->topk_idx; e.topk_w = r->topk_w; e.margin = r->margin;
+  e.tok_class = r->tok_class; e.group_mask = r->group_mask; e.expert_count = r->expert_count;
+  e.expert_offset = r->expert_offset; e.perm = r->perm; e.active = r->active; e.n_active = r->n_active;
+  e.n_rows_active = r->n_rows_active;
+  return e;
+}
+
+bool use_tensor_path(const team_ctx* ctx) { return ctx->cfg.dtype == TEAM_DTYPE_BF16 && !ctx->force_simt; }
+
+int pick_item_tile(const team_config& c) {
+  const char* env = getenv("TEAM_ITEM_TILE");
+  if (env != nullptr) {
+    const int v = atoi(env);
+    if (v == 32 || v == 64 || v == 128) return v;
+  }
+  if (c.max_rows <= 64) return 32;
+  if (c.max_rows <= 256) return 64;
+  return 128;
+}
+
+}  // namespace
+
+extern "C" {
+
+int team_version(void) { return 1; }
+
+const char* team_strerror(int code) {
+  switch (code) {
+    case TEAM_OK: return "ok";
+    case TEAM_ERR_ARG: return "invalid argument";
+    case TEAM_ERR_SHAPE: return "unsupported shape or configuration";
+    case TEAM_ERR_CUDA: return "CUDA error";
+    case TEAM_ERR_TIMEOUT: return "device wait expired";
+    case TEAM_ERR_STATE: return "row layout contract broken or index out of range";
+    default: return "unknown error";
+  }
+}
+
+const char* team_last_cuda_error(const team_ctx* ctx) { return ctx ? ctx->cuda_err : ""; }
+
+int team_create(const team_config* cfg, team_ctx** out) {
+  if (out == nullptr) return TEAM_ERR_ARG;
+  *out = nullptr;
+  int rc = check_config(cfg);
+  if (rc != TEAM_OK) return rc;
+  int ndev = 0;
+  if (cudaGetDeviceCount(&ndev) != cudaSuccess || ndev == 0) {
+    cudaGetLastError();
+    return TEAM_ERR_CUDA;
+  }
+  team_ctx* ctx = new (std::nothrow) team_ctx();
+  if (ctx == nullptr) return TEAM_ERR_ARG;
+  ctx->cfg = *cfg;
+  ctx->has_weights = false;
+  ctx->last_launches = 0;
+  ctx->force_simt = 0;
+  ctx->simt_act = nullptr;
+  ctx->cuda_err[0] = 0;
+  ctx->timing = false;
+  ctx->ev_used = 0;
+  cudaError_t e = cudaGetDevice(&ctx->device);
+  if (e == cudaSuccess) e = cudaDeviceGetAttribute(&ctx->n_sms, cudaDevAttrMultiProcessorCount, ctx->device);
+  if (e != cudaSuccess) {
+    delete ctx;
+    return TEAM_ERR_CUDA;
+  }
+  ctx->item_tile = pick_item_tile(*cfg);
+
+  const size_t T = cfg->max_rows, E = cfg->n_experts, k = cfg->top_k, ns = cfg->n_shared, EN = E + ns;
+  const size_t S = T * (k + ns);
+  size_t off = 0;
+  auto take = [&](size_t bytes) {
+    size_t at = off;
+    off += (bytes + 255) & ~size_t(255);
+    return at;
+  };
+  const size_t o_logits = take(T * E * 4), o_idx = take(T * k * 4), o_w = take(T * k * 4), o_margin = take(T * 4);
+  const size_t o_cls = take(T), o_gm = take((size_t)cfg->max_groups * ((E + 63) / 64) * 8);
+  const size_t o_cnt = take(EN * 4), o_off = take((EN + 1) * 4), o_perm = take(S * 4), o_act_list = take(EN * 4);
+  const size_t o_scal = take(64), o_items = take((EN + S / 32 + 2) * sizeof(team::WorkItem));
+  const size_t o_act = take(cfg->dtype == TEAM_DTYPE_F32 ? S * cfg->inter * 4 : 256);
+  ctx->ws_bytes = off;
+  e = cudaMalloc(&ctx->ws_base, ctx->ws_bytes);
+  if (e != cudaSuccess) {
+    delete ctx;
+    return TEAM_ERR_CUDA;
+  }
+  cudaMemset(ctx->ws_base, 0, ctx->ws_bytes);
+  unsigned char* b = static_cast<unsigned char*>(ctx->ws_base);
+  team::Workspace& ws = ctx->ws;
+  ws.logits = reinterpret_cast<float*>(b + o_logits);
+  ws.r.probs = nullptr;
+  ws.r.topk_idx = reinterpret_cast<int32_t*>(b + o_idx);
+  ws.r.topk_w = reinterpret_cast<float*>(b + o_w);
+  ws.r.margin = reinterpret_cast<float*>(b + o_margin);
+  ws.r.tok_class = b + o_cls;
+  ws.r.group_mask = reinterpret_cast<uint64_t*>(b + o_gm);
+  ws.r.expert_count = reinterpret_cast<int32_t*>(b + o_cnt);
+  ws.r.expert_offset = reinterpret_cast<int32_t*>(b + o_off);
+  ws.r.perm = reinterpret_cast<int32_t*>(b + o_perm);
+  ws.r.active = reinterpret_cast<int32_t*>(b + o_act_list);
+  int32_t* scal = reinterpret_cast<int32_t*>(b + o_scal);
+  ws.r.n_active = scal + 0;
+  ws.r.n_rows_active = scal + 1;
+  ws.n_items = scal + 2;
+  ws.status = scal + 4;
+  ws.items = reinterpret_cast<team::WorkItem*>(b + o_items);
+  ws.act = reinterpret_cast<float*>(b + o_act);
+  *out = ctx;
+  return TEAM_OK;
+}
+
+int team_destroy(team_ctx* ctx) {
+  if (ctx == nullptr) return TEAM_ERR_ARG;
+  for (cudaEvent_t e : ctx->ev) cudaEventDestroy(e);
+  cudaFree(ctx->ws_base);
+  if (ctx->simt_act) cudaFree(ctx->simt_act);
+  delete ctx;
+  return TEAM_OK;
+}
+
+int team_set_weights(team_ctx* ctx, const team_weights* w) {
+  if (ctx == nullptr || w == nullptr) return TEAM_ERR_ARG;
+  if (!w->w_router || !w->w_gate || !w->w_up || !w->w_down) return TEAM_ERR_ARG;
+  const uintptr_t align = ctx->cfg.dtype == TEAM_DTYPE_BF16 ? 127 : 15;
+  if (((uintptr_t)w->w_router & 15) || ((uintptr_t)w->w_gate & align) || ((uintptr_t)w->w_up & align) ||
+      ((uintptr_t)w->w_down & align))
+    return TEAM_ERR_ARG;
+  if (ctx->cfg.dtype == TEAM_DTYPE_BF16) {
+    const uint64_t EN = ctx->cfg.n_experts + ctx->cfg.n_shared, I = ctx->cfg.inter, H = ctx->cfg.hidden;
+    int r = team::make_weight_map(&ctx->maps[0], w->w_gate, EN * I, H, 16);
+    if (r == 0) r = team::make_weight_map(&ctx->maps[1], w->w_up, EN * I, H, 16);
+    if (r == 0) r = team::make_weight_map(&ctx->maps[2], w->w_down, EN * H, I, 128);
+    if (r != 0) {
+      snprintf(ctx->cuda_err, sizeof(ctx->cuda_err), "cuTensorMapEncodeTiled failed (%d)", r);
+      return TEAM_ERR_CUDA;
+    }
+  }
+  ctx->w = *w;
+  ctx->has_weights = true;
+  return TEAM_OK;
+}
+
+int team_set_policy(team_ctx* ctx, const team_config* cfg) {
+  if (ctx == nullptr || cfg == nullptr) return TEAM_ERR_ARG;
+  const team_config& c = ctx->cfg;
+  if (cfg->hidden != c.hidden || cfg->n_experts != c.n_experts || cfg->top_k != c.top_k || cfg->inter != c.inter ||
+      cfg->n_shared != c.n_shared || cfg->max_rows != c.max_rows || cfg->max_groups != c.max_groups ||
+      cfg->dtype != c.dtype)
+    return TEAM_ERR_SHAPE;
+  if (cfg->L_hot < 0) return TEAM_ERR_ARG;
+  ctx->cfg = *cfg;
+  return TEAM_OK;
+}
+
+int team_debug_force_simt(team_ctx* ctx, int on) {
+  if (ctx == nullptr) return TEAM_ERR_ARG;
+  if (on && ctx->cfg.dtype == TEAM_DTYPE_BF16 && ctx->simt_act == nullptr) {
+    const size_t S = (size_t)ctx->cfg.max_rows * (ctx->cfg.top_k + ctx->cfg.n_shared);
+    cudaError_t e = cudaMalloc(&ctx->simt_act, S * ctx->cfg.inter * 4);
+    if (e != cudaSuccess) return fail_cuda(ctx, e, "diagnostic scratch");
+    ctx->ws.act = static_cast<float*>(ctx->simt_act);
+  }
+  ctx->force_simt = on;
+  return TEAM_OK;
+}
+
+int team_route(team_ctx* ctx, const void* x, const team_step_state* st, team_routing* out, void* stream) {
+  int rc = check_state(ctx, st);
+  if (rc != TEAM_OK) return rc;
+  if (x == nullptr || out == nullptr || !ctx->has_weights) return TEAM_ERR_ARG;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const team::Dims d = dims_of(ctx->cfg, st->n_rows);
+  ctx->last_launches = 0;
+  cudaError_t e = team::launch_router_logits(x, ctx->cfg.dtype, static_cast<const float*>(ctx->w.w_router),
+                                             st->tok_state, ctx->ws.logits, nullptr, d, ctx->cfg.flags, s);
+  if (e != cudaSuccess) return fail_cuda(ctx, e, "router logits");
+  ++ctx->last_launches;
+  e = team::launch_router_topk(ctx->ws.logits, st->tok_state, export_ptrs(out), d, policy_of(ctx->cfg), s);
+  if (e != cudaSuccess) return fail_cuda(ctx, e, "router top-k");
+  ++ctx->last_launches;
+  return TEAM_OK;
+}
+
+int team_select_experts(team_ctx* ctx, const team_step_state* st, team_routing* out, void* stream) {
+  int rc = check_state(ctx, st);
+  if (rc != TEAM_OK) return rc;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const team::Dims d = dims_of(ctx->cfg, st->n_rows);
+  ctx->last_launches = 0;
+  cudaError_t e = team::launch_select(ctx->ws.logits, step_ptrs(st), ctx->ws, export_ptrs(out), d,
+                                      policy_of(ctx->cfg), ctx->item_tile, s);
+  if (e != cudaSuccess) return fail_cuda(ctx, e, "select");
+  ++ctx->last_launches;
+  return TEAM_OK;
+}
+
+int team_moe_forward(team_ctx* ctx, const void* x, const team_step_state* st, team_routing* out, float* y,
+                     void* stream) {
+  int rc = check_state(ctx, st);
+  if (rc != TEAM_OK) return rc;
+  if (x == nullptr || y == nullptr || !ctx->has_weights) return TEAM_ERR_ARG;
+  if (((uintptr_t)x & 15) || ((uintptr_t)y & 15)) return TEAM_ERR_ARG;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const team::Dims d = dims_of(ctx->cfg, st->n_rows);
+  const bool tc = use_tensor_path(ctx);
+  ctx->last_launches = 0;
+  cudaError_t e = team::launch_router_logits(x, ctx->cfg.dtype, static_cast<const float*>(ctx->w.w_router),
+                                             st->tok_state, ctx->ws.logits, tc ? y : nullptr, d, ctx->cfg.flags, s);
+  if (e != cudaSuccess) return fail_cuda(ctx, e, "router logits");
+  ++ctx->last_launches;
+  e = team::launch_select(ctx->ws.logits, step_ptrs(st), ctx->ws, export_ptrs(out), d, policy_of(ctx->cfg),
+                          ctx->item_tile, s);
+  if (e != cudaSuccess) return fail_cuda(ctx, e, "select");
+  ++ctx->last_launches;
+  cudaEvent_t ev0 = nullptr, ev1 = nullptr;
+  if (ctx->timing) {
+    if (ctx->ev_used + 2 > ctx->ev.size()) {
+      for (int i = 0; i < 2; ++i) {
+        cudaEvent_t ne;
+        if ((e = cudaEventCreate(&ne)) != cudaSuccess) return fail_cuda(ctx, e, "event create");
+        ctx->ev.push_back(ne);
+      }
+    }
+    ev0 = ctx->ev[ctx->ev_used];
+    ev1 = ctx->ev[ctx->ev_used + 1];
+    ctx->ev_used += 2;
+    cudaEventRecord(ev0, s);
+  }
+  if (tc) {
+    const int EN = d.E + d.ns;
+    long max_work = ((long)EN + (long)d.T * (d.k + d.ns) / ctx->item_tile) * (d.I / 64);
+    int grid = (int)(max_work < ctx->n_sms ? max_work : ctx->n_sms);
+    e = team::launch_experts_tc(ctx->maps, ctx->item_tile, x, ctx->ws, y, d, grid, s);
+    if (e != cudaSuccess) return fail_cuda(ctx, e, "expert kernel");
+    ++ctx->last_launches;
+  } else {
+    e = team::launch_experts_simt(x, ctx->cfg.dtype, ctx->w.w_gate, ctx->w.w_up, ctx->w.w_down, ctx->ws, y, d, s);
+    if (e != cudaSuccess) return fail_cuda(ctx, e, "expert kernels (fp32)");
+    ctx->last_launches += 2;
+  }
+  if (ev1) cudaEventRecord(ev1, s);
+  return TEAM_OK;
+}
+
+int team_residual_add(team_ctx* ctx, void* x, const float* y, int32_t n_rows, void* stream) {
+  if (ctx == nullptr || x == nullptr || y == nullptr || n_rows < 1 || n_rows > ctx->cfg.max_rows) return TEAM_ERR_ARG;
+  cudaError_t e = team::launch_residual_add(x, ctx->cfg.dtype, y, ctx->ws.r.tok_class, n_rows, ctx->cfg.hidden,
+                                            static_cast<cudaStream_t>(stream));
+  if (e != cudaSuccess) return fail_cuda(ctx, e, "residual add");
+  ctx->last_launches = 1;
+  return TEAM_OK;
+}
+
+int team_read_status(team_ctx* ctx, void* stream, int32_t* detail_out) {
+  if (ctx == nullptr) return TEAM_ERR_ARG;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  int32_t host[2] = {0, 0};
+  cudaError_t e = cudaMemcpyAsync(host, ctx->ws.status, sizeof(host), cudaMemcpyDeviceToHost, s);
+  if (e == cudaSuccess) e = cudaMemsetAsync(ctx->ws.status, 0, sizeof(host), s);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+  if (e != cudaSuccess) return fail_cuda(ctx, e, "read status");
+  if (detail_out) *detail_out = host[1];
+  return host[0];
+}
+
+int team_last_launch_count(const team_ctx* ctx) { return ctx ? ctx->last_launches : 0; }
+
+int team_expert_timing(team_ctx* ctx, int32_t enable, void* stream, float* avg_ms_out, int32_t* launches_out) {
+  if (ctx == nullptr) return TEAM_ERR_ARG;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  cudaError_t e = cudaStreamSynchronize(s);
+  if (e != cudaSuccess) return fail_cuda(ctx, e, "timing sync");
+  double total = 0.0;
+  const int n = (int)(ctx->ev_used / 2);
+  for (int i = 0; i < n; ++i) {
+    float ms = 0.f;
+    if ((e = cudaEventElapsedTime(&ms, ctx->ev[2 * i], ctx->ev[2 * i + 1])) != cudaSuccess)
+      return fail_cuda(ctx, e, "event elapsed");
+    total += ms;
+  }
+  if (avg_ms_out) *avg_ms_out = n > 0 ? (float)(total / n) : 0.f;
+  if (launches_out) *launches_out = n;
+  ctx->ev_used = 0;
+  ctx->timing = enable != 0;
+  return TEAM_OK;
+}
+
+}  // extern "C"

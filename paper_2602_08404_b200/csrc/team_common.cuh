@@ -1,0 +1,106 @@
+// Shared declarations of the TEAM MoE-layer kernels (device-side structs, small helpers).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "team.h"
+
+namespace team {
+
+// Shapes of one call.
+struct Dims {
+  int T;   // rows presented
+  int H;   // hidden
+  int E;   // routed experts
+  int k;   // top-k
+  int I;   // expert intermediate
+  int ns;  // shared experts
+  int G;   // max groups
+};
+
+// Eq. 4 / Algorithm 1 policy knobs.
+struct Policy {
+  int flags;
+  float tau_hot;
+  int L_hot;
+  int inclusive;
+  int prefix_decoded;
+  int norm_topk;
+};
+
+// Previous-step state (device pointers).
+struct StepPtrs {
+  const uint8_t* tok_state;
+  const float* conf;
+  const int32_t* pos;
+  const int32_t* group;
+  const int32_t* branch;
+};
+
+// Routing tables.  `ws` pointers are never null; `ex` (caller exports) may be.
+struct RoutePtrs {
+  float* probs;
+  int32_t* topk_idx;
+  float* topk_w;
+  float* margin;
+  uint8_t* tok_class;
+  uint64_t* group_mask;
+  int32_t* expert_count;
+  int32_t* expert_offset;
+  int32_t* perm;
+  int32_t* active;
+  int32_t* n_active;
+  int32_t* n_rows_active;
+};
+
+// One unit of expert work: `n` consecutive entries of perm starting at `begin`, all of expert `e`.
+struct WorkItem {
+  int32_t e;
+  int32_t begin;
+  int32_t n;
+  int32_t pad;
+};
+
+struct Workspace {
+  float* logits;        // [max_rows, E]
+  RoutePtrs r;          // context-owned routing tables (probs is null here)
+  WorkItem* items;      // [E + ns + max_rows*(k+ns)/tile + 1]
+  int32_t* n_items;     // [1]
+  float* act;           // fp32 path: [max_rows*(k+ns), I] SwiGLU activations
+  int32_t* status;      // [2] code, detail
+};
+
+__device__ __forceinline__ void set_status(int32_t* status, int code, int detail) {
+  if (atomicCAS(status, 0, code) == 0) status[1] = detail;
+}
+
+__device__ __forceinline__ float to_f32(float v) { return v; }
+__device__ __forceinline__ float to_f32(__nv_bfloat16 v) { return __bfloat162float(v); }
+
+// Row and combine weight of a slot id (routed: t*k+j, shared: T*k + s*T + t).
+__device__ __forceinline__ void slot_row_weight(int slot, int T, int k, const float* topk_w, int& row, float& w) {
+  if (slot < T * k) {
+    row = slot / k;
+    w = topk_w[slot];
+  } else {
+    row = (slot - T * k) % T;
+    w = 1.0f;
+  }
+}
+
+// Kernel launchers (host side), one per translation unit.
+cudaError_t launch_router_logits(const void* x, int dtype, const float* w_router, const uint8_t* tok_state,
+                                 float* logits, float* y_zero, Dims d, int flags, cudaStream_t s);
+cudaError_t launch_router_topk(const float* logits, const uint8_t* tok_state, RoutePtrs out, Dims d, Policy p,
+                               cudaStream_t s);
+cudaError_t launch_select(const float* logits, StepPtrs st, Workspace ws, RoutePtrs ex, Dims d, Policy p,
+                          int item_tile, cudaStream_t s);
+size_t select_smem_bytes(Dims d);
+cudaError_t launch_experts_simt(const void* x, int dtype, const void* w_gate, const void* w_up, const void* w_down,
+                                Workspace ws, float* y, Dims d, cudaStream_t s);
+cudaError_t launch_residual_add(void* x, int dtype, const float* y, const uint8_t* tok_class, int T, int H,
+                                cudaStream_t s);
+
+}  // namespace team

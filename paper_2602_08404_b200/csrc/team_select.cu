@@ -1,0 +1,357 @@
+// Selection / permutation kernel: Eq. 4 classification, Algorithm 1's two routing rounds, the
+// necessary expert set E_A per group, and the dispatch tables (per-expert counts, exclusive
+// offsets, the expert-sorted slot permutation, the active-expert list and the expert kernel's
+// work items).  One CTA of 1024 threads; all cross-row state (group masks, histograms, scans)
+// lives in shared memory.
+//
+// Layout contract: rows with equal (group, branch) are contiguous (one decoding block, at most
+// TEAM_MAX_BLOCK rows), so the "distance to a decoded token" test of Eq. 4 only walks a row's own run.
+#include "team_common.cuh"
+#include "team_topk.cuh"
+
+namespace team {
+
+constexpr int kSelThreads = 1024;
+constexpr int kSelWarps = kSelThreads / 32;
+
+struct SelSmem {
+  // carved from dynamic shared memory in this order
+  uint32_t* mask;      // [G][8]  E_A bits (256 experts max)
+  int32_t* hist;       // [kSelWarps][E+ns]
+  int32_t* off;        // [E+ns+1]
+  int32_t* key;        // [T] group*256 + branch
+  int32_t* pos;        // [T]
+  int32_t* warp_cnt;   // [kSelWarps + 1]
+  uint8_t* state;      // [T]
+  uint8_t* cls;        // [T]
+  uint8_t* has_first;  // [G]
+};
+
+__host__ __device__ inline size_t sel_smem_layout(Dims d, SelSmem* s, unsigned char* base) {
+  size_t o = 0;
+  auto take = [&](size_t bytes) {
+    size_t at = o;
+    o += (bytes + 15) & ~size_t(15);
+    return at;
+  };
+  const int EN = d.E + d.ns;
+  size_t a_mask = take((size_t)d.G * 8 * 4);
+  size_t a_hist = take((size_t)kSelWarps * EN * 4);
+  size_t a_off = take((size_t)(EN + 1) * 4);
+  size_t a_key = take((size_t)d.T * 4);
+  size_t a_pos = take((size_t)d.T * 4);
+  size_t a_wc = take((size_t)(kSelWarps + 1) * 4);
+  size_t a_state = take((size_t)d.T);
+  size_t a_cls = take((size_t)d.T);
+  size_t a_hf = take((size_t)d.G);
+  if (s != nullptr) {
+    s->mask = reinterpret_cast<uint32_t*>(base + a_mask);
+    s->hist = reinterpret_cast<int32_t*>(base + a_hist);
+    s->off = reinterpret_cast<int32_t*>(base + a_off);
+    s->key = reinterpret_cast<int32_t*>(base + a_key);
+    s->pos = reinterpret_cast<int32_t*>(base + a_pos);
+    s->warp_cnt = reinterpret_cast<int32_t*>(base + a_wc);
+    s->state = base + a_state;
+    s->cls = base + a_cls;
+    s->has_first = base + a_hf;
+  }
+  return o;
+}
+
+size_t select_smem_bytes(Dims d) { return sel_smem_layout(d, nullptr, nullptr); }
+
+__device__ __forceinline__ bool is_decoded(uint8_t s) { return s == TEAM_TOK_NEW || s == TEAM_TOK_CACHED; }
+
+__global__ void __launch_bounds__(kSelThreads, 1)
+k_select(const float* __restrict__ logits, StepPtrs st, Workspace ws, RoutePtrs ex, Dims d, Policy p, int item_tile) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  SelSmem s;
+  sel_smem_layout(d, &s, smem_raw);
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int T = d.T, E = d.E, k = d.k, ns = d.ns, EN = d.E + d.ns;
+  const int n_words32 = 8;
+  RoutePtrs& r = ws.r;
+
+  // ---- stage the step state ------------------------------------------------------------
+  for (int i = tid; i < d.G * n_words32; i += kSelThreads) s.mask[i] = 0u;
+  for (int i = tid; i < d.G; i += kSelThreads) s.has_first[i] = 0;
+  for (int i = tid; i < kSelWarps * EN; i += kSelThreads) s.hist[i] = 0;
+  for (int t = tid; t < T; t += kSelThreads) {
+    int g = st.group[t], b = st.branch[t];
+    if (g < 0 || g >= d.G || b < 0 || b > 255) {
+      set_status(ws.status, TEAM_ERR_STATE, 1);
+      g = min(max(g, 0), d.G - 1);
+      b = min(max(b, 0), 255);
+    }
+    s.key[t] = g * 256 + b;
+    s.pos[t] = st.pos[t];
+    s.state[t] = st.tok_state[t];
+  }
+  __syncthreads();
+
+  // ---- Eq. 4: classification --------------------------------------------------------------
+  for (int t = tid; t < T; t += kSelThreads) {
+    const uint8_t state = s.state[t];
+    uint8_t c;
+    if (state == TEAM_TOK_CACHED) {
+      c = (p.flags & TEAM_F_DCD) ? TEAM_CLS_SKIP : TEAM_CLS_FIRST;
+    } else if (state == TEAM_TOK_NEW || !(p.flags & TEAM_F_LAC)) {
+      c = TEAM_CLS_FIRST;
+    } else {
+      const int key = s.key[t], mypos = s.pos[t];
+      const int lim = p.inclusive ? p.L_hot : p.L_hot - 1;   // |pos - j| <= lim
+      bool hot = st.conf[t] > p.tau_hot;
+      if (p.prefix_decoded && mypos + 1 <= lim) hot = true;
+      for (int u = t - 1; !hot && u >= 0 && s.key[u] == key; --u) {
+        if (t - u > TEAM_MAX_BLOCK) { set_status(ws.status, TEAM_ERR_STATE, 2); break; }
+        if (is_decoded(s.state[u]) && abs(mypos - s.pos[u]) <= lim) hot = true;
+      }
+      for (int u = t + 1; !hot && u < T && s.key[u] == key; ++u) {
+        if (u - t > TEAM_MAX_BLOCK) { set_status(ws.status, TEAM_ERR_STATE, 2); break; }
+        if (is_decoded(s.state[u]) && abs(mypos - s.pos[u]) <= lim) hot = true;
+      }
+      c = hot ? TEAM_CLS_FIRST : TEAM_CLS_COLD;
+    }
+    s.cls[t] = c;
+    if (c == TEAM_CLS_FIRST) s.has_first[s.key[t] >> 8] = 1;
+  }
+  __syncthreads();
+  // A group with no first-round row: its masked rows are all routed freely.
+  for (int t = tid; t < T; t += kSelThreads)
+    if (s.cls[t] == TEAM_CLS_COLD && !s.has_first[s.key[t] >> 8]) s.cls[t] = TEAM_CLS_FIRST;
+  __syncthreads();
+
+  // ---- Algorithm 1, round 1 (free top-k) then round 2 (top-k inside E_A) -------------------
+  for (int round = 1; round <= 2; ++round) {
+    for (int t = warp; t < T; t += kSelWarps) {
+      const uint8_t c = s.cls[t];
+      if (round == 1 && c == TEAM_CLS_SKIP) {
+        if (lane < k) {
+          r.topk_idx[t * k + lane] = -1;
+          r.topk_w[t * k + lane] = 0.f;
+          if (ex.topk_idx) ex.topk_idx[t * k + lane] = -1;
+          if (ex.topk_w) ex.topk_w[t * k + lane] = 0.f;
+        }
+        if (lane == 0) {
+          r.margin[t] = __builtin_huge_valf();
+          if (ex.margin) ex.margin[t] = __builtin_huge_valf();
+        }
+        if (ex.probs)
+          for (int e = lane; e < E; e += 32) ex.probs[(size_t)t * E + e] = 0.f;
+        continue;
+      }
+      if ((round == 1 && c != TEAM_CLS_FIRST) || (round == 2 && c != TEAM_CLS_COLD)) continue;
+      const int g = s.key[t] >> 8;
+      float v[kMaxPerLane];
+      float row_max, denom;
+      load_row(logits + (size_t)t * E, E, lane, v, row_max, denom);
+      if (ex.probs) {
+#pragma unroll
+        for (int i = 0; i < kMaxPerLane; ++i) {
+          const int e = i * 32 + lane;
+          if (e < E) ex.probs[(size_t)t * E + e] = expf(v[i] - row_max) / denom;
+        }
+      }
+      if (round == 2) {
+#pragma unroll
+        for (int i = 0; i < kMaxPerLane; ++i)
+          if (!((s.mask[g * n_words32 + i] >> lane) & 1u)) v[i] = kNegInf;
+      }
+      TopkResult tr = warp_topk(v, k, lane);
+      const float w = routing_weight(tr, k, lane, row_max, denom, p.norm_topk);
+      if (lane < k) {
+        r.topk_idx[t * k + lane] = tr.idx;
+        r.topk_w[t * k + lane] = w;
+        if (ex.topk_idx) ex.topk_idx[t * k + lane] = tr.idx;
+        if (ex.topk_w) ex.topk_w[t * k + lane] = w;
+        if (tr.idx < 0) set_status(ws.status, TEAM_ERR_STATE, 3);
+        else if (round == 1) atomicOr(&s.mask[g * n_words32 + (tr.idx >> 5)], 1u << (tr.idx & 31));
+      }
+      if (lane == 0) {
+        r.margin[t] = tr.margin;
+        if (ex.margin) ex.margin[t] = tr.margin;
+      }
+    }
+    __syncthreads();
+  }
+
+  // ---- exports that need no further work ---------------------------------------------------
+  for (int t = tid; t < T; t += kSelThreads) {
+    r.tok_class[t] = s.cls[t];
+    if (ex.tok_class) ex.tok_class[t] = s.cls[t];
+  }
+  {
+    const int n_words64 = (E + 63) / 64;
+    for (int i = tid; i < d.G * n_words64; i += kSelThreads) {
+      const int g = i / n_words64, wd = i % n_words64;
+      const uint64_t m = (uint64_t)s.mask[g * n_words32 + 2 * wd] | ((uint64_t)s.mask[g * n_words32 + 2 * wd + 1] << 32);
+      r.group_mask[i] = m;
+      if (ex.group_mask) ex.group_mask[i] = m;
+    }
+  }
+
+  // ---- dispatch: stable counting sort of slots by expert ------------------------------------
+  // Routed slots t*k+j are walked in ascending order, warp w owning a contiguous range, so the
+  // rank of a slot inside its expert is (slots of that expert in earlier warps) + (earlier in this warp).
+  const int S = T * k;
+  const int per_warp = ((S + kSelWarps - 1) / kSelWarps + 31) & ~31;
+  const int lo = warp * per_warp, hi = min(S, lo + per_warp);
+  int32_t* my_hist = s.hist + warp * EN;
+  for (int base = lo; base < hi; base += 32) {
+    const int slot = base + lane;
+    const int e = (slot < hi) ? r.topk_idx[slot] : -1;
+    const unsigned peers = __match_any_sync(0xffffffffu, e);
+    if (e >= 0 && (__ffs(peers) - 1) == lane) my_hist[e] += __popc(peers);
+    __syncwarp();
+  }
+  // active rows (ascending) and their count; shared experts take every active row
+  int n_rows_active = 0;
+  {
+    int c = 0;
+    for (int base = warp * 32; base < T; base += kSelThreads) {
+      const int t = base + lane;
+      const bool a = t < T && s.cls[t] != TEAM_CLS_SKIP;
+      c += __popc(__ballot_sync(0xffffffffu, a));
+    }
+    // rows are dealt to warps in an interleaved way; only the total is needed here
+    if (lane == 0) s.warp_cnt[warp] = c;
+  }
+  __syncthreads();
+  for (int w = 0; w < kSelWarps; ++w) n_rows_active += s.warp_cnt[w];
+  // per expert: turn per-warp counts into per-warp starting ranks, total into off[e+1]
+  for (int e = tid; e < EN; e += kSelThreads) {
+    int run = 0;
+    if (e < E) {
+      for (int w = 0; w < kSelWarps; ++w) {
+        const int c = s.hist[w * EN + e];
+        s.hist[w * EN + e] = run;
+        run += c;
+      }
+    } else {
+      run = n_rows_active;
+    }
+    s.off[e + 1] = run;   // counts for now
+  }
+  if (tid == 0) s.off[0] = 0;
+  __syncthreads();
+  // exclusive scan over experts (EN <= 260) by warp 0; also active list and work items
+  if (warp == 0) {
+    int carry = 0, n_act = 0, n_items = 0;
+    for (int base = 0; base < EN; base += 32) {
+      const int e = base + lane;
+      const int c = (e < EN) ? s.off[e + 1] : 0;
+      int incl = c;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int n = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += n;
+      }
+      const int excl = carry + incl - c;
+      // active list
+      const unsigned act = __ballot_sync(0xffffffffu, c > 0);
+      const int arank = n_act + __popc(act & ((1u << lane) - 1));
+      // work items: ceil(c / item_tile) per expert
+      const int tiles = (c + item_tile - 1) / item_tile;
+      int tincl = tiles;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int n = __shfl_up_sync(0xffffffffu, tincl, o);
+        if (lane >= o) tincl += n;
+      }
+      const int tbase = n_items + tincl - tiles;
+      if (e < EN) {
+        r.expert_count[e] = c;
+        r.expert_offset[e] = excl;
+        if (ex.expert_count) ex.expert_count[e] = c;
+        if (ex.expert_offset) ex.expert_offset[e] = excl;
+        if (c > 0) {
+          r.active[arank] = e;
+          if (ex.active) ex.active[arank] = e;
+          for (int i = 0; i < tiles; ++i) {
+            WorkItem it;
+            it.e = e;
+            it.begin = excl + i * item_tile;
+            it.n = min(item_tile, c - i * item_tile);
+            it.pad = 0;
+            ws.items[tbase + i] = it;
+          }
+        }
+      }
+      __syncwarp();
+      if (e < EN) s.off[e] = excl;
+      carry += __shfl_sync(0xffffffffu, incl, 31);
+      n_act += __popc(act);
+      n_items += __shfl_sync(0xffffffffu, tincl, 31);
+    }
+    // inactive tail of the active list
+    for (int i = n_act + lane; i < EN; i += 32) {
+      r.active[i] = -1;
+      if (ex.active) ex.active[i] = -1;
+    }
+    if (lane == 0) {
+      s.off[EN] = carry;
+      r.expert_offset[EN] = carry;
+      if (ex.expert_offset) ex.expert_offset[EN] = carry;
+      *r.n_active = n_act;
+      *r.n_rows_active = n_rows_active;
+      *ws.n_items = n_items;
+      if (ex.n_active) *ex.n_active = n_act;
+      if (ex.n_rows_active) *ex.n_rows_active = n_rows_active;
+    }
+  }
+  __syncthreads();
+  // second walk: place the routed slots
+  for (int base = lo; base < hi; base += 32) {
+    const int slot = base + lane;
+    const int e = (slot < hi) ? r.topk_idx[slot] : -1;
+    const unsigned peers = __match_any_sync(0xffffffffu, e);
+    if (e >= 0) {
+      const int rank = my_hist[e] + __popc(peers & ((1u << lane) - 1));
+      const int at = s.off[e] + rank;
+      r.perm[at] = slot;
+      if (ex.perm) ex.perm[at] = slot;
+    }
+    __syncwarp();
+    if (e >= 0 && (__ffs(peers) - 1) == lane) my_hist[e] += __popc(peers);
+    __syncwarp();
+  }
+  // shared experts: slot T*k + s*T + t for every active row t, ascending t.
+  if (ns > 0) {
+    // ordered compaction of active rows by warp 0 (T <= TEAM_MAX_ROWS: at most 64 ballots)
+    if (warp == 0) {
+      int run = 0;
+      for (int base = 0; base < T; base += 32) {
+        const int t = base + lane;
+        const bool a = t < T && s.cls[t] != TEAM_CLS_SKIP;
+        const unsigned b = __ballot_sync(0xffffffffu, a);
+        if (a) {
+          const int rank = run + __popc(b & ((1u << lane) - 1));
+          for (int sh = 0; sh < ns; ++sh) {
+            const int at = s.off[E + sh] + rank;
+            const int slot = T * k + sh * T + t;
+            r.perm[at] = slot;
+            if (ex.perm) ex.perm[at] = slot;
+          }
+        }
+        run += __popc(b);
+      }
+    }
+  }
+  // unused tail of perm
+  const int total = s.off[EN];
+  for (int i = total + tid; i < T * (k + ns); i += kSelThreads) {
+    r.perm[i] = -1;
+    if (ex.perm) ex.perm[i] = -1;
+  }
+}
+
+cudaError_t launch_select(const float* logits, StepPtrs st, Workspace ws, RoutePtrs ex, Dims d, Policy p,
+                          int item_tile, cudaStream_t s) {
+  const size_t smem = select_smem_bytes(d);
+  cudaError_t err = cudaFuncSetAttribute(k_select, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (err != cudaSuccess) return err;
+  k_select<<<1, kSelThreads, smem, s>>>(logits, st, ws, ex, d, p, item_tile);
+  return cudaGetLastError();
+}
+
+}  // namespace team
