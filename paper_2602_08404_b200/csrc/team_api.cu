@@ -158,6 +158,13 @@ int team_create(const team_config* cfg, team_ctx** out) {
     return TEAM_ERR_CUDA;
   }
   ctx->item_tile = pick_item_tile(*cfg);
+  e = team::configure_router(cfg->dtype, cfg->hidden);
+  if (e == cudaSuccess) e = team::configure_select(dims_of(*cfg, cfg->max_rows));
+  if (e == cudaSuccess && cfg->dtype == TEAM_DTYPE_BF16) e = team::configure_experts_tc(ctx->item_tile);
+  if (e != cudaSuccess) {
+    delete ctx;
+    return TEAM_ERR_CUDA;
+  }
 
   const size_t T = cfg->max_rows, E = cfg->n_experts, k = cfg->top_k, ns = cfg->n_shared, EN = E + ns;
   const size_t S = T * (k + ns);

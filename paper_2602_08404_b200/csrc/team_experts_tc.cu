@@ -329,7 +329,13 @@ k_experts_tc(const __grid_constant__ CUtensorMap map_gate, const __grid_constant
       if (ok)
         for (int j = pending; j > 0; --j) mbar_arrive(smem_u32(bar_fullB + (it - j) % C::kStages));
       __syncwarp();
-      it += HT;
+      // Phase-2 stages carry no B tile, but the ring's empty barriers must still be observed one
+      // round at a time: a parity wait that skipped a round could be satisfied by an older phase.
+      for (int ht = 0; ok && ht < HT; ++ht, ++it) {
+        const uint32_t s = it % C::kStages, par = (it / C::kStages) & 1;
+        ok = mbar_wait(smem_u32(bar_empty + s), par ^ 1, abort_flag, a.status, 12);
+        ok = __all_sync(0xffffffffu, ok);
+      }
     }
   } else if (warp >= 4) {
     // ------------------------------ epilogue ------------------------------
@@ -452,15 +458,18 @@ int experts_tc_item_tile(int max_rows_per_expert) { return max_rows_per_expert <
 template <int NT>
 static cudaError_t launch_tc(const void* maps, TcArgs args, int grid, cudaStream_t s) {
   using C = TcCfg<NT>;
-  static bool configured = false;
-  if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(k_experts_tc<NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
-    if (e != cudaSuccess) return e;
-    configured = true;
-  }
   const CUtensorMap* m = reinterpret_cast<const CUtensorMap*>(maps);
   k_experts_tc<NT><<<grid, kTcThreads, C::kSmemBytes, s>>>(m[0], m[1], m[2], args);
   return cudaGetLastError();
+}
+
+cudaError_t configure_experts_tc(int item_tile) {
+  switch (item_tile) {
+    case 32: return cudaFuncSetAttribute(k_experts_tc<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, TcCfg<32>::kSmemBytes);
+    case 64: return cudaFuncSetAttribute(k_experts_tc<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, TcCfg<64>::kSmemBytes);
+    case 128: return cudaFuncSetAttribute(k_experts_tc<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, TcCfg<128>::kSmemBytes);
+    default: return cudaErrorInvalidValue;
+  }
 }
 
 cudaError_t launch_experts_tc(const void* maps, int item_tile, const void* x, Workspace ws, float* y, Dims d,

@@ -102,17 +102,23 @@ k_router_topk(const float* __restrict__ logits, const uint8_t* __restrict__ tok_
   if (lane == 0 && out.margin) out.margin[t] = r.margin;
 }
 
+// Opt in to the dynamic shared memory the kernels need (done once per context, outside any stream capture).
+cudaError_t configure_router(int dtype, int hidden) {
+  const int smem = kRowTile * hidden * (int)sizeof(float);
+  if (dtype == TEAM_DTYPE_F32)
+    return cudaFuncSetAttribute(k_router_logits<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  return cudaFuncSetAttribute(k_router_logits<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+}
+
 cudaError_t launch_router_logits(const void* x, int dtype, const float* w_router, const uint8_t* tok_state,
                                  float* logits, float* y_zero, Dims d, int flags, cudaStream_t s) {
   dim3 grid((d.E + kExpertsPerCta - 1) / kExpertsPerCta, (d.T + kRowTile - 1) / kRowTile);
   dim3 block(kExpertsPerCta * 32);
   const size_t smem = (size_t)kRowTile * d.H * sizeof(float);
   if (dtype == TEAM_DTYPE_F32) {
-    cudaFuncSetAttribute(k_router_logits<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     k_router_logits<float><<<grid, block, smem, s>>>(static_cast<const float*>(x), w_router, tok_state, logits,
                                                      y_zero, d, flags);
   } else {
-    cudaFuncSetAttribute(k_router_logits<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     k_router_logits<__nv_bfloat16><<<grid, block, smem, s>>>(static_cast<const __nv_bfloat16*>(x), w_router,
                                                              tok_state, logits, y_zero, d, flags);
   }

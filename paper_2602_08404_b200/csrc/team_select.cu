@@ -345,11 +345,14 @@ k_select(const float* __restrict__ logits, StepPtrs st, Workspace ws, RoutePtrs 
   }
 }
 
+cudaError_t configure_select(Dims max_dims) {
+  return cudaFuncSetAttribute(k_select, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              (int)select_smem_bytes(max_dims));
+}
+
 cudaError_t launch_select(const float* logits, StepPtrs st, Workspace ws, RoutePtrs ex, Dims d, Policy p,
                           int item_tile, cudaStream_t s) {
   const size_t smem = select_smem_bytes(d);
-  cudaError_t err = cudaFuncSetAttribute(k_select, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-  if (err != cudaSuccess) return err;
   k_select<<<1, kSelThreads, smem, s>>>(logits, st, ws, ex, d, p, item_tile);
   return cudaGetLastError();
 }

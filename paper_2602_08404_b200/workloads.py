@@ -66,6 +66,12 @@ MINI_SHARED = Shape("mini_shared_bf16", 128, 24, 3, 64, 1, "bf16", 12, 5, 2, 1, 
                     seqs=2, branches=2, seed=12)
 
 
+# Enough k-blocks to wrap the expert kernel's smem ring inside one GEMM phase and enough work
+# units that every CTA of a 148-SM grid processes several.
+MINI_WRAP = Shape("mini_wrap_bf16", 768, 64, 4, 192, 0, "bf16", 16, 4, 3, 1, 2, 0.7,
+                  seqs=2, branches=2, seed=13)
+
+
 def round_to_bf16(a):
     """Round fp32 values to the nearest bf16-representable value (ties to even); returns fp32."""
     a = np.ascontiguousarray(a, dtype=np.float32)
