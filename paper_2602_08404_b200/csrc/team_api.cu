@@ -10,9 +10,11 @@
 #include "team_common.cuh"
 
 namespace team {
-int make_weight_map(void* out_map, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows);
-cudaError_t launch_experts_tc(const void* maps, int item_tile, const void* x, Workspace ws, float* y, Dims d,
-                              int grid, cudaStream_t s);
+int make_expert_maps(void* out_maps, const void* w_gate, const void* w_up, const void* w_down, uint64_t rows_gu,
+                     uint64_t H, uint64_t rows_d, uint64_t I, int* gate_first);
+size_t experts_tc_maps_bytes();
+cudaError_t launch_experts_tc(const void* maps, int gate_first, int item_tile, const void* x, Workspace ws, float* y,
+                              Dims d, int grid, cudaStream_t s);
 }  // namespace team
 
 struct team_ctx {
@@ -22,7 +24,8 @@ struct team_ctx {
   size_t ws_bytes;
   team_weights w;
   bool has_weights;
-  alignas(64) CUtensorMap maps[3];
+  alignas(64) CUtensorMap maps[5];   // four gate/up views (1-4 groups per box) and W_down
+  int gate_first;
   int device;
   int n_sms;
   int item_tile;
@@ -228,9 +231,9 @@ int team_set_weights(team_ctx* ctx, const team_weights* w) {
     return TEAM_ERR_ARG;
   if (ctx->cfg.dtype == TEAM_DTYPE_BF16) {
     const uint64_t EN = ctx->cfg.n_experts + ctx->cfg.n_shared, I = ctx->cfg.inter, H = ctx->cfg.hidden;
-    int r = team::make_weight_map(&ctx->maps[0], w->w_gate, EN * I, H, 16);
-    if (r == 0) r = team::make_weight_map(&ctx->maps[1], w->w_up, EN * I, H, 16);
-    if (r == 0) r = team::make_weight_map(&ctx->maps[2], w->w_down, EN * H, I, 128);
+    if (team::experts_tc_maps_bytes() != sizeof(ctx->maps)) return TEAM_ERR_SHAPE;
+    const int r = team::make_expert_maps(ctx->maps, w->w_gate, w->w_up, w->w_down, EN * I, H, EN * H, I,
+                                         &ctx->gate_first);
     if (r != 0) {
       snprintf(ctx->cuda_err, sizeof(ctx->cuda_err), "cuTensorMapEncodeTiled failed (%d)", r);
       return TEAM_ERR_CUDA;
@@ -328,10 +331,7 @@ int team_moe_forward(team_ctx* ctx, const void* x, const team_step_state* st, te
     cudaEventRecord(ev0, s);
   }
   if (tc) {
-    const int EN = d.E + d.ns;
-    long max_work = ((long)EN + (long)d.T * (d.k + d.ns) / ctx->item_tile) * (d.I / 64);
-    int grid = (int)(max_work < ctx->n_sms ? max_work : ctx->n_sms);
-    e = team::launch_experts_tc(ctx->maps, ctx->item_tile, x, ctx->ws, y, d, grid, s);
+    e = team::launch_experts_tc(ctx->maps, ctx->gate_first, ctx->item_tile, x, ctx->ws, y, d, ctx->n_sms, s);
     if (e != cudaSuccess) return fail_cuda(ctx, e, "expert kernel");
     ++ctx->last_launches;
   } else {

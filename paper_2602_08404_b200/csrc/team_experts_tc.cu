@@ -1,18 +1,24 @@
 // Grouped SwiGLU expert kernel for bf16 weights on sm_100a: TMA-staged weight tiles, tcgen05.mma
 // with accumulators in tensor memory, SwiGLU and the routing-weight scatter-combine fused in.
 //
-// Work unit = (work item, 64-wide slice of the expert's intermediate dimension).  A work item is a
-// run of up to NT token-slots of one activated expert (built by the selection kernel).  For its unit
-// a CTA
-//   phase 1  streams W_gate[e, slice, :] and W_up[e, slice, :] (64 + 64 rows, interleaved in 16-row
-//            groups so that a gate row and its up row land in the same warp's TMEM lanes) against the
-//            gathered token rows:  D1[128, N] = A[128, H] * X[N, H]^T          (weights on M, tokens on N)
+// Work is measured in "groups": 16 consecutive columns of one work item's intermediate dimension
+// (a work item is a run of up to NT token-slots of one activated expert, built by the selection
+// kernel).  A group costs the same HBM bytes everywhere (16 gate rows + 16 up rows + a 16-column
+// strip of W_down), so the global list of groups is cut into one contiguous range per CTA and every
+// SM streams the same number of bytes (+- one group).  A CTA walks its range in chunks: the part of
+// the range that falls into one 64-column window of one item (1 to 4 groups).  For a chunk it
+//   phase 1  streams the chunk's W_gate / W_up rows against the gathered token rows,
+//            D1[128, N] = A[128, H] * X[N, H]^T  (weights on M, tokens on N).  One 4-D TMA box per
+//            64-wide k-block delivers the rows already interleaved as [group][gate 16 | up 16], so a
+//            gate row and its up row sit in the same warp's TMEM lanes.
 //   SwiGLU   reads D1 from TMEM, a = silu(gate) * up, writes a as bf16 into shared memory in the
 //            K-major 128B-swizzled layout the tensor core reads as a B operand
-//   phase 2  streams W_down[e, :, slice] in 128-row tiles: D2[128, N] = Wd_tile[128, 64] * a[N, 64]^T,
-//            multiplies by the slot's routing weight and adds into y[row, h] with fp32 reductions.
-// Every weight byte of an activated expert is read from HBM exactly once per step (when the expert
-// has at most NT slots); nothing but y is written.
+//   phase 2  streams W_down[e, :, window] in 128-row tiles: D2[128, N] = Wd_tile[128, cols] * a[N, cols]^T
+//            over the chunk's columns, multiplies by the slot's routing weight and adds into y[row, h]
+//            with fp32 reductions.
+// Every weight byte of an activated expert is read from HBM once per step (two CTAs that share a
+// window read its W_down tiles at the same time, odd CTAs walking their range backwards, so the
+// second read is served by L2); nothing but y is written.
 //
 // Warp roles (256 threads): warp 0 = TMA producer, warp 1 = MMA issuer + TMEM owner, warp 2 = token
 // gather (cp.async into the swizzled B tile), warp 3 idle, warps 4-7 = epilogue (one TMEM lane
@@ -26,7 +32,8 @@ namespace team {
 
 constexpr int kTcThreads = 256;
 constexpr int kATileBytes = 128 * 128;          // 128 rows x 64 bf16
-constexpr int kSliceI = 64;                     // intermediate columns per work unit
+constexpr int kGroupCols = 16;                  // intermediate columns per group (the unit of balance)
+constexpr int kWindowCols = 64;                 // columns per window (one 128-byte swizzle row of W_down)
 constexpr unsigned long long kWaitCycles = 2000000000ull;   // ~1 s at 2 GHz
 
 template <int NT>
@@ -91,6 +98,14 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
       : "memory");
 }
 
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, int c0, int c1, int c2, int c3,
+                                            uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
+      ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(bar)
+      : "memory");
+}
+
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
@@ -148,12 +163,55 @@ struct TcArgs {
   float* y;                    // [T, H], pre-zeroed rows of computed tokens
   int32_t* status;
   Dims d;
+  int gate_first;              // 1: the 4-D box delivers [gate | up] per group, 0: [up | gate]
+};
+
+// Tensor maps: gu[g-1] = W_gate/W_up viewed as {H, 16 rows, 2 (gate, up), rows/16} with a box of g
+// groups; down = W_down as {I, rows} with a [128 x 64] box.
+struct TcMaps {
+  CUtensorMap gu[4];
+  CUtensorMap down;
+};
+
+// One step of a CTA's walk over its group range.
+struct Chunk {
+  int item;     // work item
+  int window;   // 64-column window of the intermediate dimension
+  int g0;       // first group of the window that belongs to the chunk (0..3)
+  int g;        // groups in the chunk (1..4)
+};
+
+struct ChunkWalker {
+  long long lo, hi, cur;
+  int NG;
+  bool reverse;
+  __device__ ChunkWalker(long long lo_, long long hi_, int ng, bool rev)
+      : lo(lo_), hi(hi_), cur(rev ? hi_ : lo_), NG(ng), reverse(rev) {}
+  __device__ bool next(Chunk& c) {
+    if (!reverse) {
+      if (cur >= hi) return false;
+      const long long item = cur / NG;
+      const int j = (int)(cur - item * NG);
+      long long end = item * NG + (j / 4 + 1) * 4;
+      if (end > hi) end = hi;
+      c.item = (int)item; c.window = j / 4; c.g0 = j % 4; c.g = (int)(end - cur);
+      cur = end;
+    } else {
+      if (cur <= lo) return false;
+      const long long last = cur - 1, item = last / NG;
+      const int j = (int)(last - item * NG);
+      long long begin = item * NG + (j / 4) * 4;
+      if (begin < lo) begin = lo;
+      c.item = (int)item; c.window = j / 4; c.g0 = (int)(begin - item * NG) % 4; c.g = (int)(cur - begin);
+      cur = begin;
+    }
+    return true;
+  }
 };
 
 template <int NT>
 __global__ void __launch_bounds__(kTcThreads, 1)
-k_experts_tc(const __grid_constant__ CUtensorMap map_gate, const __grid_constant__ CUtensorMap map_up,
-             const __grid_constant__ CUtensorMap map_down, TcArgs a) {
+k_experts_tc(const __grid_constant__ TcMaps maps, TcArgs a) {
   using C = TcCfg<NT>;
   extern __shared__ unsigned char smem_dyn[];
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~uintptr_t(1023));
@@ -173,7 +231,7 @@ k_experts_tc(const __grid_constant__ CUtensorMap map_gate, const __grid_constant
   const Dims d = a.d;
   const int KB = d.H / 64;          // k-blocks of phase 1
   const int HT = d.H / 128;         // row tiles of phase 2
-  const int n_slices = d.I / kSliceI;
+  const int NG = d.I / kGroupCols;  // groups per work item
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < C::kStages; ++s) {
@@ -203,27 +261,31 @@ k_experts_tc(const __grid_constant__ CUtensorMap map_gate, const __grid_constant
   const uint32_t tmem_base = *tmem_slot;
   const uint32_t tmem_acc1 = tmem_base;
 
-  const int n_work = (*a.n_items) * n_slices;
+  // This CTA's contiguous range of groups; odd CTAs walk it backwards so that the two CTAs sharing a
+  // window touch its W_down tiles at the same time.
+  const long long n_groups = (long long)(*a.n_items) * NG;
+  const long long g_lo = n_groups * blockIdx.x / gridDim.x, g_hi = n_groups * (blockIdx.x + 1) / gridDim.x;
+  const bool reverse = (blockIdx.x & 1) != 0;
 
   if (warp == 0) {
     // ------------------------------ TMA producer ------------------------------
     if (lane == 0) {
       uint32_t it = 0;
       bool ok = true;
-      for (int w = blockIdx.x; ok && w < n_work; w += gridDim.x) {
-        const WorkItem item = a.items[w / n_slices];
-        const int slice = w % n_slices;
-        const int row_gu = item.e * d.I + slice * kSliceI;
+      ChunkWalker walk(g_lo, g_hi, NG, reverse);
+      Chunk c;
+      while (ok && walk.next(c)) {
+        const WorkItem item = a.items[c.item];
+        const int col0 = c.window * kWindowCols + c.g0 * kGroupCols;
+        const int grp = (item.e * d.I + col0) / kGroupCols;          // coordinate in units of 16 rows
+        const CUtensorMap* gu = &maps.gu[c.g - 1];
+        const uint32_t bytes1 = (uint32_t)c.g * 4096u;
         for (int kb = 0; kb < KB; ++kb, ++it) {
           const uint32_t s = it % C::kStages, par = (it / C::kStages) & 1;
           if (!(ok = mbar_wait(smem_u32(bar_empty + s), par ^ 1, abort_flag, a.status, 1))) break;
           const uint32_t dst = smem_u32(smem + s * C::kStageBytes), bar = smem_u32(bar_fullA + s);
-          mbar_arrive_expect_tx(bar, kATileBytes);
-#pragma unroll
-          for (int q = 0; q < 4; ++q) {
-            tma_load_2d(dst + (q * 32) * 128, &map_gate, kb * 64, row_gu + q * 16, bar);
-            tma_load_2d(dst + (q * 32 + 16) * 128, &map_up, kb * 64, row_gu + q * 16, bar);
-          }
+          mbar_arrive_expect_tx(bar, bytes1);
+          tma_load_4d(dst, gu, kb * 64, 0, 0, grp, bar);
         }
         if (!ok) break;
         for (int ht = 0; ht < HT; ++ht, ++it) {
@@ -231,7 +293,7 @@ k_experts_tc(const __grid_constant__ CUtensorMap map_gate, const __grid_constant
           if (!(ok = mbar_wait(smem_u32(bar_empty + s), par ^ 1, abort_flag, a.status, 2))) break;
           const uint32_t dst = smem_u32(smem + s * C::kStageBytes), bar = smem_u32(bar_fullA + s);
           mbar_arrive_expect_tx(bar, kATileBytes);
-          tma_load_2d(dst, &map_down, slice * kSliceI, item.e * d.H + ht * 128, bar);
+          tma_load_2d(dst, &maps.down, c.window * kWindowCols, item.e * d.H + ht * 128, bar);
         }
       }
       if (*abort_flag) {
@@ -244,17 +306,20 @@ k_experts_tc(const __grid_constant__ CUtensorMap map_gate, const __grid_constant
         }
       }
     }
+    __syncwarp();
   } else if (warp == 1) {
     // ------------------------------ MMA issuer ------------------------------
     if (lane == 0) {
-      uint32_t it = 0, item_i = 0, t2 = 0, bphase = 0;
+      uint32_t it = 0, chunk_i = 0, t2 = 0, bphase = 0;
       bool ok = true;
       const uint64_t act_desc = make_kmajor_sw128_desc(smem_u32(act_tile));
-      for (int w = blockIdx.x; ok && w < n_work; w += gridDim.x, ++item_i) {
-        const WorkItem item = a.items[w / n_slices];
+      ChunkWalker walk(g_lo, g_hi, NG, reverse);
+      Chunk c;
+      for (; ok && walk.next(c); ++chunk_i) {
+        const WorkItem item = a.items[c.item];
         const int N = (item.n + 15) & ~15;
         const uint32_t idesc = make_idesc_bf16(N);
-        if (!(ok = mbar_wait(smem_u32(bar_misc + 1), (item_i & 1) ^ 1, abort_flag, a.status, 3))) break;
+        if (!(ok = mbar_wait(smem_u32(bar_misc + 1), (chunk_i & 1) ^ 1, abort_flag, a.status, 3))) break;
         tc_fence_after();
         for (int kb = 0; kb < KB; ++kb, ++it) {
           const uint32_t s = it % C::kStages, par = (it / C::kStages) & 1;
@@ -271,7 +336,7 @@ k_experts_tc(const __grid_constant__ CUtensorMap map_gate, const __grid_constant
         }
         if (!ok) break;
         tc_commit(smem_u32(bar_misc + 0));
-        if (!(ok = mbar_wait(smem_u32(bar_misc + 2), item_i & 1, abort_flag, a.status, 6))) break;
+        if (!(ok = mbar_wait(smem_u32(bar_misc + 2), chunk_i & 1, abort_flag, a.status, 6))) break;
         tc_fence_after();
         for (int ht = 0; ht < HT; ++ht, ++it, ++t2) {
           const uint32_t b = t2 & 1, u = t2 >> 1;
@@ -281,20 +346,23 @@ k_experts_tc(const __grid_constant__ CUtensorMap map_gate, const __grid_constant
           tc_fence_after();
           const uint64_t da = make_kmajor_sw128_desc(smem_u32(smem + s * C::kStageBytes));
           const uint32_t acc2 = tmem_base + NT * (1 + b);
-#pragma unroll
-          for (int k4 = 0; k4 < 4; ++k4) tc_mma(acc2, da + 2 * k4, act_desc + 2 * k4, idesc, k4 != 0);
+          // the chunk's columns are k-steps g0 .. g0+g-1 of the window tile and 0 .. g-1 of the activation tile
+          for (int kk = 0; kk < c.g; ++kk) tc_mma(acc2, da + 2 * (c.g0 + kk), act_desc + 2 * kk, idesc, kk != 0);
           tc_commit(smem_u32(bar_empty + s));
           tc_commit(smem_u32(bar_misc + 3 + b));
         }
       }
     }
+    __syncwarp();
   } else if (warp == 2) {
     // ------------------------------ token gather (B operand of phase 1) ------------------------------
     constexpr int kLag = 3;   // stages of cp.async kept in flight
     uint32_t it = 0;
     bool ok = true;
-    for (int w = blockIdx.x; ok && w < n_work; w += gridDim.x) {
-      const WorkItem item = a.items[w / n_slices];
+    ChunkWalker walk(g_lo, g_hi, NG, reverse);
+    Chunk c;
+    while (ok && walk.next(c)) {
+      const WorkItem item = a.items[c.item];
       for (int r = lane; r < item.n; r += 32) {
         int row;
         float wt;
@@ -310,8 +378,8 @@ k_experts_tc(const __grid_constant__ CUtensorMap map_gate, const __grid_constant
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
         const uint32_t dstB = smem_u32(smem + s * C::kStageBytes + kATileBytes);
-        for (int c = lane; c < chunks; c += 32) {
-          const int r = c >> 3, ch = c & 7;
+        for (int ch16 = lane; ch16 < chunks; ch16 += 32) {
+          const int r = ch16 >> 3, ch = ch16 & 7;
           const __nv_bfloat16* src = a.x + (size_t)gather_row[r] * d.H + kb * 64 + ch * 8;
           const uint32_t dst = dstB + r * 128 + ((ch ^ (r & 7)) << 4);
           asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
@@ -339,14 +407,16 @@ k_experts_tc(const __grid_constant__ CUtensorMap map_gate, const __grid_constant
     }
   } else if (warp >= 4) {
     // ------------------------------ epilogue ------------------------------
-    const int q = warp - 4;                       // TMEM lane quarter == warp_id % 4
+    const int q = warp - 4;                       // TMEM lane quarter == warp_id % 4 == group inside the chunk
     int32_t* my_row = tbl_row + q * NT;
     float* my_wt = tbl_wt + q * NT;
     const uint32_t lane_off = (uint32_t)(q * 32) << 16;
-    uint32_t item_i = 0, t2 = 0;
+    uint32_t chunk_i = 0, t2 = 0;
     bool ok = true;
-    for (int w = blockIdx.x; ok && w < n_work; w += gridDim.x, ++item_i) {
-      const WorkItem item = a.items[w / n_slices];
+    ChunkWalker walk(g_lo, g_hi, NG, reverse);
+    Chunk c;
+    for (; ok && walk.next(c); ++chunk_i) {
+      const WorkItem item = a.items[c.item];
       const int N = (item.n + 15) & ~15;
       __syncwarp();
       for (int r = lane; r < item.n; r += 32) {
@@ -358,28 +428,32 @@ k_experts_tc(const __grid_constant__ CUtensorMap map_gate, const __grid_constant
       }
       __syncwarp();
       // ---- SwiGLU: TMEM -> registers -> bf16 activation tile (B operand of phase 2) ----
-      ok = mbar_wait(smem_u32(bar_misc + 0), item_i & 1, abort_flag, a.status, 10);
+      ok = mbar_wait(smem_u32(bar_misc + 0), chunk_i & 1, abort_flag, a.status, 10);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
-      const int i_local = q * 16 + (lane & 15);     // column of the 64-wide slice this lane pair owns
-      for (int c0 = 0; c0 < N; c0 += 8) {
-        float v[8];
-        tmem_ld8(tmem_acc1 + lane_off + c0, v);
+      if (q < c.g) {
+        const int i_local = q * 16 + (lane & 15);     // column of the activation tile this lane pair owns
+        const bool first_half = lane < 16;
+        for (int c0 = 0; c0 < N; c0 += 8) {
+          float v[8];
+          tmem_ld8(tmem_acc1 + lane_off + c0, v);
 #pragma unroll
-        for (int j = 0; j < 8; ++j) {
-          const float o = __shfl_xor_sync(0xffffffffu, v[j], 16);
-          const float g = (lane < 16) ? v[j] : o;
-          const float u = (lane < 16) ? o : v[j];
-          v[j] = g / (1.f + expf(-g)) * u;
-        }
-        // lanes 0-15 store columns c0..c0+3, lanes 16-31 store c0+4..c0+7
-        const int jb = (lane < 16) ? 0 : 4;
+          for (int j = 0; j < 8; ++j) {
+            const float o = __shfl_xor_sync(0xffffffffu, v[j], 16);
+            const bool mine_is_gate = (first_half == (a.gate_first != 0));
+            const float g = mine_is_gate ? v[j] : o;
+            const float u = mine_is_gate ? o : v[j];
+            v[j] = g / (1.f + expf(-g)) * u;
+          }
+          // lanes 0-15 store columns c0..c0+3, lanes 16-31 store c0+4..c0+7
+          const int jb = first_half ? 0 : 4;
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-          const int n = c0 + jb + j;
-          const uint32_t off = n * 128 + (((i_local >> 3) ^ (n & 7)) << 4) + (i_local & 7) * 2;
-          *reinterpret_cast<__nv_bfloat16*>(act_tile + off) = __float2bfloat16_rn(v[jb + j]);
+          for (int j = 0; j < 4; ++j) {
+            const int n = c0 + jb + j;
+            const uint32_t off = n * 128 + (((i_local >> 3) ^ (n & 7)) << 4) + (i_local & 7) * 2;
+            *reinterpret_cast<__nv_bfloat16*>(act_tile + off) = __float2bfloat16_rn(v[jb + j]);
+          }
         }
       }
       tc_fence_before();
@@ -439,27 +513,44 @@ static EncodeTiledFn get_encode_fn() {
   return fn;
 }
 
-// 2-D bf16 tensor [rows, cols] row-major, box [box_rows, 64 cols], 128-byte swizzle.
-int make_weight_map(void* out_map, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows) {
+size_t experts_tc_maps_bytes() { return sizeof(TcMaps); }
+
+// Builds the five tensor maps for a layer.  w_gate / w_up: bf16 [rows_gu, H]; w_down: bf16 [rows_d, I].
+// Returns 0, or a driver error code / -1.  *gate_first tells the kernel which of gate / up comes
+// first inside a group (the 4-D view needs a positive stride between the two matrices).
+int make_expert_maps(void* out_maps, const void* w_gate, const void* w_up, const void* w_down, uint64_t rows_gu,
+                     uint64_t H, uint64_t rows_d, uint64_t I, int* gate_first) {
   EncodeTiledFn fn = get_encode_fn();
   if (fn == nullptr) return -1;
-  cuuint64_t dims[2] = {cols, rows};
-  cuuint64_t strides[1] = {cols * 2};
-  cuuint32_t box[2] = {64, box_rows};
+  TcMaps* m = reinterpret_cast<TcMaps*>(out_maps);
+  const uintptr_t pg = reinterpret_cast<uintptr_t>(w_gate), pu = reinterpret_cast<uintptr_t>(w_up);
+  *gate_first = pu > pg ? 1 : 0;
+  const uintptr_t base = pu > pg ? pg : pu, delta = pu > pg ? pu - pg : pg - pu;
+  if (delta == 0 || (delta & 15) || delta >= (1ull << 40)) return -2;
+  for (int g = 1; g <= 4; ++g) {
+    cuuint64_t dims[4] = {H, 16, 2, rows_gu / 16};
+    cuuint64_t strides[3] = {H * 2, delta, 16 * H * 2};
+    cuuint32_t box[4] = {64, 16, 2, (cuuint32_t)g};
+    cuuint32_t estr[4] = {1, 1, 1, 1};
+    CUresult r = fn(&m->gu[g - 1], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, reinterpret_cast<void*>(base), dims, strides,
+                    box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                    CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return (int)r;
+  }
+  cuuint64_t dims[2] = {I, rows_d};
+  cuuint64_t strides[1] = {I * 2};
+  cuuint32_t box[2] = {64, 128};
   cuuint32_t estr[2] = {1, 1};
-  CUresult r = fn(reinterpret_cast<CUtensorMap*>(out_map), CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2,
-                  const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                  CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  CUresult r = fn(&m->down, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(w_down), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS ? 0 : (int)r;
 }
-
-int experts_tc_item_tile(int max_rows_per_expert) { return max_rows_per_expert <= 32 ? 32 : (max_rows_per_expert <= 64 ? 64 : 128); }
 
 template <int NT>
 static cudaError_t launch_tc(const void* maps, TcArgs args, int grid, cudaStream_t s) {
   using C = TcCfg<NT>;
-  const CUtensorMap* m = reinterpret_cast<const CUtensorMap*>(maps);
-  k_experts_tc<NT><<<grid, kTcThreads, C::kSmemBytes, s>>>(m[0], m[1], m[2], args);
+  k_experts_tc<NT><<<grid, kTcThreads, C::kSmemBytes, s>>>(*reinterpret_cast<const TcMaps*>(maps), args);
   return cudaGetLastError();
 }
 
@@ -472,8 +563,8 @@ cudaError_t configure_experts_tc(int item_tile) {
   }
 }
 
-cudaError_t launch_experts_tc(const void* maps, int item_tile, const void* x, Workspace ws, float* y, Dims d,
-                              int grid, cudaStream_t s) {
+cudaError_t launch_experts_tc(const void* maps, int gate_first, int item_tile, const void* x, Workspace ws, float* y,
+                              Dims d, int grid, cudaStream_t s) {
   TcArgs a;
   a.x = static_cast<const __nv_bfloat16*>(x);
   a.perm = ws.r.perm;
@@ -483,6 +574,7 @@ cudaError_t launch_experts_tc(const void* maps, int item_tile, const void* x, Wo
   a.y = y;
   a.status = ws.status;
   a.d = d;
+  a.gate_first = gate_first;
   switch (item_tile) {
     case 32: return launch_tc<32>(maps, a, grid, s);
     case 64: return launch_tc<64>(maps, a, grid, s);

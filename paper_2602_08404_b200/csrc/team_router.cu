@@ -25,15 +25,28 @@ k_router_logits(const XT* __restrict__ x, const float* __restrict__ w_router, co
   const int tid = threadIdx.x;
   const int H = d.H;
 
-  for (int i = tid; i < nt * H; i += blockDim.x) s_x[i] = to_f32(x[(size_t)t0 * H + i]);
+  if constexpr (sizeof(XT) == 2) {
+    const uint2* src = reinterpret_cast<const uint2*>(x + (size_t)t0 * H);
+    for (int i = tid; i < nt * H / 4; i += blockDim.x) {
+      const uint2 v = __ldg(src + i);
+      const float2 a = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&v.x));
+      const float2 b = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&v.y));
+      reinterpret_cast<float4*>(s_x)[i] = make_float4(a.x, a.y, b.x, b.y);
+    }
+  } else {
+    const float4* src = reinterpret_cast<const float4*>(x + (size_t)t0 * H);
+    for (int i = tid; i < nt * H / 4; i += blockDim.x) reinterpret_cast<float4*>(s_x)[i] = __ldg(src + i);
+  }
   for (int i = nt * H + tid; i < kRowTile * H; i += blockDim.x) s_x[i] = 0.f;
 
-  // Output rows of computed tokens start from zero (the expert kernel adds partial sums into them).
-  if (y_zero != nullptr && blockIdx.x == 0) {
+  // Output rows of computed tokens start from zero (the expert kernel adds partial sums into them);
+  // the CTAs of one row tile share the job.
+  if (y_zero != nullptr) {
     for (int r = 0; r < nt; ++r) {
       const bool skip = (flags & TEAM_F_DCD) && tok_state[t0 + r] == TEAM_TOK_CACHED;
       if (!skip)
-        for (int i = tid; i < H; i += blockDim.x) y_zero[(size_t)(t0 + r) * H + i] = 0.f;
+        for (int i = blockIdx.x * blockDim.x + tid; i < H; i += gridDim.x * blockDim.x)
+          y_zero[(size_t)(t0 + r) * H + i] = 0.f;
     }
   }
   __syncthreads();
@@ -62,6 +75,101 @@ k_router_logits(const XT* __restrict__ x, const float* __restrict__ w_router, co
   for (int r = 0; r < kRowTile; ++r) {
     const float s = warp_sum(acc[r]);
     if (lane == 0 && r < nt) logits[(size_t)(t0 + r) * d.E + e] = s;
+  }
+}
+
+
+// Few rows (T <= kRowTile): the whole job is one pass over the 4*E*H bytes of router weights, so it
+// is spread as widely as possible -- two experts per CTA, four warps per expert, each lane issuing all
+// of its 128-bit weight loads before anything else -- and the activations are staged once per CTA.
+constexpr int kSmallExperts = 2;   // experts per CTA
+constexpr int kSmallSplit = 4;     // warps per expert (each takes H/4 of the dot product)
+constexpr int kSmallMaxVec = 8;    // float4 per lane: supports H <= 4096
+
+template <typename XT>
+__global__ void __launch_bounds__(kSmallExperts * kSmallSplit * 32)
+k_router_logits_small(const XT* __restrict__ x, const float* __restrict__ w_router,
+                      const uint8_t* __restrict__ tok_state, float* __restrict__ logits, float* __restrict__ y_zero,
+                      Dims d, int flags) {
+  extern __shared__ __align__(16) float s_x[];   // [T][H] then partial sums
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int H = d.H, T = d.T;
+  const int e = blockIdx.x * kSmallExperts + warp / kSmallSplit;
+  const int part = warp % kSmallSplit;
+  const int n4 = H >> 2, per_part = n4 / kSmallSplit;   // float4 per warp
+
+  // 1. weights first: every load in flight at once
+  float4 w[kSmallMaxVec];
+  const float4* wrow = reinterpret_cast<const float4*>(w_router + (size_t)min(e, d.E - 1) * H) + part * per_part;
+#pragma unroll
+  for (int i = 0; i < kSmallMaxVec; ++i)
+    w[i] = (lane + 32 * i < per_part) ? __ldg(wrow + lane + 32 * i) : make_float4(0.f, 0.f, 0.f, 0.f);
+
+  // 2. stage the rows (16-byte loads), zero this CTA's share of the output rows
+  if constexpr (sizeof(XT) == 2) {
+    const uint4* src = reinterpret_cast<const uint4*>(x);
+    for (int i = tid; i < T * H / 8; i += blockDim.x) {
+      const uint4 v = __ldg(src + i);
+      const __nv_bfloat162* p = reinterpret_cast<const __nv_bfloat162*>(&v);
+      float4 lo, hi;
+      float2 f;
+      f = __bfloat1622float2(p[0]); lo.x = f.x; lo.y = f.y;
+      f = __bfloat1622float2(p[1]); lo.z = f.x; lo.w = f.y;
+      f = __bfloat1622float2(p[2]); hi.x = f.x; hi.y = f.y;
+      f = __bfloat1622float2(p[3]); hi.z = f.x; hi.w = f.y;
+      reinterpret_cast<float4*>(s_x)[2 * i] = lo;
+      reinterpret_cast<float4*>(s_x)[2 * i + 1] = hi;
+    }
+  } else {
+    const float4* src = reinterpret_cast<const float4*>(x);
+    for (int i = tid; i < T * H / 4; i += blockDim.x) reinterpret_cast<float4*>(s_x)[i] = __ldg(src + i);
+  }
+  if (y_zero != nullptr) {
+    const int total4 = T * H / 4;
+    for (int i = blockIdx.x * blockDim.x + tid; i < total4; i += gridDim.x * blockDim.x) {
+      const int t = (i * 4) / H;
+      const bool skip = (flags & TEAM_F_DCD) && tok_state[t] == TEAM_TOK_CACHED;
+      if (!skip) reinterpret_cast<float4*>(y_zero)[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+  }
+  __syncthreads();
+
+  // 3. partial dot products, warp reduction, then the four parts of each expert are added in a fixed order
+  float acc[kRowTile];
+#pragma unroll
+  for (int r = 0; r < kRowTile; ++r) acc[r] = 0.f;
+#pragma unroll
+  for (int i = 0; i < kSmallMaxVec; ++i) {
+    if (lane + 32 * i < per_part) {
+      const int c = part * per_part + lane + 32 * i;
+#pragma unroll
+      for (int r = 0; r < kRowTile; ++r) {
+        if (r < T) {
+          const float4 xv = *reinterpret_cast<const float4*>(s_x + r * H + c * 4);
+          acc[r] = fmaf(w[i].x, xv.x, acc[r]);
+          acc[r] = fmaf(w[i].y, xv.y, acc[r]);
+          acc[r] = fmaf(w[i].z, xv.z, acc[r]);
+          acc[r] = fmaf(w[i].w, xv.w, acc[r]);
+        }
+      }
+    }
+  }
+  float* s_part = s_x + T * H;   // [warps][kRowTile]
+#pragma unroll
+  for (int r = 0; r < kRowTile; ++r) {
+    const float sum = warp_sum(acc[r]);
+    if (lane == 0) s_part[warp * kRowTile + r] = sum;
+  }
+  __syncthreads();
+  if (tid < kSmallExperts * kRowTile) {
+    const int le = tid / kRowTile, r = tid % kRowTile;
+    const int ee = blockIdx.x * kSmallExperts + le;
+    if (ee < d.E && r < T) {
+      float sum = 0.f;
+#pragma unroll
+      for (int q = 0; q < kSmallSplit; ++q) sum += s_part[(le * kSmallSplit + q) * kRowTile + r];
+      logits[(size_t)r * d.E + ee] = sum;
+    }
   }
 }
 
@@ -103,15 +211,38 @@ k_router_topk(const float* __restrict__ logits, const uint8_t* __restrict__ tok_
 }
 
 // Opt in to the dynamic shared memory the kernels need (done once per context, outside any stream capture).
+static bool small_router_ok(const Dims& d) {
+  return d.T <= kRowTile && d.H % (4 * kSmallSplit) == 0 && d.H / (4 * kSmallSplit) <= 32 * kSmallMaxVec;
+}
+
 cudaError_t configure_router(int dtype, int hidden) {
-  const int smem = kRowTile * hidden * (int)sizeof(float);
-  if (dtype == TEAM_DTYPE_F32)
-    return cudaFuncSetAttribute(k_router_logits<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-  return cudaFuncSetAttribute(k_router_logits<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  const int smem = kRowTile * hidden * (int)sizeof(float) + 1024;
+  cudaError_t e;
+  if (dtype == TEAM_DTYPE_F32) {
+    e = cudaFuncSetAttribute(k_router_logits<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e == cudaSuccess)
+      e = cudaFuncSetAttribute(k_router_logits_small<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  } else {
+    e = cudaFuncSetAttribute(k_router_logits<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e == cudaSuccess)
+      e = cudaFuncSetAttribute(k_router_logits_small<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  }
+  return e;
 }
 
 cudaError_t launch_router_logits(const void* x, int dtype, const float* w_router, const uint8_t* tok_state,
                                  float* logits, float* y_zero, Dims d, int flags, cudaStream_t s) {
+  if (small_router_ok(d)) {
+    dim3 grid((d.E + kSmallExperts - 1) / kSmallExperts), block(kSmallExperts * kSmallSplit * 32);
+    const size_t smem = (size_t)d.T * d.H * sizeof(float) + kSmallExperts * kSmallSplit * kRowTile * sizeof(float);
+    if (dtype == TEAM_DTYPE_F32)
+      k_router_logits_small<float><<<grid, block, smem, s>>>(static_cast<const float*>(x), w_router, tok_state,
+                                                             logits, y_zero, d, flags);
+    else
+      k_router_logits_small<__nv_bfloat16><<<grid, block, smem, s>>>(static_cast<const __nv_bfloat16*>(x), w_router,
+                                                                     tok_state, logits, y_zero, d, flags);
+    return cudaGetLastError();
+  }
   dim3 grid((d.E + kExpertsPerCta - 1) / kExpertsPerCta, (d.T + kRowTile - 1) / kRowTile);
   dim3 block(kExpertsPerCta * 32);
   const size_t smem = (size_t)kRowTile * d.H * sizeof(float);

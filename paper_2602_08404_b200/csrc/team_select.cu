@@ -14,6 +14,8 @@ namespace team {
 constexpr int kSelThreads = 1024;
 constexpr int kSelWarps = kSelThreads / 32;
 
+constexpr int kIdxInSmemMax = 8192;   // routed slots kept in shared memory between the rounds and the dispatch
+
 struct SelSmem {
   // carved from dynamic shared memory in this order
   uint32_t* mask;      // [G][8]  E_A bits (256 experts max)
@@ -22,6 +24,7 @@ struct SelSmem {
   int32_t* key;        // [T] group*256 + branch
   int32_t* pos;        // [T]
   int32_t* warp_cnt;   // [kSelWarps + 1]
+  int32_t* idx;        // [min(T*k, kIdxInSmemMax)]
   uint8_t* state;      // [T]
   uint8_t* cls;        // [T]
   uint8_t* has_first;  // [G]
@@ -35,12 +38,14 @@ __host__ __device__ inline size_t sel_smem_layout(Dims d, SelSmem* s, unsigned c
     return at;
   };
   const int EN = d.E + d.ns;
+  const int n_idx = d.T * d.k <= kIdxInSmemMax ? d.T * d.k : 0;
   size_t a_mask = take((size_t)d.G * 8 * 4);
   size_t a_hist = take((size_t)kSelWarps * EN * 4);
   size_t a_off = take((size_t)(EN + 1) * 4);
   size_t a_key = take((size_t)d.T * 4);
   size_t a_pos = take((size_t)d.T * 4);
   size_t a_wc = take((size_t)(kSelWarps + 1) * 4);
+  size_t a_idx = take((size_t)n_idx * 4);
   size_t a_state = take((size_t)d.T);
   size_t a_cls = take((size_t)d.T);
   size_t a_hf = take((size_t)d.G);
@@ -51,6 +56,7 @@ __host__ __device__ inline size_t sel_smem_layout(Dims d, SelSmem* s, unsigned c
     s->key = reinterpret_cast<int32_t*>(base + a_key);
     s->pos = reinterpret_cast<int32_t*>(base + a_pos);
     s->warp_cnt = reinterpret_cast<int32_t*>(base + a_wc);
+    s->idx = n_idx ? reinterpret_cast<int32_t*>(base + a_idx) : nullptr;
     s->state = base + a_state;
     s->cls = base + a_cls;
     s->has_first = base + a_hf;
@@ -63,7 +69,8 @@ size_t select_smem_bytes(Dims d) { return sel_smem_layout(d, nullptr, nullptr); 
 __device__ __forceinline__ bool is_decoded(uint8_t s) { return s == TEAM_TOK_NEW || s == TEAM_TOK_CACHED; }
 
 __global__ void __launch_bounds__(kSelThreads, 1)
-k_select(const float* __restrict__ logits, StepPtrs st, Workspace ws, RoutePtrs ex, Dims d, Policy p, int item_tile) {
+k_select(const float* __restrict__ logits, StepPtrs st, Workspace ws, RoutePtrs ex, Dims d, Policy p, int item_tile,
+         int wait_prior) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   SelSmem s;
   sel_smem_layout(d, &s, smem_raw);
@@ -71,11 +78,15 @@ k_select(const float* __restrict__ logits, StepPtrs st, Workspace ws, RoutePtrs 
   const int T = d.T, E = d.E, k = d.k, ns = d.ns, EN = d.E + d.ns;
   const int n_words32 = 8;
   RoutePtrs& r = ws.r;
+  const int S = T * k;
+  // warps taking part in the dispatch walk: enough for 32 slots each, so small steps scan little
+  const int nw = min(kSelWarps, (S + 31) / 32);
+  const bool one_row_per_warp = T <= kSelWarps;
 
-  // ---- stage the step state ------------------------------------------------------------
+  // ---- stage the step state (inputs of the call, not produced by the preceding kernel) ---------
   for (int i = tid; i < d.G * n_words32; i += kSelThreads) s.mask[i] = 0u;
   for (int i = tid; i < d.G; i += kSelThreads) s.has_first[i] = 0;
-  for (int i = tid; i < kSelWarps * EN; i += kSelThreads) s.hist[i] = 0;
+  for (int i = tid; i < nw * EN; i += kSelThreads) s.hist[i] = 0;
   for (int t = tid; t < T; t += kSelThreads) {
     int g = st.group[t], b = st.branch[t];
     if (g < 0 || g >= d.G || b < 0 || b > 255) {
@@ -87,6 +98,13 @@ k_select(const float* __restrict__ logits, StepPtrs st, Workspace ws, RoutePtrs 
     s.pos[t] = st.pos[t];
     s.state[t] = st.tok_state[t];
   }
+  // The logits come from the preceding kernel of the stream.
+  if (wait_prior) asm volatile("griddepcontrol.wait;" ::: "memory");
+  // With at most one row per warp the row's logits are fetched now and stay in registers through
+  // both routing rounds.
+  float keep[kMaxPerLane];
+  float keep_max = 0.f, keep_denom = 1.f;
+  if (one_row_per_warp && warp < T) load_row(logits + (size_t)warp * E, E, lane, keep, keep_max, keep_denom);
   __syncthreads();
 
   // ---- Eq. 4: classification --------------------------------------------------------------
@@ -116,7 +134,8 @@ k_select(const float* __restrict__ logits, StepPtrs st, Workspace ws, RoutePtrs 
     if (c == TEAM_CLS_FIRST) s.has_first[s.key[t] >> 8] = 1;
   }
   __syncthreads();
-  // A group with no first-round row: its masked rows are all routed freely.
+  // A group with no first-round row: its masked rows are all routed freely.  (Each thread only
+  // rewrites rows it classified itself, so the next barrier is the one after round 1's reads.)
   for (int t = tid; t < T; t += kSelThreads)
     if (s.cls[t] == TEAM_CLS_COLD && !s.has_first[s.key[t] >> 8]) s.cls[t] = TEAM_CLS_FIRST;
   __syncthreads();
@@ -127,6 +146,7 @@ k_select(const float* __restrict__ logits, StepPtrs st, Workspace ws, RoutePtrs 
       const uint8_t c = s.cls[t];
       if (round == 1 && c == TEAM_CLS_SKIP) {
         if (lane < k) {
+          if (s.idx) s.idx[t * k + lane] = -1;
           r.topk_idx[t * k + lane] = -1;
           r.topk_w[t * k + lane] = 0.f;
           if (ex.topk_idx) ex.topk_idx[t * k + lane] = -1;
@@ -144,7 +164,14 @@ k_select(const float* __restrict__ logits, StepPtrs st, Workspace ws, RoutePtrs 
       const int g = s.key[t] >> 8;
       float v[kMaxPerLane];
       float row_max, denom;
-      load_row(logits + (size_t)t * E, E, lane, v, row_max, denom);
+      if (one_row_per_warp) {
+#pragma unroll
+        for (int i = 0; i < kMaxPerLane; ++i) v[i] = keep[i];
+        row_max = keep_max;
+        denom = keep_denom;
+      } else {
+        load_row(logits + (size_t)t * E, E, lane, v, row_max, denom);
+      }
       if (ex.probs) {
 #pragma unroll
         for (int i = 0; i < kMaxPerLane; ++i) {
@@ -160,6 +187,7 @@ k_select(const float* __restrict__ logits, StepPtrs st, Workspace ws, RoutePtrs 
       TopkResult tr = warp_topk(v, k, lane);
       const float w = routing_weight(tr, k, lane, row_max, denom, p.norm_topk);
       if (lane < k) {
+        if (s.idx) s.idx[t * k + lane] = tr.idx;
         r.topk_idx[t * k + lane] = tr.idx;
         r.topk_w[t * k + lane] = w;
         if (ex.topk_idx) ex.topk_idx[t * k + lane] = tr.idx;
@@ -174,6 +202,7 @@ k_select(const float* __restrict__ logits, StepPtrs st, Workspace ws, RoutePtrs 
     }
     __syncthreads();
   }
+  const int32_t* idx_src = s.idx ? s.idx : r.topk_idx;
 
   // ---- exports that need no further work ---------------------------------------------------
   for (int t = tid; t < T; t += kSelThreads) {
@@ -191,21 +220,19 @@ k_select(const float* __restrict__ logits, StepPtrs st, Workspace ws, RoutePtrs 
   }
 
   // ---- dispatch: stable counting sort of slots by expert ------------------------------------
-  // Routed slots t*k+j are walked in ascending order, warp w owning a contiguous range, so the
+  // Routed slots t*k+j are walked in ascending order, warp w < nw owning a contiguous range, so the
   // rank of a slot inside its expert is (slots of that expert in earlier warps) + (earlier in this warp).
-  const int S = T * k;
-  const int per_warp = ((S + kSelWarps - 1) / kSelWarps + 31) & ~31;
-  const int lo = warp * per_warp, hi = min(S, lo + per_warp);
-  int32_t* my_hist = s.hist + warp * EN;
+  const int per_warp = ((S + nw - 1) / nw + 31) & ~31;
+  const int lo = min(S, warp * per_warp), hi = warp < nw ? min(S, lo + per_warp) : lo;
+  int32_t* my_hist = s.hist + (warp < nw ? warp : 0) * EN;
   for (int base = lo; base < hi; base += 32) {
     const int slot = base + lane;
-    const int e = (slot < hi) ? r.topk_idx[slot] : -1;
+    const int e = (slot < hi) ? idx_src[slot] : -1;
     const unsigned peers = __match_any_sync(0xffffffffu, e);
     if (e >= 0 && (__ffs(peers) - 1) == lane) my_hist[e] += __popc(peers);
     __syncwarp();
   }
-  // active rows (ascending) and their count; shared experts take every active row
-  int n_rows_active = 0;
+  // number of computed rows; shared experts take every one of them
   {
     int c = 0;
     for (int base = warp * 32; base < T; base += kSelThreads) {
@@ -213,16 +240,19 @@ k_select(const float* __restrict__ logits, StepPtrs st, Workspace ws, RoutePtrs 
       const bool a = t < T && s.cls[t] != TEAM_CLS_SKIP;
       c += __popc(__ballot_sync(0xffffffffu, a));
     }
-    // rows are dealt to warps in an interleaved way; only the total is needed here
     if (lane == 0) s.warp_cnt[warp] = c;
   }
   __syncthreads();
-  for (int w = 0; w < kSelWarps; ++w) n_rows_active += s.warp_cnt[w];
+  int n_rows_active = 0;
+  {
+    const int used = min(kSelWarps, (T + 31) / 32);
+    for (int w = 0; w < used; ++w) n_rows_active += s.warp_cnt[w];
+  }
   // per expert: turn per-warp counts into per-warp starting ranks, total into off[e+1]
   for (int e = tid; e < EN; e += kSelThreads) {
     int run = 0;
     if (e < E) {
-      for (int w = 0; w < kSelWarps; ++w) {
+      for (int w = 0; w < nw; ++w) {
         const int c = s.hist[w * EN + e];
         s.hist[w * EN + e] = run;
         run += c;
@@ -303,7 +333,7 @@ k_select(const float* __restrict__ logits, StepPtrs st, Workspace ws, RoutePtrs 
   // second walk: place the routed slots
   for (int base = lo; base < hi; base += 32) {
     const int slot = base + lane;
-    const int e = (slot < hi) ? r.topk_idx[slot] : -1;
+    const int e = (slot < hi) ? idx_src[slot] : -1;
     const unsigned peers = __match_any_sync(0xffffffffu, e);
     if (e >= 0) {
       const int rank = my_hist[e] + __popc(peers & ((1u << lane) - 1));
@@ -316,25 +346,22 @@ k_select(const float* __restrict__ logits, StepPtrs st, Workspace ws, RoutePtrs 
     __syncwarp();
   }
   // shared experts: slot T*k + s*T + t for every active row t, ascending t.
-  if (ns > 0) {
-    // ordered compaction of active rows by warp 0 (T <= TEAM_MAX_ROWS: at most 64 ballots)
-    if (warp == 0) {
-      int run = 0;
-      for (int base = 0; base < T; base += 32) {
-        const int t = base + lane;
-        const bool a = t < T && s.cls[t] != TEAM_CLS_SKIP;
-        const unsigned b = __ballot_sync(0xffffffffu, a);
-        if (a) {
-          const int rank = run + __popc(b & ((1u << lane) - 1));
-          for (int sh = 0; sh < ns; ++sh) {
-            const int at = s.off[E + sh] + rank;
-            const int slot = T * k + sh * T + t;
-            r.perm[at] = slot;
-            if (ex.perm) ex.perm[at] = slot;
-          }
+  if (ns > 0 && warp == kSelWarps - 1) {
+    int run = 0;
+    for (int base = 0; base < T; base += 32) {
+      const int t = base + lane;
+      const bool a = t < T && s.cls[t] != TEAM_CLS_SKIP;
+      const unsigned b = __ballot_sync(0xffffffffu, a);
+      if (a) {
+        const int rank = run + __popc(b & ((1u << lane) - 1));
+        for (int sh = 0; sh < ns; ++sh) {
+          const int at = s.off[E + sh] + rank;
+          const int slot = T * k + sh * T + t;
+          r.perm[at] = slot;
+          if (ex.perm) ex.perm[at] = slot;
         }
-        run += __popc(b);
       }
+      run += __popc(b);
     }
   }
   // unused tail of perm
@@ -353,7 +380,7 @@ cudaError_t configure_select(Dims max_dims) {
 cudaError_t launch_select(const float* logits, StepPtrs st, Workspace ws, RoutePtrs ex, Dims d, Policy p,
                           int item_tile, cudaStream_t s) {
   const size_t smem = select_smem_bytes(d);
-  k_select<<<1, kSelThreads, smem, s>>>(logits, st, ws, ex, d, p, item_tile);
+  k_select<<<1, kSelThreads, smem, s>>>(logits, st, ws, ex, d, p, item_tile, 0);
   return cudaGetLastError();
 }
 
