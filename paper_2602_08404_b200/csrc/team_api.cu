@@ -103,16 +103,7 @@ team::RoutePtrs export_ptrs(const team_routing* r) {
 
 bool use_tensor_path(const team_ctx* ctx) { return ctx->cfg.dtype == TEAM_DTYPE_BF16 && !ctx->force_simt; }
 
-int pick_item_tile(const team_config& c) {
-  const char* env = getenv("TEAM_ITEM_TILE");
-  if (env != nullptr) {
-    const int v = atoi(env);
-    if (v == 32 || v == 64 || v == 128) return v;
-  }
-  if (c.max_rows <= 64) return 32;
-  if (c.max_rows <= 256) return 64;
-  return 128;
-}
+int pick_item_tile(const team_config& c) { return team::experts_tc_item_tile(c.max_rows, c.hidden); }
 
 }  // namespace
 
@@ -163,7 +154,7 @@ int team_create(const team_config* cfg, team_ctx** out) {
   ctx->item_tile = pick_item_tile(*cfg);
   e = team::configure_router(cfg->dtype, cfg->hidden);
   if (e == cudaSuccess) e = team::configure_select(dims_of(*cfg, cfg->max_rows));
-  if (e == cudaSuccess && cfg->dtype == TEAM_DTYPE_BF16) e = team::configure_experts_tc(ctx->item_tile);
+  if (e == cudaSuccess && cfg->dtype == TEAM_DTYPE_BF16) e = team::configure_experts_tc(ctx->item_tile, cfg->hidden);
   if (e != cudaSuccess) {
     delete ctx;
     return TEAM_ERR_CUDA;
@@ -180,8 +171,13 @@ int team_create(const team_config* cfg, team_ctx** out) {
   const size_t o_logits = take(T * E * 4), o_idx = take(T * k * 4), o_w = take(T * k * 4), o_margin = take(T * 4);
   const size_t o_cls = take(T), o_gm = take((size_t)cfg->max_groups * ((E + 63) / 64) * 8);
   const size_t o_cnt = take(EN * 4), o_off = take((EN + 1) * 4), o_perm = take(S * 4), o_act_list = take(EN * 4);
-  const size_t o_scal = take(64), o_items = take((EN + S / 32 + 2) * sizeof(team::WorkItem));
+  const size_t o_scal = take(64), o_items = take((EN + S / 16 + 2) * sizeof(team::WorkItem));
   const size_t o_act = take(cfg->dtype == TEAM_DTYPE_F32 ? S * cfg->inter * 4 : 256);
+  const bool bf16 = cfg->dtype == TEAM_DTYPE_BF16;
+  const size_t max_items = EN + S / ctx->item_tile + 2;
+  const size_t n_flags = bf16 ? max_items * (cfg->inter / 64) : 0;
+  const size_t o_flags = take(n_flags * 4 + 4);
+  const size_t o_actg = take(bf16 ? max_items * ctx->item_tile * cfg->inter * 2 : 256);
   ctx->ws_bytes = off;
   e = cudaMalloc(&ctx->ws_base, ctx->ws_bytes);
   if (e != cudaSuccess) {
@@ -209,6 +205,9 @@ int team_create(const team_config* cfg, team_ctx** out) {
   ws.status = scal + 4;
   ws.items = reinterpret_cast<team::WorkItem*>(b + o_items);
   ws.act = reinterpret_cast<float*>(b + o_act);
+  ws.win_flags = reinterpret_cast<int32_t*>(b + o_flags);
+  ws.n_flags = (int32_t)n_flags;
+  ws.act_g = reinterpret_cast<__nv_bfloat16*>(b + o_actg);
   *out = ctx;
   return TEAM_OK;
 }

@@ -70,6 +70,9 @@ struct Workspace {
   int32_t* n_items;     // [1]
   float* act;           // fp32 path: [max_rows*(k+ns), I] SwiGLU activations
   int32_t* status;      // [2] code, detail
+  __nv_bfloat16* act_g; // bf16 path: [items][item_tile][I] activations published between CTAs
+  int32_t* win_flags;   // bf16 path: [n_flags] groups published per 64-column window, zeroed per step
+  int32_t n_flags;
 };
 
 __device__ __forceinline__ void set_status(int32_t* status, int code, int detail) {
@@ -93,7 +96,8 @@ __device__ __forceinline__ void slot_row_weight(int slot, int T, int k, const fl
 // Kernel launchers (host side), one per translation unit.
 cudaError_t configure_router(int dtype, int hidden);
 cudaError_t configure_select(Dims max_dims);
-cudaError_t configure_experts_tc(int item_tile);
+cudaError_t configure_experts_tc(int item_tile, int hidden);
+int experts_tc_item_tile(int max_rows, int hidden);
 cudaError_t launch_router_logits(const void* x, int dtype, const float* w_router, const uint8_t* tok_state,
                                  float* logits, float* y_zero, Dims d, int flags, cudaStream_t s);
 cudaError_t launch_router_topk(const float* logits, const uint8_t* tok_state, RoutePtrs out, Dims d, Policy p,

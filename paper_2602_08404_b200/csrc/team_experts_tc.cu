@@ -1,29 +1,41 @@
 // Grouped SwiGLU expert kernel for bf16 weights on sm_100a: TMA-staged weight tiles, tcgen05.mma
 // with accumulators in tensor memory, SwiGLU and the routing-weight scatter-combine fused in.
 //
-// Work is measured in "groups": 16 consecutive columns of one work item's intermediate dimension
-// (a work item is a run of up to NT token-slots of one activated expert, built by the selection
-// kernel).  A group costs the same HBM bytes everywhere (16 gate rows + 16 up rows + a 16-column
-// strip of W_down), so the global list of groups is cut into one contiguous range per CTA and every
-// SM streams the same number of bytes (+- one group).  A CTA walks its range in chunks: the part of
-// the range that falls into one 64-column window of one item (1 to 4 groups).  For a chunk it
-//   phase 1  streams the chunk's W_gate / W_up rows against the gathered token rows,
-//            D1[128, N] = A[128, H] * X[N, H]^T  (weights on M, tokens on N).  One 4-D TMA box per
-//            64-wide k-block delivers the rows already interleaved as [group][gate 16 | up 16], so a
-//            gate row and its up row sit in the same warp's TMEM lanes.
-//   SwiGLU   reads D1 from TMEM, a = silu(gate) * up, writes a as bf16 into shared memory in the
-//            K-major 128B-swizzled layout the tensor core reads as a B operand
-//   phase 2  streams W_down[e, :, window] in 128-row tiles: D2[128, N] = Wd_tile[128, cols] * a[N, cols]^T
-//            over the chunk's columns, multiplies by the slot's routing weight and adds into y[row, h]
-//            with fp32 reductions.
-// Every weight byte of an activated expert is read from HBM once per step (two CTAs that share a
-// window read its W_down tiles at the same time, odd CTAs walking their range backwards, so the
-// second read is served by L2); nothing but y is written.
+// Unit of work and balance.  A work item is a run of up to NT token-slots of one activated expert
+// (built by the selection kernel).  Its intermediate dimension is cut into "groups" of 16 columns.
+// A group costs the same HBM bytes everywhere:
+//     phase 1   16 rows of W_gate + 16 rows of W_up (full hidden width), and
+//     phase 2   a quarter of the W_down tiles of the group's 64-column "window": the g-th group of
+//               a window owns the hidden-row tiles [g*HT/4, (g+1)*HT/4) of that window,
+// so the global list of groups is cut into one contiguous range per CTA and every SM streams the
+// same number of bytes (+- one group), every TMA box is a full 128-byte-row box and every weight
+// byte of an activated expert is requested exactly once per step.
+//
+// A CTA walks its range in super-chunks of up to kScWindows windows of one item:
+//   phase 1   D1[128, N] = A[128, H] * X[N, H]^T per tile of up to 4 groups (weights on M, tokens on
+//             N).  One 4-D TMA box per 64-wide k-block delivers the rows already interleaved as
+//             [group][gate 16 | up 16], so a gate row and its up row sit in the same warp's TMEM lanes.
+//   SwiGLU    a = silu(gate) * up from TMEM, rounded to bf16 and published to a small global
+//             scratch [item][token][I]; a per-window counter says how many of its 4 groups are there.
+//   phase 2   for each of its groups' W_down tiles: D2[128, N] = Wd[128, 64] * a[N, 64]^T over the
+//             whole window (the window's activations are read back from the scratch once all four
+//             groups are published, whichever CTAs computed them), times the slot's routing weight,
+//             added into y[row, h] with fp32 reductions.
+// A window cut by a range boundary is shared by neighbouring CTAs.  Its phase-2 tiles wait for the
+// neighbours' activations; the tiles of a CTA's first (head) window are therefore done last.  No
+// publish ever waits on another CTA, so the waits cannot form a cycle; the launch is cooperative so
+// that all CTAs are resident, and every wait is bounded.
+//
+// Two operand modes:
+//   resident  (T <= 16 rows, N = 16): all rows of x sit in shared memory for the whole kernel and
+//             every expert is applied to all of them; rows not routed to the expert get weight 0.
+//             With no per-stage token tile, partial tiles (1-2 groups) pack several k-blocks into
+//             one 16 KB stage.
+//   gather    (N = 16..NT): a warp gathers the item's token rows per k-block with cp.async.
 //
 // Warp roles (256 threads): warp 0 = TMA producer, warp 1 = MMA issuer + TMEM owner, warp 2 = token
-// gather (cp.async into the swizzled B tile), warp 3 idle, warps 4-7 = epilogue (one TMEM lane
-// quarter each).  All waits are bounded; on expiry the kernel records TEAM_ERR_TIMEOUT, drains and
-// frees its tensor memory.
+// gather, warp 3 = activation-window loader, warps 4-7 = epilogue (one TMEM lane quarter each).
+// On a wait's expiry the kernel records TEAM_ERR_TIMEOUT, drains and frees its tensor memory.
 #include <cuda.h>
 
 #include "team_common.cuh"
@@ -34,18 +46,34 @@ constexpr int kTcThreads = 256;
 constexpr int kATileBytes = 128 * 128;          // 128 rows x 64 bf16
 constexpr int kGroupCols = 16;                  // intermediate columns per group (the unit of balance)
 constexpr int kWindowCols = 64;                 // columns per window (one 128-byte swizzle row of W_down)
+constexpr int kActBufs = 2;                     // activation windows staged in shared memory
+constexpr int kResidentRows = 16;               // N of the resident mode
+constexpr int kResidentMaxHidden = 2048;        // 16 rows x H x 2 B must fit beside the ring
 constexpr unsigned long long kWaitCycles = 2000000000ull;   // ~1 s at 2 GHz
 
-template <int NT>
+template <int NT, bool RES>
 struct TcCfg {
-  static constexpr int kBTileBytes = NT * 128;
+  static constexpr int kBTileBytes = RES ? 0 : NT * 128;
   static constexpr int kStageBytes = kATileBytes + kBTileBytes;
-  static constexpr int kStages = (NT <= 32) ? 10 : (NT <= 64 ? 8 : 6);
-  static constexpr int kActBytes = NT * 128;
-  static constexpr int kTmemCols = (3 * NT <= 128) ? 128 : (3 * NT <= 256 ? 256 : 512);
-  static constexpr int kBarBytes = (3 * kStages + 8) * 8;
-  static constexpr int kTableBytes = 4 * NT * 8 + NT * 4;   // per-epilogue-warp (row, weight) + gather rows
-  static constexpr int kSmemBytes = 1024 + kStages * kStageBytes + kActBytes + kBarBytes + kTableBytes + 64;
+  static constexpr int kStages = RES ? 9 : (NT <= 32 ? 10 : (NT <= 64 ? 8 : 5));
+  static constexpr int kLag = kStages >= 8 ? 5 : 3;             // gather stages kept in flight
+  static constexpr int kActBytes = NT * 128;                    // NT tokens x 64 columns bf16
+  static constexpr int kScWindows = NT <= 32 ? 3 : 2;           // windows per super-chunk = phase-1 accumulators
+  static constexpr int kAcc2 = NT <= 16 ? 8 : (NT <= 32 ? 4 : 2);
+  static constexpr int kTmemUsed = (kScWindows + kAcc2) * NT;
+  static constexpr int kTmemCols = kTmemUsed <= 128 ? 128 : (kTmemUsed <= 256 ? 256 : 512);
+  static constexpr int kNumBars = 3 * kStages + kScWindows + 1 + 2 * kActBufs + 2 * kAcc2 + 2;
+  static constexpr int kBarBytes = ((kNumBars * 8 + 15) / 16) * 16;
+  static constexpr int kTableBytes = 4 * NT * 8 + NT * 4;       // per-epilogue-warp (row, weight) + gather rows
+  static constexpr int kRingBytes = kStages * kStageBytes;
+  // Partial resident tiles are read by the tensor core as full 128-row tiles starting at a 4 KB
+  // multiple inside the stage, i.e. up to 12 KB past the ring's end: the resident rows (or padding)
+  // sit there.
+  static __host__ __device__ int x_bytes(int H) { return RES ? kResidentRows * H * 2 : 0; }
+  static __host__ __device__ int pad_bytes(int H) { return RES ? (x_bytes(H) >= 12288 ? 0 : 12288 - x_bytes(H)) : 0; }
+  static __host__ __device__ int smem_bytes(int H) {
+    return 1024 + kRingBytes + x_bytes(H) + pad_bytes(H) + kActBufs * kActBytes + kBarBytes + kTableBytes + 64;
+  }
 };
 
 // ---------------------------------------------------------------------------------------------
@@ -151,6 +179,12 @@ __device__ __forceinline__ void tmem_ld8(uint32_t taddr, float (&v)[8]) {
   v[4] = __uint_as_float(r4); v[5] = __uint_as_float(r5); v[6] = __uint_as_float(r6); v[7] = __uint_as_float(r7);
 }
 
+__device__ __forceinline__ int ld_acquire(const int32_t* p) {
+  int v;
+  asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+
 // ---------------------------------------------------------------------------------------------
 // The kernel
 // ---------------------------------------------------------------------------------------------
@@ -160,6 +194,8 @@ struct TcArgs {
   const float* topk_w;         // [T, k]
   const WorkItem* items;
   const int32_t* n_items;
+  __nv_bfloat16* act_g;        // [items][NT][I] published activations
+  int32_t* win_flags;          // [items * I/64] groups published per window (zeroed by the selection kernel)
   float* y;                    // [T, H], pre-zeroed rows of computed tokens
   int32_t* status;
   Dims d;
@@ -173,54 +209,101 @@ struct TcMaps {
   CUtensorMap down;
 };
 
-// One step of a CTA's walk over its group range.
-struct Chunk {
-  int item;     // work item
-  int window;   // 64-column window of the intermediate dimension
-  int g0;       // first group of the window that belongs to the chunk (0..3)
-  int g;        // groups in the chunk (1..4)
+// The sequence of operations a CTA performs on its group range [lo, hi); every warp role walks the
+// same sequence.  Group indices are global (item * NG + group in item); since NG is a multiple of
+// 4, window W = group >> 2 never straddles two items.
+enum { OP_P1 = 0, OP_PUBLISH = 1, OP_P2 = 2 };
+struct Op {
+  int kind;
+  int item;     // P1, P2: work item
+  int j, g;     // P1: first group inside the item, number of groups (1..4)
+  int tile;     // P1: accumulator index inside the super-chunk
+  int W;        // P2: global window index
+  int a, b;     // P2: the CTA's groups [a, b) of the window (0..4); PUBLISH: the super-chunk [a, b)
 };
 
-struct ChunkWalker {
-  long long lo, hi, cur;
-  int NG;
-  bool reverse;
-  __device__ ChunkWalker(long long lo_, long long hi_, int ng, bool rev)
-      : lo(lo_), hi(hi_), cur(rev ? hi_ : lo_), NG(ng), reverse(rev) {}
-  __device__ bool next(Chunk& c) {
-    if (!reverse) {
-      if (cur >= hi) return false;
-      const long long item = cur / NG;
-      const int j = (int)(cur - item * NG);
-      long long end = item * NG + (j / 4 + 1) * 4;
-      if (end > hi) end = hi;
-      c.item = (int)item; c.window = j / 4; c.g0 = j % 4; c.g = (int)(end - cur);
-      cur = end;
-    } else {
-      if (cur <= lo) return false;
-      const long long last = cur - 1, item = last / NG;
-      const int j = (int)(last - item * NG);
-      long long begin = item * NG + (j / 4) * 4;
-      if (begin < lo) begin = lo;
-      c.item = (int)item; c.window = j / 4; c.g0 = (int)(begin - item * NG) % 4; c.g = (int)(cur - begin);
-      cur = begin;
+struct Walker {
+  int lo, hi, NG, HT, scg;
+  int s_lo, s_hi, t0, W, tile, state;
+  __device__ Walker(int lo_, int hi_, int ng, int ht, int sc_groups)
+      : lo(lo_), hi(hi_), NG(ng), HT(ht), scg(sc_groups), s_lo(lo_), s_hi(lo_), t0(0), W(0), tile(0), state(0) {}
+  __device__ bool defer_head() const { return (lo & 3) != 0; }
+  __device__ bool p2(Op& op, int w, int from, int to) const {
+    op.kind = OP_P2;
+    op.W = w;
+    op.a = max(from, 4 * w) - 4 * w;
+    op.b = min(to, 4 * w + 4) - 4 * w;
+    op.item = (4 * w) / NG;
+    return op.a * HT / 4 < op.b * HT / 4;     // jobs without a tile are skipped
+  }
+  __device__ bool next(Op& op) {
+    for (;;) {
+      switch (state) {
+        case 0: {                                   // open the next super-chunk
+          if (s_hi >= hi) { state = 4; break; }
+          s_lo = s_hi;
+          const int item_end = (s_lo / NG + 1) * NG;
+          s_hi = min(hi, min(item_end, (s_lo & ~3) + scg));
+          t0 = s_lo;
+          tile = 0;
+          state = 1;
+          break;
+        }
+        case 1:                                     // phase-1 tiles of up to 4 groups
+          if (t0 >= s_hi) { state = 2; break; }
+          op.kind = OP_P1;
+          op.item = t0 / NG;
+          op.j = t0 - op.item * NG;
+          op.g = min(4, s_hi - t0);
+          op.tile = tile++;
+          t0 += op.g;
+          return true;
+        case 2:
+          op.kind = OP_PUBLISH;
+          op.a = s_lo;
+          op.b = s_hi;
+          W = s_lo >> 2;
+          state = 3;
+          return true;
+        case 3: {                                   // phase-2 jobs, one per window touched
+          if (W > ((s_hi - 1) >> 2)) { state = 0; break; }
+          const int w = W++;
+          if (w == (lo >> 2) && defer_head()) break;
+          if (p2(op, w, s_lo, s_hi)) return true;
+          break;
+        }
+        case 4:                                     // the head window, shared with the previous CTA, comes last
+          state = 5;
+          if (lo < hi && defer_head() && p2(op, lo >> 2, lo, hi)) return true;
+          break;
+        default:
+          return false;
+      }
     }
-    return true;
   }
 };
 
-template <int NT>
+template <int NT, bool RES>
 __global__ void __launch_bounds__(kTcThreads, 1)
 k_experts_tc(const __grid_constant__ TcMaps maps, TcArgs a) {
-  using C = TcCfg<NT>;
+  using C = TcCfg<NT, RES>;
   extern __shared__ unsigned char smem_dyn[];
+  const Dims d = a.d;
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~uintptr_t(1023));
-  unsigned char* act_tile = smem + C::kStages * C::kStageBytes;
-  uint64_t* bars = reinterpret_cast<uint64_t*>(act_tile + C::kActBytes);
+  unsigned char* x_res = smem + C::kRingBytes;                                   // resident rows: [H/64][16][128 B]
+  unsigned char* act_buf = x_res + C::x_bytes(d.H) + C::pad_bytes(d.H);          // [kActBufs][NT][128 B]
+  uint64_t* bars = reinterpret_cast<uint64_t*>(act_buf + kActBufs * C::kActBytes);
   uint64_t* bar_fullA = bars;
   uint64_t* bar_fullB = bars + C::kStages;
   uint64_t* bar_empty = bars + 2 * C::kStages;
-  uint64_t* bar_misc = bars + 3 * C::kStages;   // 0 acc1_full, 1 acc1_empty, 2 act_ready, 3-4 acc2_full, 5-6 acc2_empty
+  uint64_t* bar_acc1_full = bars + 3 * C::kStages;                 // [kScWindows]
+  uint64_t* bar_acc1_empty = bar_acc1_full + C::kScWindows;        // [1]
+  uint64_t* bar_act_full = bar_acc1_empty + 1;                     // [kActBufs]
+  uint64_t* bar_act_empty = bar_act_full + kActBufs;               // [kActBufs]
+  uint64_t* bar_acc2_full = bar_act_empty + kActBufs;              // [kAcc2]
+  uint64_t* bar_acc2_empty = bar_acc2_full + C::kAcc2;             // [kAcc2]
+  uint64_t* bar_x = bar_acc2_empty + C::kAcc2;                     // [1] resident rows staged
+  uint64_t* bar_pub = bar_x + 1;                                   // [1] a super-chunk's activations stored
   int32_t* tbl_row = reinterpret_cast<int32_t*>(reinterpret_cast<unsigned char*>(bars) + C::kBarBytes);   // [4][NT]
   float* tbl_wt = reinterpret_cast<float*>(tbl_row + 4 * NT);                                             // [4][NT]
   int32_t* gather_row = reinterpret_cast<int32_t*>(tbl_wt + 4 * NT);                                      // [NT]
@@ -228,10 +311,11 @@ k_experts_tc(const __grid_constant__ TcMaps maps, TcArgs a) {
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const Dims d = a.d;
   const int KB = d.H / 64;          // k-blocks of phase 1
-  const int HT = d.H / 128;         // row tiles of phase 2
+  const int HT = d.H / 128;         // row tiles of W_down
   const int NG = d.I / kGroupCols;  // groups per work item
+  const int WPI = NG / 4;           // windows per work item
+  constexpr int kXLoaders = kTcThreads - 64;   // warps 2-7 stage the resident rows
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < C::kStages; ++s) {
@@ -239,13 +323,18 @@ k_experts_tc(const __grid_constant__ TcMaps maps, TcArgs a) {
       mbar_init(smem_u32(bar_fullB + s), 32);
       mbar_init(smem_u32(bar_empty + s), 1);
     }
-    mbar_init(smem_u32(bar_misc + 0), 1);
-    mbar_init(smem_u32(bar_misc + 1), 128);
-    mbar_init(smem_u32(bar_misc + 2), 128);
-    mbar_init(smem_u32(bar_misc + 3), 1);
-    mbar_init(smem_u32(bar_misc + 4), 1);
-    mbar_init(smem_u32(bar_misc + 5), 128);
-    mbar_init(smem_u32(bar_misc + 6), 128);
+    for (int i = 0; i < C::kScWindows; ++i) mbar_init(smem_u32(bar_acc1_full + i), 1);
+    mbar_init(smem_u32(bar_acc1_empty), 128);
+    for (int i = 0; i < kActBufs; ++i) {
+      mbar_init(smem_u32(bar_act_full + i), 32);
+      mbar_init(smem_u32(bar_act_empty + i), 1);
+    }
+    for (int i = 0; i < C::kAcc2; ++i) {
+      mbar_init(smem_u32(bar_acc2_full + i), 1);
+      mbar_init(smem_u32(bar_acc2_empty + i), 128);
+    }
+    mbar_init(smem_u32(bar_x), kXLoaders);
+    mbar_init(smem_u32(bar_pub), 128);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -259,41 +348,66 @@ k_experts_tc(const __grid_constant__ TcMaps maps, TcArgs a) {
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
-  const uint32_t tmem_acc1 = tmem_base;
 
-  // This CTA's contiguous range of groups; odd CTAs walk it backwards so that the two CTAs sharing a
-  // window touch its W_down tiles at the same time.
+  // This CTA's contiguous range of groups.
   const long long n_groups = (long long)(*a.n_items) * NG;
-  const long long g_lo = n_groups * blockIdx.x / gridDim.x, g_hi = n_groups * (blockIdx.x + 1) / gridDim.x;
-  const bool reverse = (blockIdx.x & 1) != 0;
+  const int g_lo = (int)(n_groups * blockIdx.x / gridDim.x), g_hi = (int)(n_groups * (blockIdx.x + 1) / gridDim.x);
+  constexpr int kScGroups = C::kScWindows * 4;
+
+  // ------------------------------ resident rows (warps 2-7) ------------------------------
+  if (RES && warp >= 2) {
+    const int tid = threadIdx.x - 64;
+    const int per_row = d.H / 8;                       // 16-byte pieces per row
+    if (g_lo < g_hi) {
+      for (int c = tid; c < kResidentRows * per_row; c += kXLoaders) {
+        const int r = c / per_row, cc = c - r * per_row, kb = cc >> 3, ch = cc & 7;
+        const uint32_t dst = smem_u32(x_res + kb * (kResidentRows * 128) + r * 128 + ((ch ^ (r & 7)) << 4));
+        if (r < d.T) {
+          const __nv_bfloat16* src = a.x + (size_t)r * d.H + cc * 8;
+          asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+        } else {
+          asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(dst), "r"(0) : "memory");
+        }
+      }
+      asm volatile("cp.async.commit_group;" ::: "memory");
+      asm volatile("cp.async.wait_group 0;" ::: "memory");
+      fence_async_smem();
+    }
+    mbar_arrive(smem_u32(bar_x));
+  }
 
   if (warp == 0) {
     // ------------------------------ TMA producer ------------------------------
     if (lane == 0) {
       uint32_t it = 0;
       bool ok = true;
-      ChunkWalker walk(g_lo, g_hi, NG, reverse);
-      Chunk c;
-      while (ok && walk.next(c)) {
-        const WorkItem item = a.items[c.item];
-        const int col0 = c.window * kWindowCols + c.g0 * kGroupCols;
-        const int grp = (item.e * d.I + col0) / kGroupCols;          // coordinate in units of 16 rows
-        const CUtensorMap* gu = &maps.gu[c.g - 1];
-        const uint32_t bytes1 = (uint32_t)c.g * 4096u;
-        for (int kb = 0; kb < KB; ++kb, ++it) {
-          const uint32_t s = it % C::kStages, par = (it / C::kStages) & 1;
-          if (!(ok = mbar_wait(smem_u32(bar_empty + s), par ^ 1, abort_flag, a.status, 1))) break;
-          const uint32_t dst = smem_u32(smem + s * C::kStageBytes), bar = smem_u32(bar_fullA + s);
-          mbar_arrive_expect_tx(bar, bytes1);
-          tma_load_4d(dst, gu, kb * 64, 0, 0, grp, bar);
-        }
-        if (!ok) break;
-        for (int ht = 0; ht < HT; ++ht, ++it) {
-          const uint32_t s = it % C::kStages, par = (it / C::kStages) & 1;
-          if (!(ok = mbar_wait(smem_u32(bar_empty + s), par ^ 1, abort_flag, a.status, 2))) break;
-          const uint32_t dst = smem_u32(smem + s * C::kStageBytes), bar = smem_u32(bar_fullA + s);
-          mbar_arrive_expect_tx(bar, kATileBytes);
-          tma_load_2d(dst, &maps.down, c.window * kWindowCols, item.e * d.H + ht * 128, bar);
+      Walker walk(g_lo, g_hi, NG, HT, kScGroups);
+      Op op;
+      while (ok && walk.next(op)) {
+        if (op.kind == OP_PUBLISH) continue;
+        const WorkItem item = a.items[op.item];
+        if (op.kind == OP_P1) {
+          const int grp = item.e * NG + op.j;                       // coordinate in units of 16 rows
+          const CUtensorMap* gu = &maps.gu[op.g - 1];
+          const uint32_t box_bytes = (uint32_t)op.g * 4096u;
+          const int nb = RES ? (op.g == 1 ? 4 : (op.g == 2 ? 2 : 1)) : 1;   // k-blocks per stage
+          for (int kb0 = 0; kb0 < KB; kb0 += nb, ++it) {
+            const uint32_t s = it % C::kStages, par = (it / C::kStages) & 1;
+            if (!(ok = mbar_wait(smem_u32(bar_empty + s), par ^ 1, abort_flag, a.status, 1))) break;
+            const uint32_t dst = smem_u32(smem + s * C::kStageBytes), bar = smem_u32(bar_fullA + s);
+            const int n = min(nb, KB - kb0);
+            mbar_arrive_expect_tx(bar, (uint32_t)n * box_bytes);
+            for (int i = 0; i < n; ++i) tma_load_4d(dst + i * box_bytes, gu, (kb0 + i) * 64, 0, 0, grp, bar);
+          }
+        } else {
+          const int w = op.W - op.item * WPI;
+          for (int ht = op.a * HT / 4; ht < op.b * HT / 4; ++ht, ++it) {
+            const uint32_t s = it % C::kStages, par = (it / C::kStages) & 1;
+            if (!(ok = mbar_wait(smem_u32(bar_empty + s), par ^ 1, abort_flag, a.status, 2))) break;
+            const uint32_t dst = smem_u32(smem + s * C::kStageBytes), bar = smem_u32(bar_fullA + s);
+            mbar_arrive_expect_tx(bar, kATileBytes);
+            tma_load_2d(dst, &maps.down, w * kWindowCols, item.e * d.H + ht * 128, bar);
+          }
         }
       }
       if (*abort_flag) {
@@ -310,176 +424,285 @@ k_experts_tc(const __grid_constant__ TcMaps maps, TcArgs a) {
   } else if (warp == 1) {
     // ------------------------------ MMA issuer ------------------------------
     if (lane == 0) {
-      uint32_t it = 0, chunk_i = 0, t2 = 0, bphase = 0;
+      uint32_t it = 0, sc_i = 0, t2 = 0, jc = 0, bphase = 0;
       bool ok = true;
-      const uint64_t act_desc = make_kmajor_sw128_desc(smem_u32(act_tile));
-      ChunkWalker walk(g_lo, g_hi, NG, reverse);
-      Chunk c;
-      for (; ok && walk.next(c); ++chunk_i) {
-        const WorkItem item = a.items[c.item];
-        const int N = (item.n + 15) & ~15;
+      if (RES) ok = mbar_wait(smem_u32(bar_x), 0, abort_flag, a.status, 13);
+      Walker walk(g_lo, g_hi, NG, HT, kScGroups);
+      Op op;
+      while (ok && walk.next(op)) {
+        if (op.kind == OP_PUBLISH) { ++sc_i; continue; }
+        const WorkItem item = a.items[op.item];
+        const int N = RES ? kResidentRows : ((item.n + 15) & ~15);
         const uint32_t idesc = make_idesc_bf16(N);
-        if (!(ok = mbar_wait(smem_u32(bar_misc + 1), (chunk_i & 1) ^ 1, abort_flag, a.status, 3))) break;
-        tc_fence_after();
-        for (int kb = 0; kb < KB; ++kb, ++it) {
-          const uint32_t s = it % C::kStages, par = (it / C::kStages) & 1;
-          if (!(ok = mbar_wait(smem_u32(bar_fullA + s), par, abort_flag, a.status, 4))) break;
-          if (!(ok = mbar_wait(smem_u32(bar_fullB + s), (bphase >> s) & 1, abort_flag, a.status, 5))) break;
-          bphase ^= 1u << s;
-          tc_fence_after();
-          const uint32_t sa = smem_u32(smem + s * C::kStageBytes);
-          const uint64_t da = make_kmajor_sw128_desc(sa), db = make_kmajor_sw128_desc(sa + kATileBytes);
+        if (op.kind == OP_P1) {
+          if (op.tile == 0) {
+            // the epilogue has read the previous super-chunk's accumulators
+            if (!(ok = mbar_wait(smem_u32(bar_acc1_empty), (sc_i & 1) ^ 1, abort_flag, a.status, 3))) break;
+            tc_fence_after();
+          }
+          const uint32_t acc1 = tmem_base + op.tile * NT;
+          const uint32_t box_bytes = (uint32_t)op.g * 4096u;
+          const int nb = RES ? (op.g == 1 ? 4 : (op.g == 2 ? 2 : 1)) : 1;
+          for (int kb0 = 0; kb0 < KB; kb0 += nb, ++it) {
+            const uint32_t s = it % C::kStages, par = (it / C::kStages) & 1;
+            if (!(ok = mbar_wait(smem_u32(bar_fullA + s), par, abort_flag, a.status, 4))) break;
+            if (!RES) {
+              if (!(ok = mbar_wait(smem_u32(bar_fullB + s), (bphase >> s) & 1, abort_flag, a.status, 5))) break;
+              bphase ^= 1u << s;
+            }
+            tc_fence_after();
+            const uint32_t sa = smem_u32(smem + s * C::kStageBytes);
+            const int n = min(nb, KB - kb0);
+            for (int i = 0; i < n; ++i) {
+              const int kb = kb0 + i;
+              const uint64_t da = make_kmajor_sw128_desc(sa + i * box_bytes);
+              const uint64_t db = make_kmajor_sw128_desc(RES ? smem_u32(x_res) + kb * (kResidentRows * 128)
+                                                             : sa + kATileBytes);
 #pragma unroll
-          for (int k4 = 0; k4 < 4; ++k4)
-            tc_mma(tmem_acc1, da + 2 * k4, db + 2 * k4, idesc, (kb | k4) != 0);
-          tc_commit(smem_u32(bar_empty + s));
-        }
-        if (!ok) break;
-        tc_commit(smem_u32(bar_misc + 0));
-        if (!(ok = mbar_wait(smem_u32(bar_misc + 2), chunk_i & 1, abort_flag, a.status, 6))) break;
-        tc_fence_after();
-        for (int ht = 0; ht < HT; ++ht, ++it, ++t2) {
-          const uint32_t b = t2 & 1, u = t2 >> 1;
-          if (!(ok = mbar_wait(smem_u32(bar_misc + 5 + b), (u & 1) ^ 1, abort_flag, a.status, 7))) break;
-          const uint32_t s = it % C::kStages, par = (it / C::kStages) & 1;
-          if (!(ok = mbar_wait(smem_u32(bar_fullA + s), par, abort_flag, a.status, 8))) break;
+              for (int k4 = 0; k4 < 4; ++k4) tc_mma(acc1, da + 2 * k4, db + 2 * k4, idesc, (kb | k4) != 0);
+            }
+            tc_commit(smem_u32(bar_empty + s));
+          }
+          if (!ok) break;
+          tc_commit(smem_u32(bar_acc1_full + op.tile));
+        } else {
+          const uint32_t ab = jc % kActBufs;
+          if (!(ok = mbar_wait(smem_u32(bar_act_full + ab), (jc / kActBufs) & 1, abort_flag, a.status, 6))) break;
           tc_fence_after();
-          const uint64_t da = make_kmajor_sw128_desc(smem_u32(smem + s * C::kStageBytes));
-          const uint32_t acc2 = tmem_base + NT * (1 + b);
-          // the chunk's columns are k-steps g0 .. g0+g-1 of the window tile and 0 .. g-1 of the activation tile
-          for (int kk = 0; kk < c.g; ++kk) tc_mma(acc2, da + 2 * (c.g0 + kk), act_desc + 2 * kk, idesc, kk != 0);
-          tc_commit(smem_u32(bar_empty + s));
-          tc_commit(smem_u32(bar_misc + 3 + b));
+          const uint64_t act_desc = make_kmajor_sw128_desc(smem_u32(act_buf + ab * C::kActBytes));
+          for (int ht = op.a * HT / 4; ht < op.b * HT / 4; ++ht, ++it, ++t2) {
+            const uint32_t b = t2 % C::kAcc2, u = t2 / C::kAcc2;
+            if (!(ok = mbar_wait(smem_u32(bar_acc2_empty + b), (u & 1) ^ 1, abort_flag, a.status, 7))) break;
+            const uint32_t s = it % C::kStages, par = (it / C::kStages) & 1;
+            if (!(ok = mbar_wait(smem_u32(bar_fullA + s), par, abort_flag, a.status, 8))) break;
+            tc_fence_after();
+            const uint64_t da = make_kmajor_sw128_desc(smem_u32(smem + s * C::kStageBytes));
+            const uint32_t acc2 = tmem_base + (C::kScWindows + b) * NT;
+#pragma unroll
+            for (int kk = 0; kk < 4; ++kk) tc_mma(acc2, da + 2 * kk, act_desc + 2 * kk, idesc, kk != 0);
+            tc_commit(smem_u32(bar_empty + s));
+            tc_commit(smem_u32(bar_acc2_full + b));
+          }
+          if (!ok) break;
+          tc_commit(smem_u32(bar_act_empty + ab));
+          ++jc;
         }
       }
     }
     __syncwarp();
   } else if (warp == 2) {
-    // ------------------------------ token gather (B operand of phase 1) ------------------------------
-    constexpr int kLag = 3;   // stages of cp.async kept in flight
-    uint32_t it = 0;
-    bool ok = true;
-    ChunkWalker walk(g_lo, g_hi, NG, reverse);
-    Chunk c;
-    while (ok && walk.next(c)) {
-      const WorkItem item = a.items[c.item];
-      for (int r = lane; r < item.n; r += 32) {
-        int row;
-        float wt;
-        slot_row_weight(a.perm[item.begin + r], d.T, d.k, a.topk_w, row, wt);
-        gather_row[r] = row;
-      }
-      __syncwarp();
-      const int chunks = item.n * 8;
-      int pending = 0;
-      for (int kb = 0; kb < KB; ++kb, ++it) {
-        const uint32_t s = it % C::kStages, par = (it / C::kStages) & 1;
-        ok = mbar_wait(smem_u32(bar_empty + s), par ^ 1, abort_flag, a.status, 9);
-        ok = __all_sync(0xffffffffu, ok);
-        if (!ok) break;
-        const uint32_t dstB = smem_u32(smem + s * C::kStageBytes + kATileBytes);
-        for (int ch16 = lane; ch16 < chunks; ch16 += 32) {
-          const int r = ch16 >> 3, ch = ch16 & 7;
-          const __nv_bfloat16* src = a.x + (size_t)gather_row[r] * d.H + kb * 64 + ch * 8;
-          const uint32_t dst = dstB + r * 128 + ((ch ^ (r & 7)) << 4);
-          asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
-        }
-        asm volatile("cp.async.commit_group;" ::: "memory");
-        if (++pending > kLag) {
-          asm volatile("cp.async.wait_group %0;" ::"n"(kLag) : "memory");
+    // ------------------------------ token gather (B operand of phase 1, gather mode) ------------------------------
+    if (!RES) {
+      constexpr int kLag = C::kLag;
+      uint32_t it = 0;
+      bool ok = true;
+      Walker walk(g_lo, g_hi, NG, HT, kScGroups);
+      Op op;
+      while (ok && walk.next(op)) {
+        if (op.kind == OP_PUBLISH) continue;
+        if (op.kind == OP_P1) {
+          const WorkItem item = a.items[op.item];
+          __syncwarp();
+          for (int r = lane; r < item.n; r += 32) {
+            int row;
+            float wt;
+            slot_row_weight(a.perm[item.begin + r], d.T, d.k, a.topk_w, row, wt);
+            gather_row[r] = row;
+          }
+          __syncwarp();
+          const int chunks = item.n * 8;
+          int pending = 0;
+          for (int kb = 0; kb < KB; ++kb, ++it) {
+            const uint32_t s = it % C::kStages, par = (it / C::kStages) & 1;
+            ok = mbar_wait(smem_u32(bar_empty + s), par ^ 1, abort_flag, a.status, 9);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            const uint32_t dstB = smem_u32(smem + s * C::kStageBytes + kATileBytes);
+            for (int ch16 = lane; ch16 < chunks; ch16 += 32) {
+              const int r = ch16 >> 3, ch = ch16 & 7;
+              const __nv_bfloat16* src = a.x + (size_t)gather_row[r] * d.H + kb * 64 + ch * 8;
+              const uint32_t dst = dstB + r * 128 + ((ch ^ (r & 7)) << 4);
+              asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+            }
+            asm volatile("cp.async.commit_group;" ::: "memory");
+            if (++pending > kLag) {
+              asm volatile("cp.async.wait_group %0;" ::"n"(kLag) : "memory");
+              fence_async_smem();
+              mbar_arrive(smem_u32(bar_fullB + (it - kLag) % C::kStages));
+              --pending;
+            }
+          }
+          asm volatile("cp.async.wait_group 0;" ::: "memory");
           fence_async_smem();
-          mbar_arrive(smem_u32(bar_fullB + (it - kLag) % C::kStages));
-          --pending;
+          if (ok)
+            for (int j = pending; j > 0; --j) mbar_arrive(smem_u32(bar_fullB + (it - j) % C::kStages));
+          __syncwarp();
+        } else {
+          // Phase-2 stages carry no token tile, but the ring's empty barriers must still be observed one
+          // round at a time: a parity wait that skipped a round could be satisfied by an older phase.
+          for (int ht = op.a * HT / 4; ok && ht < op.b * HT / 4; ++ht, ++it) {
+            const uint32_t s = it % C::kStages, par = (it / C::kStages) & 1;
+            ok = mbar_wait(smem_u32(bar_empty + s), par ^ 1, abort_flag, a.status, 12);
+            ok = __all_sync(0xffffffffu, ok);
+          }
         }
       }
+    }
+  } else if (warp == 3) {
+    // ------------------------------ activation-window loader (B operand of phase 2) ------------------------------
+    uint32_t jc = 0;
+    bool ok = true;
+    Walker walk(g_lo, g_hi, NG, HT, kScGroups);
+    Op op;
+    while (ok && walk.next(op)) {
+      if (op.kind != OP_P2) continue;
+      const WorkItem item = a.items[op.item];
+      const uint32_t ab = jc % kActBufs;
+      ok = mbar_wait(smem_u32(bar_act_empty + ab), ((jc / kActBufs) & 1) ^ 1, abort_flag, a.status, 14);
+      // all four groups of the window published (by this CTA and / or its neighbours)?
+      if (ok && lane == 0) {
+        const int32_t* flag = a.win_flags + op.W;
+        if (ld_acquire(flag) < 4) {
+          const unsigned long long t0 = clock64();
+          while (ld_acquire(flag) < 4) {
+            if (*abort_flag) { ok = false; break; }
+            if (clock64() - t0 > kWaitCycles) {
+              *abort_flag = 1;
+              set_status(a.status, TEAM_ERR_TIMEOUT, 15);
+              ok = false;
+              break;
+            }
+          }
+        }
+      }
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      const int ncols = RES ? d.T : item.n;
+      const int w = op.W - op.item * WPI;
+      const uint32_t dstB = smem_u32(act_buf + ab * C::kActBytes);
+      const __nv_bfloat16* base = a.act_g + (size_t)op.item * NT * d.I + w * kWindowCols;
+      for (int ch16 = lane; ch16 < ncols * 8; ch16 += 32) {
+        const int r = ch16 >> 3, ch = ch16 & 7;
+        const uint32_t dst = dstB + r * 128 + ((ch ^ (r & 7)) << 4);
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(base + (size_t)r * d.I + ch * 8)
+                     : "memory");
+      }
+      asm volatile("cp.async.commit_group;" ::: "memory");
       asm volatile("cp.async.wait_group 0;" ::: "memory");
       fence_async_smem();
-      if (ok)
-        for (int j = pending; j > 0; --j) mbar_arrive(smem_u32(bar_fullB + (it - j) % C::kStages));
-      __syncwarp();
-      // Phase-2 stages carry no B tile, but the ring's empty barriers must still be observed one
-      // round at a time: a parity wait that skipped a round could be satisfied by an older phase.
-      for (int ht = 0; ok && ht < HT; ++ht, ++it) {
-        const uint32_t s = it % C::kStages, par = (it / C::kStages) & 1;
-        ok = mbar_wait(smem_u32(bar_empty + s), par ^ 1, abort_flag, a.status, 12);
-        ok = __all_sync(0xffffffffu, ok);
-      }
+      mbar_arrive(smem_u32(bar_act_full + ab));
+      ++jc;
     }
   } else if (warp >= 4) {
     // ------------------------------ epilogue ------------------------------
-    const int q = warp - 4;                       // TMEM lane quarter == warp_id % 4 == group inside the chunk
+    const int q = warp - 4;                       // TMEM lane quarter == warp_id % 4
     int32_t* my_row = tbl_row + q * NT;
     float* my_wt = tbl_wt + q * NT;
     const uint32_t lane_off = (uint32_t)(q * 32) << 16;
-    uint32_t chunk_i = 0, t2 = 0;
+    uint32_t sc_i = 0, t2 = 0, use1 = 0;          // use1: bit t = parity of accumulator t's full barrier
+    int tbl_item = -1;
     bool ok = true;
-    ChunkWalker walk(g_lo, g_hi, NG, reverse);
-    Chunk c;
-    for (; ok && walk.next(c); ++chunk_i) {
-      const WorkItem item = a.items[c.item];
-      const int N = (item.n + 15) & ~15;
-      __syncwarp();
-      for (int r = lane; r < item.n; r += 32) {
-        int row;
-        float wt;
-        slot_row_weight(a.perm[item.begin + r], d.T, d.k, a.topk_w, row, wt);
-        my_row[r] = row;
-        my_wt[r] = wt;
-      }
-      __syncwarp();
-      // ---- SwiGLU: TMEM -> registers -> bf16 activation tile (B operand of phase 2) ----
-      ok = mbar_wait(smem_u32(bar_misc + 0), chunk_i & 1, abort_flag, a.status, 10);
-      ok = __all_sync(0xffffffffu, ok);
-      if (!ok) break;
-      tc_fence_after();
-      if (q < c.g) {
-        const int i_local = q * 16 + (lane & 15);     // column of the activation tile this lane pair owns
-        const bool first_half = lane < 16;
-        for (int c0 = 0; c0 < N; c0 += 8) {
-          float v[8];
-          tmem_ld8(tmem_acc1 + lane_off + c0, v);
-#pragma unroll
-          for (int j = 0; j < 8; ++j) {
-            const float o = __shfl_xor_sync(0xffffffffu, v[j], 16);
-            const bool mine_is_gate = (first_half == (a.gate_first != 0));
-            const float g = mine_is_gate ? v[j] : o;
-            const float u = mine_is_gate ? o : v[j];
-            v[j] = g / (1.f + expf(-g)) * u;
-          }
-          // lanes 0-15 store columns c0..c0+3, lanes 16-31 store c0+4..c0+7
-          const int jb = first_half ? 0 : 4;
-#pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            const int n = c0 + jb + j;
-            const uint32_t off = n * 128 + (((i_local >> 3) ^ (n & 7)) << 4) + (i_local & 7) * 2;
-            *reinterpret_cast<__nv_bfloat16*>(act_tile + off) = __float2bfloat16_rn(v[jb + j]);
-          }
-        }
-      }
-      tc_fence_before();
-      mbar_arrive(smem_u32(bar_misc + 1));
-      fence_async_smem();
-      mbar_arrive(smem_u32(bar_misc + 2));
-      // ---- down projection tiles: scale by routing weight, add into y ----
-      for (int ht = 0; ht < HT; ++ht, ++t2) {
-        const uint32_t b = t2 & 1, u = t2 >> 1;
-        ok = mbar_wait(smem_u32(bar_misc + 3 + b), u & 1, abort_flag, a.status, 11);
+    Walker walk(g_lo, g_hi, NG, HT, kScGroups);
+    Op op;
+    while (ok && walk.next(op)) {
+      if (op.kind == OP_P1) {
+        // ---- SwiGLU: TMEM -> registers -> bf16 activations in the global scratch ----
+        const WorkItem item = a.items[op.item];
+        const int ncols = RES ? d.T : item.n;
+        ok = mbar_wait(smem_u32(bar_acc1_full + op.tile), (use1 >> op.tile) & 1, abort_flag, a.status, 10);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
+        use1 ^= 1u << op.tile;
         tc_fence_after();
-        const uint32_t acc2 = tmem_base + NT * (1 + b) + lane_off;
-        float* ycol = a.y + ht * 128 + q * 32 + lane;
-        for (int c0 = 0; c0 < N; c0 += 8) {
-          float v[8];
-          tmem_ld8(acc2 + c0, v);
+        if (q < op.g) {
+          const int col = (op.j + q) * kGroupCols + (lane & 15);     // intermediate column of this lane pair
+          const bool first_half = lane < 16;
+          const bool mine_is_gate = (first_half == (a.gate_first != 0));
+          __nv_bfloat16* dst = a.act_g + (size_t)op.item * NT * d.I + col;
+          const uint32_t acc1 = tmem_base + op.tile * NT + lane_off;
+          for (int c0 = 0; c0 < ncols; c0 += 8) {
+            float v[8];
+            tmem_ld8(acc1 + c0, v);
 #pragma unroll
-          for (int j = 0; j < 8; ++j) {
-            const int n = c0 + j;
-            if (n < item.n) atomicAdd(ycol + (size_t)my_row[n] * d.H, my_wt[n] * v[j]);
+            for (int j = 0; j < 8; ++j) {
+              const float o = __shfl_xor_sync(0xffffffffu, v[j], 16);
+              const float g = mine_is_gate ? v[j] : o;
+              const float u = mine_is_gate ? o : v[j];
+              v[j] = g / (1.f + expf(-g)) * u;
+            }
+            // lanes 0-15 store tokens c0..c0+3, lanes 16-31 store c0+4..c0+7
+            const int jb = first_half ? 0 : 4;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              const int n = c0 + jb + j;
+              if (n < ncols) dst[(size_t)n * d.I] = __float2bfloat16_rn(v[jb + j]);
+            }
           }
         }
+      } else if (op.kind == OP_PUBLISH) {
+        // accumulators are free again; activations of the super-chunk become visible to every CTA
         tc_fence_before();
-        mbar_arrive(smem_u32(bar_misc + 5 + b));
+        mbar_arrive(smem_u32(bar_acc1_empty));
+        __threadfence();
+        mbar_arrive(smem_u32(bar_pub));
+        if (threadIdx.x == 128) {
+          if (mbar_wait(smem_u32(bar_pub), sc_i & 1, abort_flag, a.status, 16)) {
+            __threadfence();
+            for (int w = op.a >> 2; w <= ((op.b - 1) >> 2); ++w)
+              atomicAdd(a.win_flags + w, min(op.b, 4 * w + 4) - max(op.a, 4 * w));
+          }
+        }
+        ++sc_i;
+      } else {
+        // ---- down projection tiles: scale by routing weight, add into y ----
+        const WorkItem item = a.items[op.item];
+        const int ncols = RES ? d.T : item.n;
+        if (op.item != tbl_item) {
+          __syncwarp();
+          if (RES) {
+            for (int c = lane; c < kResidentRows; c += 32) {
+              my_row[c] = c;
+              my_wt[c] = 0.f;
+            }
+            __syncwarp();
+          }
+          for (int r = lane; r < item.n; r += 32) {
+            int row;
+            float wt;
+            slot_row_weight(a.perm[item.begin + r], d.T, d.k, a.topk_w, row, wt);
+            if (RES) {
+              my_wt[row] = wt;
+            } else {
+              my_row[r] = row;
+              my_wt[r] = wt;
+            }
+          }
+          __syncwarp();
+          tbl_item = op.item;
+        }
+        for (int ht = op.a * HT / 4; ht < op.b * HT / 4; ++ht, ++t2) {
+          const uint32_t b = t2 % C::kAcc2, u = t2 / C::kAcc2;
+          ok = mbar_wait(smem_u32(bar_acc2_full + b), u & 1, abort_flag, a.status, 11);
+          ok = __all_sync(0xffffffffu, ok);
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t acc2 = tmem_base + (C::kScWindows + b) * NT + lane_off;
+          float* ycol = a.y + ht * 128 + q * 32 + lane;
+          for (int c0 = 0; c0 < ncols; c0 += 8) {
+            float v[8];
+            tmem_ld8(acc2 + c0, v);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+              const int n = c0 + j;
+              if (n < ncols) {
+                const float wt = my_wt[n];
+                if (wt != 0.f) atomicAdd(ycol + (size_t)my_row[n] * d.H, wt * v[j]);
+              }
+            }
+          }
+          tc_fence_before();
+          mbar_arrive(smem_u32(bar_acc2_empty + b));
+        }
       }
     }
   }
@@ -547,18 +770,35 @@ int make_expert_maps(void* out_maps, const void* w_gate, const void* w_up, const
   return r == CUDA_SUCCESS ? 0 : (int)r;
 }
 
-template <int NT>
-static cudaError_t launch_tc(const void* maps, TcArgs args, int grid, cudaStream_t s) {
-  using C = TcCfg<NT>;
-  k_experts_tc<NT><<<grid, kTcThreads, C::kSmemBytes, s>>>(*reinterpret_cast<const TcMaps*>(maps), args);
-  return cudaGetLastError();
+// Rows per work item for a context: 16 selects the resident mode.
+int experts_tc_item_tile(int max_rows, int hidden) {
+  if (max_rows <= kResidentRows && hidden <= kResidentMaxHidden) return 16;
+  if (max_rows <= 64) return 32;
+  if (max_rows <= 256) return 64;
+  return 128;
 }
 
-cudaError_t configure_experts_tc(int item_tile) {
+template <int NT, bool RES>
+static cudaError_t launch_tc(const void* maps, TcArgs args, int grid, cudaStream_t s) {
+  using C = TcCfg<NT, RES>;
+  // Cooperative: CTAs that share a window wait for each other's activations, so all must be resident.
+  void* params[2] = {const_cast<void*>(maps), &args};
+  return cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(&k_experts_tc<NT, RES>), dim3(grid),
+                                     dim3(kTcThreads), params, (size_t)C::smem_bytes(args.d.H), s);
+}
+
+template <int NT, bool RES>
+static cudaError_t configure_tc(int hidden) {
+  return cudaFuncSetAttribute(k_experts_tc<NT, RES>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              TcCfg<NT, RES>::smem_bytes(hidden));
+}
+
+cudaError_t configure_experts_tc(int item_tile, int hidden) {
   switch (item_tile) {
-    case 32: return cudaFuncSetAttribute(k_experts_tc<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, TcCfg<32>::kSmemBytes);
-    case 64: return cudaFuncSetAttribute(k_experts_tc<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, TcCfg<64>::kSmemBytes);
-    case 128: return cudaFuncSetAttribute(k_experts_tc<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, TcCfg<128>::kSmemBytes);
+    case 16: return configure_tc<16, true>(hidden);
+    case 32: return configure_tc<32, false>(hidden);
+    case 64: return configure_tc<64, false>(hidden);
+    case 128: return configure_tc<128, false>(hidden);
     default: return cudaErrorInvalidValue;
   }
 }
@@ -571,14 +811,17 @@ cudaError_t launch_experts_tc(const void* maps, int gate_first, int item_tile, c
   a.topk_w = ws.r.topk_w;
   a.items = ws.items;
   a.n_items = ws.n_items;
+  a.act_g = ws.act_g;
+  a.win_flags = ws.win_flags;
   a.y = y;
   a.status = ws.status;
   a.d = d;
   a.gate_first = gate_first;
   switch (item_tile) {
-    case 32: return launch_tc<32>(maps, a, grid, s);
-    case 64: return launch_tc<64>(maps, a, grid, s);
-    case 128: return launch_tc<128>(maps, a, grid, s);
+    case 16: return launch_tc<16, true>(maps, a, grid, s);
+    case 32: return launch_tc<32, false>(maps, a, grid, s);
+    case 64: return launch_tc<64, false>(maps, a, grid, s);
+    case 128: return launch_tc<128, false>(maps, a, grid, s);
     default: return cudaErrorInvalidValue;
   }
 }

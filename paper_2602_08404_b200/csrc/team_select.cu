@@ -87,6 +87,8 @@ k_select(const float* __restrict__ logits, StepPtrs st, Workspace ws, RoutePtrs 
   for (int i = tid; i < d.G * n_words32; i += kSelThreads) s.mask[i] = 0u;
   for (int i = tid; i < d.G; i += kSelThreads) s.has_first[i] = 0;
   for (int i = tid; i < nw * EN; i += kSelThreads) s.hist[i] = 0;
+  // per-window publication counters of the expert kernel start every step from zero
+  for (int i = tid; i < ws.n_flags; i += kSelThreads) ws.win_flags[i] = 0;
   for (int t = tid; t < T; t += kSelThreads) {
     int g = st.group[t], b = st.branch[t];
     if (g < 0 || g >= d.G || b < 0 || b > 255) {
