@@ -11,10 +11,11 @@
 // same number of bytes (+- one group), every TMA box is a full 128-byte-row box and every weight
 // byte of an activated expert is requested exactly once per step.
 //
-// A CTA walks its range in super-chunks of up to kScWindows windows of one item:
-//   phase 1   D1[128, N] = A[128, H] * X[N, H]^T per tile of up to 4 groups (weights on M, tokens on
-//             N).  One 4-D TMA box per 64-wide k-block delivers the rows already interleaved as
-//             [group][gate 16 | up 16], so a gate row and its up row sit in the same warp's TMEM lanes.
+// A CTA walks its range in super-chunks of up to kScWindows windows (of any items):
+//   phase 1   D1[128, N] = A[128, H] * X[N, H]^T per tile = the CTA's groups of one window (weights on
+//             M, tokens on N).  One 4-D TMA box per 64-wide k-block delivers the rows already
+//             interleaved as [group][gate 16 | up 16], so a gate row and its up row sit in the same
+//             warp's TMEM lanes.
 //   SwiGLU    a = silu(gate) * up from TMEM, rounded to bf16 and published to a small global
 //             scratch [item][token][I]; a per-window counter says how many of its 4 groups are there.
 //   phase 2   for each of its groups' W_down tiles: D2[128, N] = Wd[128, 64] * a[N, 64]^T over the
@@ -58,11 +59,11 @@ struct TcCfg {
   static constexpr int kStages = RES ? 9 : (NT <= 32 ? 10 : (NT <= 64 ? 8 : 5));
   static constexpr int kLag = kStages >= 8 ? 5 : 3;             // gather stages kept in flight
   static constexpr int kActBytes = NT * 128;                    // NT tokens x 64 columns bf16
-  static constexpr int kScWindows = NT <= 32 ? 3 : 2;           // windows per super-chunk = phase-1 accumulators
+  static constexpr int kScWindows = NT <= 16 ? 4 : (NT <= 32 ? 3 : 2);   // windows per super-chunk = phase-1 accumulators
   static constexpr int kAcc2 = NT <= 16 ? 8 : (NT <= 32 ? 4 : 2);
   static constexpr int kTmemUsed = (kScWindows + kAcc2) * NT;
   static constexpr int kTmemCols = kTmemUsed <= 128 ? 128 : (kTmemUsed <= 256 ? 256 : 512);
-  static constexpr int kNumBars = 3 * kStages + kScWindows + 1 + 2 * kActBufs + 2 * kAcc2 + 2;
+  static constexpr int kNumBars = 3 * kStages + kScWindows + 1 + 2 * kActBufs + 2 * kAcc2 + 1;
   static constexpr int kBarBytes = ((kNumBars * 8 + 15) / 16) * 16;
   static constexpr int kTableBytes = 4 * NT * 8 + NT * 4;       // per-epilogue-warp (row, weight) + gather rows
   static constexpr int kRingBytes = kStages * kStageBytes;
@@ -216,52 +217,50 @@ enum { OP_P1 = 0, OP_PUBLISH = 1, OP_P2 = 2 };
 struct Op {
   int kind;
   int item;     // P1, P2: work item
-  int j, g;     // P1: first group inside the item, number of groups (1..4)
+  int j, g;     // P1: first group inside the item, number of groups (b - a)
   int tile;     // P1: accumulator index inside the super-chunk
-  int W;        // P2: global window index
-  int a, b;     // P2: the CTA's groups [a, b) of the window (0..4); PUBLISH: the super-chunk [a, b)
+  int W;        // P1, P2: global window index
+  int a, b;     // P1, P2: the CTA's groups [a, b) of the window (0..4)
 };
 
 struct Walker {
-  int lo, hi, NG, HT, scg;
-  int s_lo, s_hi, t0, W, tile, state;
-  __device__ Walker(int lo_, int hi_, int ng, int ht, int sc_groups)
-      : lo(lo_), hi(hi_), NG(ng), HT(ht), scg(sc_groups), s_lo(lo_), s_hi(lo_), t0(0), W(0), tile(0), state(0) {}
+  int lo, hi, NG, HT, scw;
+  int s_lo, s_hi, W, tile, state;
+  __device__ Walker(int lo_, int hi_, int ng, int ht, int sc_windows)
+      : lo(lo_), hi(hi_), NG(ng), HT(ht), scw(sc_windows), s_lo(lo_), s_hi(lo_), W(0), tile(0), state(0) {}
   __device__ bool defer_head() const { return (lo & 3) != 0; }
-  __device__ bool p2(Op& op, int w, int from, int to) const {
-    op.kind = OP_P2;
+  __device__ void window_part(Op& op, int w, int from, int to) const {
     op.W = w;
     op.a = max(from, 4 * w) - 4 * w;
     op.b = min(to, 4 * w + 4) - 4 * w;
     op.item = (4 * w) / NG;
+  }
+  __device__ bool p2(Op& op, int w, int from, int to) const {
+    op.kind = OP_P2;
+    window_part(op, w, from, to);
     return op.a * HT / 4 < op.b * HT / 4;     // jobs without a tile are skipped
   }
   __device__ bool next(Op& op) {
     for (;;) {
       switch (state) {
-        case 0: {                                   // open the next super-chunk
+        case 0:                                     // open the next super-chunk: up to scw windows, any items
           if (s_hi >= hi) { state = 4; break; }
           s_lo = s_hi;
-          const int item_end = (s_lo / NG + 1) * NG;
-          s_hi = min(hi, min(item_end, (s_lo & ~3) + scg));
-          t0 = s_lo;
+          s_hi = min(hi, ((s_lo >> 2) + scw) << 2);
+          W = s_lo >> 2;
           tile = 0;
           state = 1;
           break;
-        }
-        case 1:                                     // phase-1 tiles of up to 4 groups
-          if (t0 >= s_hi) { state = 2; break; }
+        case 1:                                     // phase-1 tiles: the CTA's groups of one window each
+          if (W > ((s_hi - 1) >> 2)) { state = 2; break; }
           op.kind = OP_P1;
-          op.item = t0 / NG;
-          op.j = t0 - op.item * NG;
-          op.g = min(4, s_hi - t0);
+          window_part(op, W++, s_lo, s_hi);
+          op.j = 4 * op.W - op.item * NG + op.a;
+          op.g = op.b - op.a;
           op.tile = tile++;
-          t0 += op.g;
           return true;
         case 2:
           op.kind = OP_PUBLISH;
-          op.a = s_lo;
-          op.b = s_hi;
           W = s_lo >> 2;
           state = 3;
           return true;
@@ -303,7 +302,6 @@ k_experts_tc(const __grid_constant__ TcMaps maps, TcArgs a) {
   uint64_t* bar_acc2_full = bar_act_empty + kActBufs;              // [kAcc2]
   uint64_t* bar_acc2_empty = bar_acc2_full + C::kAcc2;             // [kAcc2]
   uint64_t* bar_x = bar_acc2_empty + C::kAcc2;                     // [1] resident rows staged
-  uint64_t* bar_pub = bar_x + 1;                                   // [1] a super-chunk's activations stored
   int32_t* tbl_row = reinterpret_cast<int32_t*>(reinterpret_cast<unsigned char*>(bars) + C::kBarBytes);   // [4][NT]
   float* tbl_wt = reinterpret_cast<float*>(tbl_row + 4 * NT);                                             // [4][NT]
   int32_t* gather_row = reinterpret_cast<int32_t*>(tbl_wt + 4 * NT);                                      // [NT]
@@ -334,7 +332,6 @@ k_experts_tc(const __grid_constant__ TcMaps maps, TcArgs a) {
       mbar_init(smem_u32(bar_acc2_empty + i), 128);
     }
     mbar_init(smem_u32(bar_x), kXLoaders);
-    mbar_init(smem_u32(bar_pub), 128);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -352,7 +349,7 @@ k_experts_tc(const __grid_constant__ TcMaps maps, TcArgs a) {
   // This CTA's contiguous range of groups.
   const long long n_groups = (long long)(*a.n_items) * NG;
   const int g_lo = (int)(n_groups * blockIdx.x / gridDim.x), g_hi = (int)(n_groups * (blockIdx.x + 1) / gridDim.x);
-  constexpr int kScGroups = C::kScWindows * 4;
+  constexpr int kScGroups = C::kScWindows;   // windows per super-chunk
 
   // ------------------------------ resident rows (warps 2-7) ------------------------------
   if (RES && warp >= 2) {
@@ -599,7 +596,7 @@ k_experts_tc(const __grid_constant__ TcMaps maps, TcArgs a) {
     int32_t* my_row = tbl_row + q * NT;
     float* my_wt = tbl_wt + q * NT;
     const uint32_t lane_off = (uint32_t)(q * 32) << 16;
-    uint32_t sc_i = 0, t2 = 0, use1 = 0;          // use1: bit t = parity of accumulator t's full barrier
+    uint32_t t2 = 0, use1 = 0;                    // use1: bit t = parity of accumulator t's full barrier
     int tbl_item = -1;
     bool ok = true;
     Walker walk(g_lo, g_hi, NG, HT, kScGroups);
@@ -638,21 +635,17 @@ k_experts_tc(const __grid_constant__ TcMaps maps, TcArgs a) {
               if (n < ncols) dst[(size_t)n * d.I] = __float2bfloat16_rn(v[jb + j]);
             }
           }
-        }
-      } else if (op.kind == OP_PUBLISH) {
-        // accumulators are free again; activations of the super-chunk become visible to every CTA
-        tc_fence_before();
-        mbar_arrive(smem_u32(bar_acc1_empty));
-        __threadfence();
-        mbar_arrive(smem_u32(bar_pub));
-        if (threadIdx.x == 128) {
-          if (mbar_wait(smem_u32(bar_pub), sc_i & 1, abort_flag, a.status, 16)) {
+          // this warp's group of the window is published: visible to every CTA before the count moves
+          __syncwarp();
+          if (lane == 0) {
             __threadfence();
-            for (int w = op.a >> 2; w <= ((op.b - 1) >> 2); ++w)
-              atomicAdd(a.win_flags + w, min(op.b, 4 * w + 4) - max(op.a, 4 * w));
+            atomicAdd(a.win_flags + op.W, 1);
           }
         }
-        ++sc_i;
+      } else if (op.kind == OP_PUBLISH) {
+        // the super-chunk's accumulators are free again
+        tc_fence_before();
+        mbar_arrive(smem_u32(bar_acc1_empty));
       } else {
         // ---- down projection tiles: scale by routing weight, add into y ----
         const WorkItem item = a.items[op.item];
