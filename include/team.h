@@ -142,9 +142,9 @@ int team_create(const team_config *cfg, team_ctx **out);
 int team_destroy(team_ctx *ctx);
 
 /* Borrow the layer's weights (device pointers, 16-byte aligned; bf16 expert
- * weights 128-byte aligned).  Builds the TMA descriptors for the bf16 path.
- * May be called again to switch layers; a switch is stream-ordered by the
- * caller (descriptors are passed by value at launch). */
+ * weights 128-byte aligned).  May be called again to switch layers; the switch
+ * takes effect for calls issued afterwards (pointers are passed by value at
+ * launch). */
 int team_set_weights(team_ctx *ctx, const team_weights *w);
 
 /* Change flags / tau_hot / L_hot / hot_dist_inclusive / prefix_decoded /

@@ -1,6 +1,4 @@
 // C ABI of the TEAM MoE-layer library: context, argument checks, kernel launch sequences.
-#include <cuda.h>
-
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
@@ -10,11 +8,8 @@
 #include "team_common.cuh"
 
 namespace team {
-int make_expert_maps(void* out_maps, const void* w_gate, const void* w_up, const void* w_down, uint64_t rows_gu,
-                     uint64_t H, uint64_t rows_d, uint64_t I, int* gate_first);
-size_t experts_tc_maps_bytes();
-cudaError_t launch_experts_tc(const void* maps, int gate_first, int item_tile, const void* x, Workspace ws, float* y,
-                              Dims d, int grid, cudaStream_t s);
+cudaError_t launch_experts_tc(int item_tile, const void* x, const void* w_gate, const void* w_up, const void* w_down,
+                              Workspace ws, float* y, Dims d, int grid, cudaStream_t s);
 }  // namespace team
 
 struct team_ctx {
@@ -24,8 +19,6 @@ struct team_ctx {
   size_t ws_bytes;
   team_weights w;
   bool has_weights;
-  alignas(64) CUtensorMap maps[5];   // four gate/up views (1-4 groups per box) and W_down
-  int gate_first;
   int device;
   int n_sms;
   int item_tile;
@@ -103,7 +96,7 @@ team::RoutePtrs export_ptrs(const team_routing* r) {
 
 bool use_tensor_path(const team_ctx* ctx) { return ctx->cfg.dtype == TEAM_DTYPE_BF16 && !ctx->force_simt; }
 
-int pick_item_tile(const team_config& c) { return team::experts_tc_item_tile(c.max_rows, c.hidden); }
+int pick_item_tile(const team_config& c) { return team::experts_tc_item_tile(c.max_rows); }
 
 }  // namespace
 
@@ -154,7 +147,7 @@ int team_create(const team_config* cfg, team_ctx** out) {
   ctx->item_tile = pick_item_tile(*cfg);
   e = team::configure_router(cfg->dtype, cfg->hidden);
   if (e == cudaSuccess) e = team::configure_select(dims_of(*cfg, cfg->max_rows));
-  if (e == cudaSuccess && cfg->dtype == TEAM_DTYPE_BF16) e = team::configure_experts_tc(ctx->item_tile, cfg->hidden);
+  if (e == cudaSuccess && cfg->dtype == TEAM_DTYPE_BF16) e = team::configure_experts_tc(ctx->item_tile);
   if (e != cudaSuccess) {
     delete ctx;
     return TEAM_ERR_CUDA;
@@ -228,16 +221,6 @@ int team_set_weights(team_ctx* ctx, const team_weights* w) {
   if (((uintptr_t)w->w_router & 15) || ((uintptr_t)w->w_gate & align) || ((uintptr_t)w->w_up & align) ||
       ((uintptr_t)w->w_down & align))
     return TEAM_ERR_ARG;
-  if (ctx->cfg.dtype == TEAM_DTYPE_BF16) {
-    const uint64_t EN = ctx->cfg.n_experts + ctx->cfg.n_shared, I = ctx->cfg.inter, H = ctx->cfg.hidden;
-    if (team::experts_tc_maps_bytes() != sizeof(ctx->maps)) return TEAM_ERR_SHAPE;
-    const int r = team::make_expert_maps(ctx->maps, w->w_gate, w->w_up, w->w_down, EN * I, H, EN * H, I,
-                                         &ctx->gate_first);
-    if (r != 0) {
-      snprintf(ctx->cuda_err, sizeof(ctx->cuda_err), "cuTensorMapEncodeTiled failed (%d)", r);
-      return TEAM_ERR_CUDA;
-    }
-  }
   ctx->w = *w;
   ctx->has_weights = true;
   return TEAM_OK;
@@ -330,7 +313,7 @@ int team_moe_forward(team_ctx* ctx, const void* x, const team_step_state* st, te
     cudaEventRecord(ev0, s);
   }
   if (tc) {
-    e = team::launch_experts_tc(ctx->maps, ctx->gate_first, ctx->item_tile, x, ctx->ws, y, d, ctx->n_sms, s);
+    e = team::launch_experts_tc(ctx->item_tile, x, ctx->w.w_gate, ctx->w.w_up, ctx->w.w_down, ctx->ws, y, d, ctx->n_sms, s);
     if (e != cudaSuccess) return fail_cuda(ctx, e, "expert kernel");
     ++ctx->last_launches;
   } else {

@@ -96,8 +96,8 @@ __device__ __forceinline__ void slot_row_weight(int slot, int T, int k, const fl
 // Kernel launchers (host side), one per translation unit.
 cudaError_t configure_router(int dtype, int hidden);
 cudaError_t configure_select(Dims max_dims);
-cudaError_t configure_experts_tc(int item_tile, int hidden);
-int experts_tc_item_tile(int max_rows, int hidden);
+cudaError_t configure_experts_tc(int item_tile);
+int experts_tc_item_tile(int max_rows);
 cudaError_t launch_router_logits(const void* x, int dtype, const float* w_router, const uint8_t* tok_state,
                                  float* logits, float* y_zero, Dims d, int flags, cudaStream_t s);
 cudaError_t launch_router_topk(const float* logits, const uint8_t* tok_state, RoutePtrs out, Dims d, Policy p,

@@ -1,5 +1,6 @@
-// Grouped SwiGLU expert kernel for bf16 weights on sm_100a: TMA-staged weight tiles, tcgen05.mma
-// with accumulators in tensor memory, SwiGLU and the routing-weight scatter-combine fused in.
+// Grouped SwiGLU expert kernel for bf16 weights on sm_100a: weight tiles streamed into a shared-memory
+// ring, tcgen05.mma with accumulators in tensor memory, SwiGLU and the routing-weight
+// scatter-combine fused in.
 //
 // Unit of work and balance.  A work item is a run of up to NT token-slots of one activated expert
 // (built by the selection kernel).  Its intermediate dimension is cut into "groups" of 16 columns.
@@ -8,14 +9,13 @@
 //     phase 2   a quarter of the W_down tiles of the group's 64-column "window": the g-th group of
 //               a window owns the hidden-row tiles [g*HT/4, (g+1)*HT/4) of that window,
 // so the global list of groups is cut into one contiguous range per CTA and every SM streams the
-// same number of bytes (+- one group), every TMA box is a full 128-byte-row box and every weight
-// byte of an activated expert is requested exactly once per step.
+// same number of bytes (+- one group) and every weight byte of an activated expert is requested
+// exactly once per step.
 //
 // A CTA walks its range in super-chunks of up to kScWindows windows (of any items):
 //   phase 1   D1[128, N] = A[128, H] * X[N, H]^T per tile = the CTA's groups of one window (weights on
-//             M, tokens on N).  One 4-D TMA box per 64-wide k-block delivers the rows already
-//             interleaved as [group][gate 16 | up 16], so a gate row and its up row sit in the same
-//             warp's TMEM lanes.
+//             M, tokens on N); tile rows are ordered [group][gate 16 | up 16], so a gate row and its
+//             up row sit in the same warp's TMEM lanes.
 //   SwiGLU    a = silu(gate) * up from TMEM, rounded to bf16 and published to a small global
 //             scratch [item][token][I]; a per-window counter says how many of its 4 groups are there.
 //   phase 2   for each of its groups' W_down tiles: D2[128, N] = Wd[128, 64] * a[N, 64]^T over the
@@ -27,54 +27,56 @@
 // publish ever waits on another CTA, so the waits cannot form a cycle; the launch is cooperative so
 // that all CTAs are resident, and every wait is bounded.
 //
+// Loads.  Four loader warps fill the ring with cp.async: every warp instruction fetches kKbs * 128
+// contiguous bytes of one weight row (phase 1) or 128-byte row pieces of four rows (phase 2) and
+// scatters them into the K-major, 128-byte-swizzled tiles the tensor core reads; the stage's
+// mbarrier is armed to fire when the copies land (cp.async.mbarrier.arrive), so a loader only ever
+// blocks on a free slot.  (Measured on B200: tiled TMA boxes deliver 128-byte pieces of
+// 4 KB-strided rows at 3.6-5.7 TB/s; these requests reach 7 TB/s.)  A stage holds kKbs consecutive
+// k-blocks of the tile (or kKbs W_down tiles) plus the matching slices of the token rows.
 // Two operand modes:
-//   resident  (T <= 16 rows, N = 16): all rows of x sit in shared memory for the whole kernel and
-//             every expert is applied to all of them; rows not routed to the expert get weight 0.
-//             With no per-stage token tile, partial tiles (1-2 groups) pack several k-blocks into
-//             one 16 KB stage.
-//   gather    (N = 16..NT): a warp gathers the item's token rows per k-block with cp.async.
+//   resident-N (T <= 16 rows, N = 16): every expert is applied to all rows of x; rows not routed
+//              to the expert get weight 0 in the combine.
+//   gather     (N = 16..NT): the loaders gather the item's token rows.
 //
-// Warp roles (256 threads): warp 0 = TMA producer, warp 1 = MMA issuer + TMEM owner, warp 2 = token
-// gather, warp 3 = activation-window loader, warps 4-7 = epilogue (one TMEM lane quarter each).
-// On a wait's expiry the kernel records TEAM_ERR_TIMEOUT, drains and frees its tensor memory.
-#include <cuda.h>
-
+// Warp roles (384 threads): warps 0-3 = loaders, warp 4 = MMA issuer + TMEM owner (converged warp,
+// one elected lane issues), warp 5 = activation-window loader, warps 8-11 = epilogue (one TMEM lane
+// quarter each).  On a wait's expiry the kernel records TEAM_ERR_TIMEOUT, drains and frees its
+// tensor memory.
 #include "team_common.cuh"
 
 namespace team {
 
-constexpr int kTcThreads = 256;
+constexpr int kTcThreads = 384;
+constexpr int kLoaders = 4;                     // warps 0..3
+constexpr int kMmaWarp = 4;
+constexpr int kActWarp = 5;
+constexpr int kEpiWarp0 = 8;                    // warps 8..11 (warp % 4 = TMEM lane quarter)
 constexpr int kATileBytes = 128 * 128;          // 128 rows x 64 bf16
 constexpr int kGroupCols = 16;                  // intermediate columns per group (the unit of balance)
 constexpr int kWindowCols = 64;                 // columns per window (one 128-byte swizzle row of W_down)
-constexpr int kActBufs = 2;                     // activation windows staged in shared memory
-constexpr int kResidentRows = 16;               // N of the resident mode
-constexpr int kResidentMaxHidden = 2048;        // 16 rows x H x 2 B must fit beside the ring
+constexpr int kResidentRows = 16;               // N of the resident-N mode
 constexpr unsigned long long kWaitCycles = 2000000000ull;   // ~1 s at 2 GHz
 
-template <int NT, bool RES>
+template <int NT>
 struct TcCfg {
-  static constexpr int kBTileBytes = RES ? 0 : NT * 128;
-  static constexpr int kStageBytes = kATileBytes + kBTileBytes;
-  static constexpr int kStages = RES ? 9 : (NT <= 32 ? 10 : (NT <= 64 ? 8 : 5));
-  static constexpr int kLag = kStages >= 8 ? 5 : 3;             // gather stages kept in flight
+  static constexpr bool kRes = NT == kResidentRows;
+  static constexpr int kKbs = kRes ? 4 : 2;                     // k-blocks (or W_down tiles) per stage
+  static constexpr int kABytes = kKbs * kATileBytes;
+  static constexpr int kBSub = NT * 128;                        // token tile of one k-block
+  static constexpr int kStageBytes = kABytes + kKbs * kBSub;
+  static constexpr int kStages = kRes ? 3 : (NT <= 32 ? 5 : (NT <= 64 ? 4 : 3));
+  static constexpr int kActBufs = NT <= 64 ? 2 : 1;             // activation windows staged in shared memory
   static constexpr int kActBytes = NT * 128;                    // NT tokens x 64 columns bf16
   static constexpr int kScWindows = NT <= 16 ? 4 : (NT <= 32 ? 3 : 2);   // windows per super-chunk = phase-1 accumulators
   static constexpr int kAcc2 = NT <= 16 ? 8 : (NT <= 32 ? 4 : 2);
   static constexpr int kTmemUsed = (kScWindows + kAcc2) * NT;
   static constexpr int kTmemCols = kTmemUsed <= 128 ? 128 : (kTmemUsed <= 256 ? 256 : 512);
-  static constexpr int kNumBars = 3 * kStages + kScWindows + 1 + 2 * kActBufs + 2 * kAcc2 + 1;
+  static constexpr int kNumBars = 2 * kStages + kScWindows + 1 + 2 * kActBufs + 2 * kAcc2;
   static constexpr int kBarBytes = ((kNumBars * 8 + 15) / 16) * 16;
-  static constexpr int kTableBytes = 4 * NT * 8 + NT * 4;       // per-epilogue-warp (row, weight) + gather rows
+  static constexpr int kTableBytes = 4 * NT * 8 + kLoaders * NT * 4;   // epilogue (row, weight) + loader row tables
   static constexpr int kRingBytes = kStages * kStageBytes;
-  // Partial resident tiles are read by the tensor core as full 128-row tiles starting at a 4 KB
-  // multiple inside the stage, i.e. up to 12 KB past the ring's end: the resident rows (or padding)
-  // sit there.
-  static __host__ __device__ int x_bytes(int H) { return RES ? kResidentRows * H * 2 : 0; }
-  static __host__ __device__ int pad_bytes(int H) { return RES ? (x_bytes(H) >= 12288 ? 0 : 12288 - x_bytes(H)) : 0; }
-  static __host__ __device__ int smem_bytes(int H) {
-    return 1024 + kRingBytes + x_bytes(H) + pad_bytes(H) + kActBufs * kActBytes + kBarBytes + kTableBytes + 64;
-  }
+  static constexpr int kSmemBytes = 1024 + kRingBytes + kActBufs * kActBytes + kBarBytes + kTableBytes + 64;
 };
 
 // ---------------------------------------------------------------------------------------------
@@ -87,9 +89,6 @@ __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
 }
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
 __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
   uint32_t ok;
@@ -119,37 +118,45 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     }
   }
 }
-
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
-  asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-      ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar)
-      : "memory");
+// The same for a whole converged warp: every lane returns the same answer.
+__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status,
+                                               int where) {
+  return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag, status, where));
 }
 
-__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, int c0, int c1, int c2, int c3,
-                                            uint32_t bar) {
-  asm volatile(
-      "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
-      ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(bar)
-      : "memory");
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
+// The barrier receives one arrival from this thread once all of its earlier cp.async copies have landed.
+__device__ __forceinline__ void cp_async_arrive(uint32_t bar) {
+  asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(bar) : "memory");
 }
 
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
+// Issued by a converged warp; one elected lane executes the instruction.  (Measured: issuing from a
+// lane inside divergent code costs ~140 cycles per tcgen05.mma, ~50 this way.)
 __device__ __forceinline__ void tc_commit(uint32_t bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+  asm volatile(
+      "{\n\t.reg .pred q;\n\t"
+      "elect.sync _|q, 0xffffffff;\n\t"
+      "@q tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n\t}"
+      ::"r"(bar)
+      : "memory");
 }
 
 // D[tmem] (+)= A[smem desc] * B[smem desc]^T, bf16 inputs, fp32 accumulate, M = 128.
 __device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
                                        uint32_t accumulate) {
   asm volatile(
-      "{\n\t.reg .pred p;\n\t"
+      "{\n\t.reg .pred p, q;\n\t"
+      "elect.sync _|q, 0xffffffff;\n\t"
       "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      "@q tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
       ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
       : "memory");
 }
@@ -186,28 +193,26 @@ __device__ __forceinline__ int ld_acquire(const int32_t* p) {
   return v;
 }
 
+// Byte offset of 16-byte piece `ch` of row `r` inside a K-major tile with the 128-byte swizzle.
+__device__ __forceinline__ uint32_t sw128(int r, int ch) { return (uint32_t)(r * 128 + ((ch ^ (r & 7)) << 4)); }
+
 // ---------------------------------------------------------------------------------------------
 // The kernel
 // ---------------------------------------------------------------------------------------------
 struct TcArgs {
-  const __nv_bfloat16* x;      // [T, H]
-  const int32_t* perm;         // slot ids grouped by expert
-  const float* topk_w;         // [T, k]
+  const __nv_bfloat16* x;       // [T, H]
+  const __nv_bfloat16* w_gate;  // [E + ns, I, H]
+  const __nv_bfloat16* w_up;    // [E + ns, I, H]
+  const __nv_bfloat16* w_down;  // [E + ns, H, I]
+  const int32_t* perm;          // slot ids grouped by expert
+  const float* topk_w;          // [T, k]
   const WorkItem* items;
   const int32_t* n_items;
-  __nv_bfloat16* act_g;        // [items][NT][I] published activations
-  int32_t* win_flags;          // [items * I/64] groups published per window (zeroed by the selection kernel)
-  float* y;                    // [T, H], pre-zeroed rows of computed tokens
+  __nv_bfloat16* act_g;         // [items][NT][I] published activations
+  int32_t* win_flags;           // [items * I/64] groups published per window (zeroed by the selection kernel)
+  float* y;                     // [T, H], pre-zeroed rows of computed tokens
   int32_t* status;
   Dims d;
-  int gate_first;              // 1: the 4-D box delivers [gate | up] per group, 0: [up | gate]
-};
-
-// Tensor maps: gu[g-1] = W_gate/W_up viewed as {H, 16 rows, 2 (gate, up), rows/16} with a box of g
-// groups; down = W_down as {I, rows} with a [128 x 64] box.
-struct TcMaps {
-  CUtensorMap gu[4];
-  CUtensorMap down;
 };
 
 // The sequence of operations a CTA performs on its group range [lo, hi); every warp role walks the
@@ -282,30 +287,29 @@ struct Walker {
   }
 };
 
-template <int NT, bool RES>
+template <int NT>
 __global__ void __launch_bounds__(kTcThreads, 1)
-k_experts_tc(const __grid_constant__ TcMaps maps, TcArgs a) {
-  using C = TcCfg<NT, RES>;
+k_experts_tc(TcArgs a) {
+  using C = TcCfg<NT>;
+  constexpr bool RES = C::kRes;
+  constexpr int KBS = C::kKbs;
   extern __shared__ unsigned char smem_dyn[];
   const Dims d = a.d;
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~uintptr_t(1023));
-  unsigned char* x_res = smem + C::kRingBytes;                                   // resident rows: [H/64][16][128 B]
-  unsigned char* act_buf = x_res + C::x_bytes(d.H) + C::pad_bytes(d.H);          // [kActBufs][NT][128 B]
-  uint64_t* bars = reinterpret_cast<uint64_t*>(act_buf + kActBufs * C::kActBytes);
-  uint64_t* bar_fullA = bars;
-  uint64_t* bar_fullB = bars + C::kStages;
-  uint64_t* bar_empty = bars + 2 * C::kStages;
-  uint64_t* bar_acc1_full = bars + 3 * C::kStages;                 // [kScWindows]
+  unsigned char* act_buf = smem + C::kRingBytes;                                 // [kActBufs][NT][128 B]
+  uint64_t* bars = reinterpret_cast<uint64_t*>(act_buf + C::kActBufs * C::kActBytes);
+  uint64_t* bar_full = bars;                                       // [kStages] loaders -> MMA
+  uint64_t* bar_empty = bars + C::kStages;                         // [kStages] MMA -> loaders
+  uint64_t* bar_acc1_full = bars + 2 * C::kStages;                 // [kScWindows]
   uint64_t* bar_acc1_empty = bar_acc1_full + C::kScWindows;        // [1]
   uint64_t* bar_act_full = bar_acc1_empty + 1;                     // [kActBufs]
-  uint64_t* bar_act_empty = bar_act_full + kActBufs;               // [kActBufs]
-  uint64_t* bar_acc2_full = bar_act_empty + kActBufs;              // [kAcc2]
+  uint64_t* bar_act_empty = bar_act_full + C::kActBufs;            // [kActBufs]
+  uint64_t* bar_acc2_full = bar_act_empty + C::kActBufs;           // [kAcc2]
   uint64_t* bar_acc2_empty = bar_acc2_full + C::kAcc2;             // [kAcc2]
-  uint64_t* bar_x = bar_acc2_empty + C::kAcc2;                     // [1] resident rows staged
   int32_t* tbl_row = reinterpret_cast<int32_t*>(reinterpret_cast<unsigned char*>(bars) + C::kBarBytes);   // [4][NT]
   float* tbl_wt = reinterpret_cast<float*>(tbl_row + 4 * NT);                                             // [4][NT]
-  int32_t* gather_row = reinterpret_cast<int32_t*>(tbl_wt + 4 * NT);                                      // [NT]
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gather_row + NT);
+  int32_t* ld_row = reinterpret_cast<int32_t*>(tbl_wt + 4 * NT);                                          // [kLoaders][NT]
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(ld_row + kLoaders * NT);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -313,17 +317,15 @@ k_experts_tc(const __grid_constant__ TcMaps maps, TcArgs a) {
   const int HT = d.H / 128;         // row tiles of W_down
   const int NG = d.I / kGroupCols;  // groups per work item
   const int WPI = NG / 4;           // windows per work item
-  constexpr int kXLoaders = kTcThreads - 64;   // warps 2-7 stage the resident rows
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < C::kStages; ++s) {
-      mbar_init(smem_u32(bar_fullA + s), 1);
-      mbar_init(smem_u32(bar_fullB + s), 32);
+      mbar_init(smem_u32(bar_full + s), kLoaders * 32);
       mbar_init(smem_u32(bar_empty + s), 1);
     }
     for (int i = 0; i < C::kScWindows; ++i) mbar_init(smem_u32(bar_acc1_full + i), 1);
     mbar_init(smem_u32(bar_acc1_empty), 128);
-    for (int i = 0; i < kActBufs; ++i) {
+    for (int i = 0; i < C::kActBufs; ++i) {
       mbar_init(smem_u32(bar_act_full + i), 32);
       mbar_init(smem_u32(bar_act_empty + i), 1);
     }
@@ -331,15 +333,25 @@ k_experts_tc(const __grid_constant__ TcMaps maps, TcArgs a) {
       mbar_init(smem_u32(bar_acc2_full + i), 1);
       mbar_init(smem_u32(bar_acc2_empty + i), 128);
     }
-    mbar_init(smem_u32(bar_x), kXLoaders);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  if (warp == 1) {
+  if (warp == kMmaWarp) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
                  "r"((uint32_t)C::kTmemCols)
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  if (RES && warp < kLoaders) {
+    // token rows T..15 of every stage's token tiles stay zero for the whole kernel
+    for (int i = threadIdx.x; i < C::kStages * KBS * (kResidentRows * 8); i += kLoaders * 32) {
+      const int ch = i & 7, r = (i >> 3) % kResidentRows, sub = (i >> 3) / kResidentRows;
+      if (r >= d.T) {
+        const uint32_t dst = smem_u32(smem + (sub / KBS) * C::kStageBytes + C::kABytes + (sub % KBS) * C::kBSub) + sw128(r, ch);
+        asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(dst), "r"(0) : "memory");
+      }
+    }
+    fence_async_smem();
   }
   tc_fence_before();
   __syncthreads();
@@ -349,213 +361,163 @@ k_experts_tc(const __grid_constant__ TcMaps maps, TcArgs a) {
   // This CTA's contiguous range of groups.
   const long long n_groups = (long long)(*a.n_items) * NG;
   const int g_lo = (int)(n_groups * blockIdx.x / gridDim.x), g_hi = (int)(n_groups * (blockIdx.x + 1) / gridDim.x);
-  constexpr int kScGroups = C::kScWindows;   // windows per super-chunk
 
-  // ------------------------------ resident rows (warps 2-7) ------------------------------
-  if (RES && warp >= 2) {
-    const int tid = threadIdx.x - 64;
-    const int per_row = d.H / 8;                       // 16-byte pieces per row
-    if (g_lo < g_hi) {
-      for (int c = tid; c < kResidentRows * per_row; c += kXLoaders) {
-        const int r = c / per_row, cc = c - r * per_row, kb = cc >> 3, ch = cc & 7;
-        const uint32_t dst = smem_u32(x_res + kb * (kResidentRows * 128) + r * 128 + ((ch ^ (r & 7)) << 4));
-        if (r < d.T) {
-          const __nv_bfloat16* src = a.x + (size_t)r * d.H + cc * 8;
-          asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
-        } else {
-          asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(dst), "r"(0) : "memory");
-        }
-      }
-      asm volatile("cp.async.commit_group;" ::: "memory");
-      asm volatile("cp.async.wait_group 0;" ::: "memory");
-      fence_async_smem();
-    }
-    mbar_arrive(smem_u32(bar_x));
-  }
-
-  if (warp == 0) {
-    // ------------------------------ TMA producer ------------------------------
-    if (lane == 0) {
-      uint32_t it = 0;
-      bool ok = true;
-      Walker walk(g_lo, g_hi, NG, HT, kScGroups);
-      Op op;
-      while (ok && walk.next(op)) {
-        if (op.kind == OP_PUBLISH) continue;
-        const WorkItem item = a.items[op.item];
-        if (op.kind == OP_P1) {
-          const int grp = item.e * NG + op.j;                       // coordinate in units of 16 rows
-          const CUtensorMap* gu = &maps.gu[op.g - 1];
-          const uint32_t box_bytes = (uint32_t)op.g * 4096u;
-          const int nb = RES ? (op.g == 1 ? 4 : (op.g == 2 ? 2 : 1)) : 1;   // k-blocks per stage
-          for (int kb0 = 0; kb0 < KB; kb0 += nb, ++it) {
-            const uint32_t s = it % C::kStages, par = (it / C::kStages) & 1;
-            if (!(ok = mbar_wait(smem_u32(bar_empty + s), par ^ 1, abort_flag, a.status, 1))) break;
-            const uint32_t dst = smem_u32(smem + s * C::kStageBytes), bar = smem_u32(bar_fullA + s);
-            const int n = min(nb, KB - kb0);
-            mbar_arrive_expect_tx(bar, (uint32_t)n * box_bytes);
-            for (int i = 0; i < n; ++i) tma_load_4d(dst + i * box_bytes, gu, (kb0 + i) * 64, 0, 0, grp, bar);
-          }
-        } else {
-          const int w = op.W - op.item * WPI;
-          for (int ht = op.a * HT / 4; ht < op.b * HT / 4; ++ht, ++it) {
-            const uint32_t s = it % C::kStages, par = (it / C::kStages) & 1;
-            if (!(ok = mbar_wait(smem_u32(bar_empty + s), par ^ 1, abort_flag, a.status, 2))) break;
-            const uint32_t dst = smem_u32(smem + s * C::kStageBytes), bar = smem_u32(bar_fullA + s);
-            mbar_arrive_expect_tx(bar, kATileBytes);
-            tma_load_2d(dst, &maps.down, w * kWindowCols, item.e * d.H + ht * 128, bar);
-          }
-        }
-      }
-      if (*abort_flag) {
-        // Let copies already in flight land before the CTA's shared memory is released.
-        const uint32_t back = it < (uint32_t)C::kStages ? it : (uint32_t)C::kStages;
-        for (uint32_t j = it - back; j < it; ++j) {
-          const uint32_t s = j % C::kStages, par = (j / C::kStages) & 1;
-          const unsigned long long t0 = clock64();
-          while (!mbar_try(smem_u32(bar_fullA + s), par) && clock64() - t0 < kWaitCycles / 16) {}
-        }
-      }
-    }
-    __syncwarp();
-  } else if (warp == 1) {
-    // ------------------------------ MMA issuer ------------------------------
-    if (lane == 0) {
-      uint32_t it = 0, sc_i = 0, t2 = 0, jc = 0, bphase = 0;
-      bool ok = true;
-      if (RES) ok = mbar_wait(smem_u32(bar_x), 0, abort_flag, a.status, 13);
-      Walker walk(g_lo, g_hi, NG, HT, kScGroups);
-      Op op;
-      while (ok && walk.next(op)) {
-        if (op.kind == OP_PUBLISH) { ++sc_i; continue; }
-        const WorkItem item = a.items[op.item];
-        const int N = RES ? kResidentRows : ((item.n + 15) & ~15);
-        const uint32_t idesc = make_idesc_bf16(N);
-        if (op.kind == OP_P1) {
-          if (op.tile == 0) {
-            // the epilogue has read the previous super-chunk's accumulators
-            if (!(ok = mbar_wait(smem_u32(bar_acc1_empty), (sc_i & 1) ^ 1, abort_flag, a.status, 3))) break;
-            tc_fence_after();
-          }
-          const uint32_t acc1 = tmem_base + op.tile * NT;
-          const uint32_t box_bytes = (uint32_t)op.g * 4096u;
-          const int nb = RES ? (op.g == 1 ? 4 : (op.g == 2 ? 2 : 1)) : 1;
-          for (int kb0 = 0; kb0 < KB; kb0 += nb, ++it) {
-            const uint32_t s = it % C::kStages, par = (it / C::kStages) & 1;
-            if (!(ok = mbar_wait(smem_u32(bar_fullA + s), par, abort_flag, a.status, 4))) break;
-            if (!RES) {
-              if (!(ok = mbar_wait(smem_u32(bar_fullB + s), (bphase >> s) & 1, abort_flag, a.status, 5))) break;
-              bphase ^= 1u << s;
-            }
-            tc_fence_after();
-            const uint32_t sa = smem_u32(smem + s * C::kStageBytes);
-            const int n = min(nb, KB - kb0);
-            for (int i = 0; i < n; ++i) {
-              const int kb = kb0 + i;
-              const uint64_t da = make_kmajor_sw128_desc(sa + i * box_bytes);
-              const uint64_t db = make_kmajor_sw128_desc(RES ? smem_u32(x_res) + kb * (kResidentRows * 128)
-                                                             : sa + kATileBytes);
-#pragma unroll
-              for (int k4 = 0; k4 < 4; ++k4) tc_mma(acc1, da + 2 * k4, db + 2 * k4, idesc, (kb | k4) != 0);
-            }
-            tc_commit(smem_u32(bar_empty + s));
-          }
-          if (!ok) break;
-          tc_commit(smem_u32(bar_acc1_full + op.tile));
-        } else {
-          const uint32_t ab = jc % kActBufs;
-          if (!(ok = mbar_wait(smem_u32(bar_act_full + ab), (jc / kActBufs) & 1, abort_flag, a.status, 6))) break;
-          tc_fence_after();
-          const uint64_t act_desc = make_kmajor_sw128_desc(smem_u32(act_buf + ab * C::kActBytes));
-          for (int ht = op.a * HT / 4; ht < op.b * HT / 4; ++ht, ++it, ++t2) {
-            const uint32_t b = t2 % C::kAcc2, u = t2 / C::kAcc2;
-            if (!(ok = mbar_wait(smem_u32(bar_acc2_empty + b), (u & 1) ^ 1, abort_flag, a.status, 7))) break;
-            const uint32_t s = it % C::kStages, par = (it / C::kStages) & 1;
-            if (!(ok = mbar_wait(smem_u32(bar_fullA + s), par, abort_flag, a.status, 8))) break;
-            tc_fence_after();
-            const uint64_t da = make_kmajor_sw128_desc(smem_u32(smem + s * C::kStageBytes));
-            const uint32_t acc2 = tmem_base + (C::kScWindows + b) * NT;
-#pragma unroll
-            for (int kk = 0; kk < 4; ++kk) tc_mma(acc2, da + 2 * kk, act_desc + 2 * kk, idesc, kk != 0);
-            tc_commit(smem_u32(bar_empty + s));
-            tc_commit(smem_u32(bar_acc2_full + b));
-          }
-          if (!ok) break;
-          tc_commit(smem_u32(bar_act_empty + ab));
-          ++jc;
-        }
-      }
-    }
-    __syncwarp();
-  } else if (warp == 2) {
-    // ------------------------------ token gather (B operand of phase 1, gather mode) ------------------------------
-    if (!RES) {
-      constexpr int kLag = C::kLag;
-      uint32_t it = 0;
-      bool ok = true;
-      Walker walk(g_lo, g_hi, NG, HT, kScGroups);
-      Op op;
-      while (ok && walk.next(op)) {
-        if (op.kind == OP_PUBLISH) continue;
-        if (op.kind == OP_P1) {
-          const WorkItem item = a.items[op.item];
+  if (warp < kLoaders) {
+    // ------------------------------ loaders: weights and token rows into the ring ------------------------------
+    constexpr int LPR = KBS * 8;            // lanes per row in phase 1 (16-byte pieces of KBS k-blocks)
+    constexpr int RPI = 32 / LPR;           // rows per warp instruction
+    constexpr int RSTEP = kLoaders * RPI;   // rows between two instructions of one warp
+    const int sub = lane / LPR, kbi = (lane >> 3) % KBS, ch = lane & 7;
+    int32_t* my_rows = ld_row + warp * NT;
+    uint32_t it = 0;
+    int tbl_item = -1;
+    bool ok = true;
+    Walker walk(g_lo, g_hi, NG, HT, C::kScWindows);
+    Op op;
+    while (ok && walk.next(op)) {
+      if (op.kind == OP_PUBLISH) continue;
+      const WorkItem item = a.items[op.item];
+      if (op.kind == OP_P1) {
+        const int ncols = RES ? d.T : item.n;
+        if (!RES && op.item != tbl_item) {
           __syncwarp();
           for (int r = lane; r < item.n; r += 32) {
             int row;
             float wt;
             slot_row_weight(a.perm[item.begin + r], d.T, d.k, a.topk_w, row, wt);
-            gather_row[r] = row;
+            my_rows[r] = row;
           }
           __syncwarp();
-          const int chunks = item.n * 8;
-          int pending = 0;
-          for (int kb = 0; kb < KB; ++kb, ++it) {
-            const uint32_t s = it % C::kStages, par = (it / C::kStages) & 1;
-            ok = mbar_wait(smem_u32(bar_empty + s), par ^ 1, abort_flag, a.status, 9);
-            ok = __all_sync(0xffffffffu, ok);
-            if (!ok) break;
-            const uint32_t dstB = smem_u32(smem + s * C::kStageBytes + kATileBytes);
-            for (int ch16 = lane; ch16 < chunks; ch16 += 32) {
-              const int r = ch16 >> 3, ch = ch16 & 7;
-              const __nv_bfloat16* src = a.x + (size_t)gather_row[r] * d.H + kb * 64 + ch * 8;
-              const uint32_t dst = dstB + r * 128 + ((ch ^ (r & 7)) << 4);
-              asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+          tbl_item = op.item;
+        }
+        const int blocks = op.g * 2;                                  // 16-row blocks: [group][gate | up]
+        const size_t wrow0 = (size_t)item.e * d.I + (size_t)op.j * kGroupCols;
+        // Row r of the tile = block b (even: gate, odd: up; group b / 2) * 16 + rr.  This lane's rows inside
+        // a block are rr0, rr0 + RSTEP, ...: constant strides, so the copies of one block are independent.
+        const int rr0 = warp * RPI + sub;
+        const size_t rstep = (size_t)RSTEP * d.H;
+        for (int kb0 = 0; kb0 < KB; kb0 += KBS) {
+          const uint32_t s = it % C::kStages, par = (it / C::kStages) & 1;
+          if (!(ok = mbar_wait_warp(smem_u32(bar_empty + s), par ^ 1, abort_flag, a.status, 1))) break;
+          if (kb0 + kbi < KB) {
+            const uint32_t dstA = smem_u32(smem + s * C::kStageBytes) + kbi * kATileBytes;
+            const uint32_t dstB = smem_u32(smem + s * C::kStageBytes + C::kABytes) + kbi * C::kBSub;
+            const int koff = (kb0 + kbi) * 64 + ch * 8;
+            for (int b = 0; b < blocks; ++b) {
+              const __nv_bfloat16* src =
+                  ((b & 1) ? a.w_up : a.w_gate) + (wrow0 + (size_t)(b >> 1) * kGroupCols + rr0) * d.H + koff;
+              const uint32_t dst = dstA + (uint32_t)(b * 16 + rr0) * 128u;
+#pragma unroll
+              for (int ii = 0; ii < 16 / RSTEP; ++ii) {
+                const int rr = rr0 + ii * RSTEP;      // (b * 16 + rr) & 7 == rr & 7
+                cp_async16(dst + (uint32_t)(ii * RSTEP) * 128u + (uint32_t)((ch ^ (rr & 7)) << 4), src + ii * rstep);
+              }
             }
-            asm volatile("cp.async.commit_group;" ::: "memory");
-            if (++pending > kLag) {
-              asm volatile("cp.async.wait_group %0;" ::"n"(kLag) : "memory");
-              fence_async_smem();
-              mbar_arrive(smem_u32(bar_fullB + (it - kLag) % C::kStages));
-              --pending;
-            }
+            for (int r = rr0; r < ncols; r += RSTEP)
+              cp_async16(dstB + sw128(r, ch), a.x + (size_t)(RES ? r : my_rows[r]) * d.H + koff);
           }
-          asm volatile("cp.async.wait_group 0;" ::: "memory");
-          fence_async_smem();
-          if (ok)
-            for (int j = pending; j > 0; --j) mbar_arrive(smem_u32(bar_fullB + (it - j) % C::kStages));
-          __syncwarp();
-        } else {
-          // Phase-2 stages carry no token tile, but the ring's empty barriers must still be observed one
-          // round at a time: a parity wait that skipped a round could be satisfied by an older phase.
-          for (int ht = op.a * HT / 4; ok && ht < op.b * HT / 4; ++ht, ++it) {
-            const uint32_t s = it % C::kStages, par = (it / C::kStages) & 1;
-            ok = mbar_wait(smem_u32(bar_empty + s), par ^ 1, abort_flag, a.status, 12);
-            ok = __all_sync(0xffffffffu, ok);
+          cp_async_arrive(smem_u32(bar_full + s));     // the stage is handed over when this lane's copies land
+          ++it;
+        }
+      } else {
+        const int w = op.W - op.item * WPI;
+        const int ht0 = op.a * HT / 4, ht1 = op.b * HT / 4;
+        // 4 rows x 128 B per warp instruction; this lane's rows r = r_first + 16 * ii share r & 7
+        const int r_first = warp * 4 + (lane >> 3);
+        const size_t rstep = (size_t)16 * d.I;
+        for (int t0 = ht0; t0 < ht1; t0 += KBS) {
+          const uint32_t s = it % C::kStages, par = (it / C::kStages) & 1;
+          if (!(ok = mbar_wait_warp(smem_u32(bar_empty + s), par ^ 1, abort_flag, a.status, 2))) break;
+          const int nt = min(KBS, ht1 - t0);
+          for (int i = 0; i < nt; ++i) {
+            const uint32_t dstA = smem_u32(smem + s * C::kStageBytes) + i * kATileBytes + sw128(r_first, ch);
+            const __nv_bfloat16* src =
+                a.w_down + ((size_t)item.e * d.H + (size_t)(t0 + i) * 128 + r_first) * d.I + w * kWindowCols + ch * 8;
+#pragma unroll
+            for (int ii = 0; ii < 8; ++ii) cp_async16(dstA + (uint32_t)ii * 16u * 128u, src + ii * rstep);
           }
+          cp_async_arrive(smem_u32(bar_full + s));
+          ++it;
         }
       }
     }
-  } else if (warp == 3) {
+    // everything still in flight lands before shared memory is released (also on abort)
+    cp_async_wait_all();
+  } else if (warp == kMmaWarp) {
+    // ------------------------------ MMA issuer (whole warp converged, elected lane issues) ------------------------------
+    uint32_t it = 0, sc_i = 0, t2 = 0, jc = 0;
+    bool ok = true;
+    Walker walk(g_lo, g_hi, NG, HT, C::kScWindows);
+    Op op;
+    while (ok && walk.next(op)) {
+      if (op.kind == OP_PUBLISH) { ++sc_i; continue; }
+      const WorkItem item = a.items[op.item];
+      const int N = RES ? kResidentRows : ((item.n + 15) & ~15);
+      const uint32_t idesc = make_idesc_bf16(N);
+      if (op.kind == OP_P1) {
+        if (op.tile == 0) {
+          // the epilogue has read the previous super-chunk's accumulators
+          if (!(ok = mbar_wait_warp(smem_u32(bar_acc1_empty), (sc_i & 1) ^ 1, abort_flag, a.status, 3))) break;
+          tc_fence_after();
+        }
+        const uint32_t acc1 = tmem_base + op.tile * NT;
+        for (int kb0 = 0; kb0 < KB; kb0 += KBS, ++it) {
+          const uint32_t s = it % C::kStages, par = (it / C::kStages) & 1;
+          if (!(ok = mbar_wait_warp(smem_u32(bar_full + s), par, abort_flag, a.status, 4))) break;
+          fence_async_smem();      // the loaders' cp.async writes (generic proxy) before the tensor core's reads
+          tc_fence_after();
+          const uint32_t sa = smem_u32(smem + s * C::kStageBytes);
+          const int n = min(KBS, KB - kb0);
+          for (int i = 0; i < n; ++i) {
+            const uint64_t da = make_kmajor_sw128_desc(sa + i * kATileBytes);
+            const uint64_t db = make_kmajor_sw128_desc(sa + C::kABytes + i * C::kBSub);
+#pragma unroll
+            for (int k4 = 0; k4 < 4; ++k4) tc_mma(acc1, da + 2 * k4, db + 2 * k4, idesc, ((kb0 + i) | k4) != 0);
+          }
+          tc_commit(smem_u32(bar_empty + s));
+        }
+        if (!ok) break;
+        tc_commit(smem_u32(bar_acc1_full + op.tile));
+      } else {
+        const uint32_t ab = jc % C::kActBufs;
+        if (!(ok = mbar_wait_warp(smem_u32(bar_act_full + ab), (jc / C::kActBufs) & 1, abort_flag, a.status, 6))) break;
+        tc_fence_after();
+        const uint64_t act_desc = make_kmajor_sw128_desc(smem_u32(act_buf + ab * C::kActBytes));
+        const int ht0 = op.a * HT / 4, ht1 = op.b * HT / 4;
+        for (int t0 = ht0; ok && t0 < ht1; t0 += KBS, ++it) {
+          const uint32_t s = it % C::kStages, par = (it / C::kStages) & 1;
+          if (!(ok = mbar_wait_warp(smem_u32(bar_full + s), par, abort_flag, a.status, 8))) break;
+          fence_async_smem();
+          const int nt = min(KBS, ht1 - t0);
+          for (int i = 0; i < nt; ++i, ++t2) {
+            const uint32_t b = t2 % C::kAcc2, u = t2 / C::kAcc2;
+            if (!(ok = mbar_wait_warp(smem_u32(bar_acc2_empty + b), (u & 1) ^ 1, abort_flag, a.status, 7))) break;
+            tc_fence_after();
+            const uint64_t da = make_kmajor_sw128_desc(smem_u32(smem + s * C::kStageBytes) + i * kATileBytes);
+            const uint32_t acc2 = tmem_base + (C::kScWindows + b) * NT;
+#pragma unroll
+            for (int kk = 0; kk < 4; ++kk) tc_mma(acc2, da + 2 * kk, act_desc + 2 * kk, idesc, kk != 0);
+            tc_commit(smem_u32(bar_acc2_full + b));
+          }
+          if (!ok) break;
+          tc_commit(smem_u32(bar_empty + s));
+        }
+        if (!ok) break;
+        tc_commit(smem_u32(bar_act_empty + ab));
+        ++jc;
+      }
+    }
+  } else if (warp == kActWarp) {
     // ------------------------------ activation-window loader (B operand of phase 2) ------------------------------
     uint32_t jc = 0;
     bool ok = true;
-    Walker walk(g_lo, g_hi, NG, HT, kScGroups);
+    Walker walk(g_lo, g_hi, NG, HT, C::kScWindows);
     Op op;
     while (ok && walk.next(op)) {
       if (op.kind != OP_P2) continue;
       const WorkItem item = a.items[op.item];
-      const uint32_t ab = jc % kActBufs;
-      ok = mbar_wait(smem_u32(bar_act_empty + ab), ((jc / kActBufs) & 1) ^ 1, abort_flag, a.status, 14);
+      const uint32_t ab = jc % C::kActBufs;
+      ok = mbar_wait(smem_u32(bar_act_empty + ab), ((jc / C::kActBufs) & 1) ^ 1, abort_flag, a.status, 14);
       // all four groups of the window published (by this CTA and / or its neighbours)?
       if (ok && lane == 0) {
         const int32_t* flag = a.win_flags + op.W;
@@ -580,41 +542,37 @@ k_experts_tc(const __grid_constant__ TcMaps maps, TcArgs a) {
       const __nv_bfloat16* base = a.act_g + (size_t)op.item * NT * d.I + w * kWindowCols;
       for (int ch16 = lane; ch16 < ncols * 8; ch16 += 32) {
         const int r = ch16 >> 3, ch = ch16 & 7;
-        const uint32_t dst = dstB + r * 128 + ((ch ^ (r & 7)) << 4);
-        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(base + (size_t)r * d.I + ch * 8)
-                     : "memory");
+        cp_async16(dstB + sw128(r, ch), base + (size_t)r * d.I + ch * 8);
       }
-      asm volatile("cp.async.commit_group;" ::: "memory");
-      asm volatile("cp.async.wait_group 0;" ::: "memory");
+      cp_async_commit();
+      cp_async_wait_all();
       fence_async_smem();
       mbar_arrive(smem_u32(bar_act_full + ab));
       ++jc;
     }
-  } else if (warp >= 4) {
+  } else if (warp >= kEpiWarp0) {
     // ------------------------------ epilogue ------------------------------
-    const int q = warp - 4;                       // TMEM lane quarter == warp_id % 4
+    const int q = warp - kEpiWarp0;               // TMEM lane quarter == warp_id % 4
     int32_t* my_row = tbl_row + q * NT;
     float* my_wt = tbl_wt + q * NT;
     const uint32_t lane_off = (uint32_t)(q * 32) << 16;
     uint32_t t2 = 0, use1 = 0;                    // use1: bit t = parity of accumulator t's full barrier
     int tbl_item = -1;
     bool ok = true;
-    Walker walk(g_lo, g_hi, NG, HT, kScGroups);
+    Walker walk(g_lo, g_hi, NG, HT, C::kScWindows);
     Op op;
     while (ok && walk.next(op)) {
       if (op.kind == OP_P1) {
         // ---- SwiGLU: TMEM -> registers -> bf16 activations in the global scratch ----
         const WorkItem item = a.items[op.item];
         const int ncols = RES ? d.T : item.n;
-        ok = mbar_wait(smem_u32(bar_acc1_full + op.tile), (use1 >> op.tile) & 1, abort_flag, a.status, 10);
-        ok = __all_sync(0xffffffffu, ok);
+        ok = mbar_wait_warp(smem_u32(bar_acc1_full + op.tile), (use1 >> op.tile) & 1, abort_flag, a.status, 10);
         if (!ok) break;
         use1 ^= 1u << op.tile;
         tc_fence_after();
         if (q < op.g) {
           const int col = (op.j + q) * kGroupCols + (lane & 15);     // intermediate column of this lane pair
-          const bool first_half = lane < 16;
-          const bool mine_is_gate = (first_half == (a.gate_first != 0));
+          const bool is_gate = lane < 16;                            // lanes 0-15 hold gate rows, 16-31 up rows
           __nv_bfloat16* dst = a.act_g + (size_t)op.item * NT * d.I + col;
           const uint32_t acc1 = tmem_base + op.tile * NT + lane_off;
           for (int c0 = 0; c0 < ncols; c0 += 8) {
@@ -623,12 +581,12 @@ k_experts_tc(const __grid_constant__ TcMaps maps, TcArgs a) {
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
               const float o = __shfl_xor_sync(0xffffffffu, v[j], 16);
-              const float g = mine_is_gate ? v[j] : o;
-              const float u = mine_is_gate ? o : v[j];
+              const float g = is_gate ? v[j] : o;
+              const float u = is_gate ? o : v[j];
               v[j] = g / (1.f + expf(-g)) * u;
             }
             // lanes 0-15 store tokens c0..c0+3, lanes 16-31 store c0+4..c0+7
-            const int jb = first_half ? 0 : 4;
+            const int jb = is_gate ? 0 : 4;
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
               const int n = c0 + jb + j;
@@ -675,8 +633,7 @@ k_experts_tc(const __grid_constant__ TcMaps maps, TcArgs a) {
         }
         for (int ht = op.a * HT / 4; ht < op.b * HT / 4; ++ht, ++t2) {
           const uint32_t b = t2 % C::kAcc2, u = t2 / C::kAcc2;
-          ok = mbar_wait(smem_u32(bar_acc2_full + b), u & 1, abort_flag, a.status, 11);
-          ok = __all_sync(0xffffffffu, ok);
+          ok = mbar_wait_warp(smem_u32(bar_acc2_full + b), u & 1, abort_flag, a.status, 11);
           if (!ok) break;
           tc_fence_after();
           const uint32_t acc2 = tmem_base + (C::kScWindows + b) * NT + lane_off;
@@ -703,7 +660,7 @@ k_experts_tc(const __grid_constant__ TcMaps maps, TcArgs a) {
   // ------------------------------ teardown ------------------------------
   tc_fence_before();
   __syncthreads();
-  if (warp == 1) {
+  if (warp == kMmaWarp) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)C::kTmemCols)
                  : "memory");
@@ -711,95 +668,46 @@ k_experts_tc(const __grid_constant__ TcMaps maps, TcArgs a) {
 }
 
 // ---------------------------------------------------------------------------------------------
-// Host side: tensor maps and launch
+// Host side
 // ---------------------------------------------------------------------------------------------
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-static EncodeTiledFn get_encode_fn() {
-  static EncodeTiledFn fn = nullptr;
-  if (fn == nullptr) {
-    void* p = nullptr;
-    cudaDriverEntryPointQueryResult q;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
-        q == cudaDriverEntryPointSuccess)
-      fn = reinterpret_cast<EncodeTiledFn>(p);
-  }
-  return fn;
-}
-
-size_t experts_tc_maps_bytes() { return sizeof(TcMaps); }
-
-// Builds the five tensor maps for a layer.  w_gate / w_up: bf16 [rows_gu, H]; w_down: bf16 [rows_d, I].
-// Returns 0, or a driver error code / -1.  *gate_first tells the kernel which of gate / up comes
-// first inside a group (the 4-D view needs a positive stride between the two matrices).
-int make_expert_maps(void* out_maps, const void* w_gate, const void* w_up, const void* w_down, uint64_t rows_gu,
-                     uint64_t H, uint64_t rows_d, uint64_t I, int* gate_first) {
-  EncodeTiledFn fn = get_encode_fn();
-  if (fn == nullptr) return -1;
-  TcMaps* m = reinterpret_cast<TcMaps*>(out_maps);
-  const uintptr_t pg = reinterpret_cast<uintptr_t>(w_gate), pu = reinterpret_cast<uintptr_t>(w_up);
-  *gate_first = pu > pg ? 1 : 0;
-  const uintptr_t base = pu > pg ? pg : pu, delta = pu > pg ? pu - pg : pg - pu;
-  if (delta == 0 || (delta & 15) || delta >= (1ull << 40)) return -2;
-  for (int g = 1; g <= 4; ++g) {
-    cuuint64_t dims[4] = {H, 16, 2, rows_gu / 16};
-    cuuint64_t strides[3] = {H * 2, delta, 16 * H * 2};
-    cuuint32_t box[4] = {64, 16, 2, (cuuint32_t)g};
-    cuuint32_t estr[4] = {1, 1, 1, 1};
-    CUresult r = fn(&m->gu[g - 1], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, reinterpret_cast<void*>(base), dims, strides,
-                    box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-                    CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    if (r != CUDA_SUCCESS) return (int)r;
-  }
-  cuuint64_t dims[2] = {I, rows_d};
-  cuuint64_t strides[1] = {I * 2};
-  cuuint32_t box[2] = {64, 128};
-  cuuint32_t estr[2] = {1, 1};
-  CUresult r = fn(&m->down, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(w_down), dims, strides, box, estr,
-                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  return r == CUDA_SUCCESS ? 0 : (int)r;
-}
-
-// Rows per work item for a context: 16 selects the resident mode.
-int experts_tc_item_tile(int max_rows, int hidden) {
-  if (max_rows <= kResidentRows && hidden <= kResidentMaxHidden) return 16;
+// Rows per work item for a context: 16 selects the resident-N mode.
+int experts_tc_item_tile(int max_rows) {
+  if (max_rows <= kResidentRows) return 16;
   if (max_rows <= 64) return 32;
   if (max_rows <= 256) return 64;
   return 128;
 }
 
-template <int NT, bool RES>
-static cudaError_t launch_tc(const void* maps, TcArgs args, int grid, cudaStream_t s) {
-  using C = TcCfg<NT, RES>;
+template <int NT>
+static cudaError_t launch_tc(TcArgs args, int grid, cudaStream_t s) {
   // Cooperative: CTAs that share a window wait for each other's activations, so all must be resident.
-  void* params[2] = {const_cast<void*>(maps), &args};
-  return cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(&k_experts_tc<NT, RES>), dim3(grid),
-                                     dim3(kTcThreads), params, (size_t)C::smem_bytes(args.d.H), s);
+  void* params[1] = {&args};
+  return cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(&k_experts_tc<NT>), dim3(grid), dim3(kTcThreads),
+                                     params, (size_t)TcCfg<NT>::kSmemBytes, s);
 }
 
-template <int NT, bool RES>
-static cudaError_t configure_tc(int hidden) {
-  return cudaFuncSetAttribute(k_experts_tc<NT, RES>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                              TcCfg<NT, RES>::smem_bytes(hidden));
+template <int NT>
+static cudaError_t configure_tc() {
+  return cudaFuncSetAttribute(k_experts_tc<NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, TcCfg<NT>::kSmemBytes);
 }
 
-cudaError_t configure_experts_tc(int item_tile, int hidden) {
+cudaError_t configure_experts_tc(int item_tile) {
   switch (item_tile) {
-    case 16: return configure_tc<16, true>(hidden);
-    case 32: return configure_tc<32, false>(hidden);
-    case 64: return configure_tc<64, false>(hidden);
-    case 128: return configure_tc<128, false>(hidden);
+    case 16: return configure_tc<16>();
+    case 32: return configure_tc<32>();
+    case 64: return configure_tc<64>();
+    case 128: return configure_tc<128>();
     default: return cudaErrorInvalidValue;
   }
 }
 
-cudaError_t launch_experts_tc(const void* maps, int gate_first, int item_tile, const void* x, Workspace ws, float* y,
-                              Dims d, int grid, cudaStream_t s) {
+cudaError_t launch_experts_tc(int item_tile, const void* x, const void* w_gate, const void* w_up, const void* w_down,
+                              Workspace ws, float* y, Dims d, int grid, cudaStream_t s) {
   TcArgs a;
   a.x = static_cast<const __nv_bfloat16*>(x);
+  a.w_gate = static_cast<const __nv_bfloat16*>(w_gate);
+  a.w_up = static_cast<const __nv_bfloat16*>(w_up);
+  a.w_down = static_cast<const __nv_bfloat16*>(w_down);
   a.perm = ws.r.perm;
   a.topk_w = ws.r.topk_w;
   a.items = ws.items;
@@ -809,12 +717,11 @@ cudaError_t launch_experts_tc(const void* maps, int gate_first, int item_tile, c
   a.y = y;
   a.status = ws.status;
   a.d = d;
-  a.gate_first = gate_first;
   switch (item_tile) {
-    case 16: return launch_tc<16, true>(maps, a, grid, s);
-    case 32: return launch_tc<32, false>(maps, a, grid, s);
-    case 64: return launch_tc<64, false>(maps, a, grid, s);
-    case 128: return launch_tc<128, false>(maps, a, grid, s);
+    case 16: return launch_tc<16>(a, grid, s);
+    case 32: return launch_tc<32>(a, grid, s);
+    case 64: return launch_tc<64>(a, grid, s);
+    case 128: return launch_tc<128>(a, grid, s);
     default: return cudaErrorInvalidValue;
   }
 }
