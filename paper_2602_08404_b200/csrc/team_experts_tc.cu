@@ -13,9 +13,9 @@
 // exactly once per step.
 //
 // A CTA walks its range in super-chunks of up to kScWindows windows (of any items):
-//   phase 1   D1[128, N] = A[128, H] * X[N, H]^T per tile = the CTA's groups of one window (weights on
-//             M, tokens on N); tile rows are ordered [group][gate 16 | up 16], so a gate row and its
-//             up row sit in the same warp's TMEM lanes.
+//   phase 1   D1[128, N] = A[128, H] * X[N, H]^T per tile of up to 4 consecutive groups (weights on M,
+//             tokens on N); tile rows are ordered [group][gate 16 | up 16], so a gate row and its up
+//             row sit in the same warp's TMEM lanes.
 //   SwiGLU    a = silu(gate) * up from TMEM, rounded to bf16 and published to a small global
 //             scratch [item][token][I]; a per-window counter says how many of its 4 groups are there.
 //   phase 2   for each of its groups' W_down tiles: D2[128, N] = Wd[128, 64] * a[N, 64]^T over the
@@ -56,6 +56,8 @@ constexpr int kATileBytes = 128 * 128;          // 128 rows x 64 bf16
 constexpr int kGroupCols = 16;                  // intermediate columns per group (the unit of balance)
 constexpr int kWindowCols = 64;                 // columns per window (one 128-byte swizzle row of W_down)
 constexpr int kResidentRows = 16;               // N of the resident-N mode
+constexpr int kRingBars = 16;                   // stages in flight at most (full / empty barrier pairs)
+constexpr int kMaxSmemBytes = 232448;           // dynamic shared memory a CTA may opt in to on sm_100
 constexpr unsigned long long kWaitCycles = 2000000000ull;   // ~1 s at 2 GHz
 
 template <int NT>
@@ -64,19 +66,20 @@ struct TcCfg {
   static constexpr int kKbs = kRes ? 4 : 2;                     // k-blocks (or W_down tiles) per stage
   static constexpr int kABytes = kKbs * kATileBytes;
   static constexpr int kBSub = NT * 128;                        // token tile of one k-block
-  static constexpr int kStageBytes = kABytes + kKbs * kBSub;
-  static constexpr int kStages = kRes ? 3 : (NT <= 32 ? 5 : (NT <= 64 ? 4 : 3));
+  static constexpr int kStageBytes = kABytes + kKbs * kBSub;    // a full (4-group) tile's stage
   static constexpr int kActBufs = NT <= 64 ? 2 : 1;             // activation windows staged in shared memory
   static constexpr int kActBytes = NT * 128;                    // NT tokens x 64 columns bf16
   static constexpr int kScWindows = NT <= 16 ? 4 : (NT <= 32 ? 3 : 2);   // windows per super-chunk = phase-1 accumulators
   static constexpr int kAcc2 = NT <= 16 ? 8 : (NT <= 32 ? 4 : 2);
   static constexpr int kTmemUsed = (kScWindows + kAcc2) * NT;
   static constexpr int kTmemCols = kTmemUsed <= 128 ? 128 : (kTmemUsed <= 256 ? 256 : 512);
-  static constexpr int kNumBars = 2 * kStages + kScWindows + 1 + 2 * kActBufs + 2 * kAcc2;
+  static constexpr int kNumBars = 2 * kRingBars + kScWindows + 1 + 2 * kActBufs + 2 * kAcc2;
   static constexpr int kBarBytes = ((kNumBars * 8 + 15) / 16) * 16;
   static constexpr int kTableBytes = 4 * NT * 8 + kLoaders * NT * 4;   // epilogue (row, weight) + loader row tables
-  static constexpr int kRingBytes = kStages * kStageBytes;
-  static constexpr int kSmemBytes = 1024 + kRingBytes + kActBufs * kActBytes + kBarBytes + kTableBytes + 64;
+  static constexpr int kOtherBytes = 1024 + kActBufs * kActBytes + kBarBytes + kTableBytes + 64;
+  static constexpr int kRingBytes = ((kMaxSmemBytes - kOtherBytes) / 1024) * 1024;   // everything that is left
+  static constexpr int kSmemBytes = kOtherBytes + kRingBytes;
+  static_assert(kRingBytes >= 3 * kStageBytes, "the ring must hold three full-tile stages");
 };
 
 // ---------------------------------------------------------------------------------------------
@@ -218,72 +221,181 @@ struct TcArgs {
 // The sequence of operations a CTA performs on its group range [lo, hi); every warp role walks the
 // same sequence.  Group indices are global (item * NG + group in item); since NG is a multiple of
 // 4, window W = group >> 2 never straddles two items.
+//
+// A super-chunk covers up to scw windows.  When the whole range is one super-chunk (the usual case
+// at small row counts) the groups of the windows it shares with its neighbours go first in phase 1
+// and the full windows last, and phase 2 starts with the shared windows: every CTA publishes what
+// its neighbours need early, and the exchange latency hides behind streaming.  With several
+// super-chunks the order is ascending and the tiles of the head window come last of all.
 enum { OP_P1 = 0, OP_PUBLISH = 1, OP_P2 = 2 };
 struct Op {
   int kind;
-  int item;     // P1, P2: work item
-  int j, g;     // P1: first group inside the item, number of groups (b - a)
+  int item;     // P1, P2: work item (all groups of a tile belong to one item)
+  int g;        // P1: number of groups (1..4)
+  int grp[4];   // P1: their global indices
   int tile;     // P1: accumulator index inside the super-chunk
-  int W;        // P1, P2: global window index
-  int a, b;     // P1, P2: the CTA's groups [a, b) of the window (0..4)
+  int W;        // P2: global window index
+  int a, b;     // P2: the CTA's groups [a, b) of the window (0..4)
 };
 
 struct Walker {
   int lo, hi, NG, HT, scw;
-  int s_lo, s_hi, W, tile, state;
+  int s_lo, s_hi, nH, nT, nM, tail0, mid0, li, ji, tile, state;
+  bool single, deferred;
   __device__ Walker(int lo_, int hi_, int ng, int ht, int sc_windows)
-      : lo(lo_), hi(hi_), NG(ng), HT(ht), scw(sc_windows), s_lo(lo_), s_hi(lo_), W(0), tile(0), state(0) {}
-  __device__ bool defer_head() const { return (lo & 3) != 0; }
-  __device__ void window_part(Op& op, int w, int from, int to) const {
+      : lo(lo_), hi(hi_), NG(ng), HT(ht), scw(sc_windows), s_lo(lo_), s_hi(lo_), nH(0), nT(0), nM(0), tail0(0),
+        mid0(0), li(0), ji(0), tile(0), state(0), single(false), deferred(false) {}
+  // phase-1 order of the super-chunk: head part, tail part, middle
+  __device__ int group_at(int i) const {
+    return i < nH ? s_lo + i : (i < nH + nT ? tail0 + (i - nH) : mid0 + (i - nH - nT));
+  }
+  __device__ bool p2(Op& op, int w, int from, int to) const {
+    op.kind = OP_P2;
     op.W = w;
     op.a = max(from, 4 * w) - 4 * w;
     op.b = min(to, 4 * w + 4) - 4 * w;
     op.item = (4 * w) / NG;
-  }
-  __device__ bool p2(Op& op, int w, int from, int to) const {
-    op.kind = OP_P2;
-    window_part(op, w, from, to);
     return op.a * HT / 4 < op.b * HT / 4;     // jobs without a tile are skipped
   }
   __device__ bool next(Op& op) {
     for (;;) {
       switch (state) {
-        case 0:                                     // open the next super-chunk: up to scw windows, any items
+        case 0:                                     // open the next super-chunk
           if (s_hi >= hi) { state = 4; break; }
           s_lo = s_hi;
           s_hi = min(hi, ((s_lo >> 2) + scw) << 2);
-          W = s_lo >> 2;
+          single = (s_lo == lo && s_hi == hi);
+          if (single) {
+            nH = (s_lo & 3) ? min(s_hi, (s_lo | 3) + 1) - s_lo : 0;
+            tail0 = max(s_hi & ~3, s_lo + nH);
+            nT = (s_hi & 3) ? max(0, s_hi - tail0) : 0;
+            mid0 = s_lo + nH;
+            nM = (s_hi - nT) - mid0;
+          } else {
+            nH = nT = 0;
+            mid0 = s_lo;
+            nM = s_hi - s_lo;
+            tail0 = s_hi;
+          }
+          li = 0;
+          ji = 0;
           tile = 0;
           state = 1;
           break;
-        case 1:                                     // phase-1 tiles: the CTA's groups of one window each
-          if (W > ((s_hi - 1) >> 2)) { state = 2; break; }
+        case 1: {                                   // phase-1 tiles: up to 4 groups of one item, shared groups apart
+          const int n = nH + nT + nM;
+          if (li >= n) { state = 2; break; }
+          const int first = group_at(li);
+          int g = 1;
+          while (g < 4 && li + g < n && li + g != nH + nT && group_at(li + g) / NG == first / NG) ++g;
           op.kind = OP_P1;
-          window_part(op, W++, s_lo, s_hi);
-          op.j = 4 * op.W - op.item * NG + op.a;
-          op.g = op.b - op.a;
+          op.item = first / NG;
+          op.g = g;
+#pragma unroll
+          for (int q = 0; q < 4; ++q) op.grp[q] = q < g ? group_at(li + q) : first;
           op.tile = tile++;
+          li += g;
           return true;
+        }
         case 2:
           op.kind = OP_PUBLISH;
-          W = s_lo >> 2;
           state = 3;
           return true;
         case 3: {                                   // phase-2 jobs, one per window touched
-          if (W > ((s_hi - 1) >> 2)) { state = 0; break; }
-          const int w = W++;
-          if (w == (lo >> 2) && defer_head()) break;
-          if (p2(op, w, s_lo, s_hi)) return true;
+          if (single) {
+            const int n_mid = (nM + 3) >> 2;
+            const int n_jobs = (nT > 0) + (nH > 0) + n_mid;
+            if (ji >= n_jobs) { state = 0; break; }
+            int j = ji++;
+            int w;
+            if (nT > 0 && j == 0) w = (s_hi - 1) >> 2;
+            else {
+              j -= (nT > 0);
+              if (nH > 0 && j == 0) w = s_lo >> 2;
+              else w = (mid0 >> 2) + j - (nH > 0);
+            }
+            if (p2(op, w, s_lo, s_hi)) return true;
+          } else {
+            const int w = (s_lo >> 2) + ji;
+            if (w > ((s_hi - 1) >> 2)) { state = 0; break; }
+            ++ji;
+            if (w == (lo >> 2) && (lo & 3) != 0) { deferred = true; break; }
+            if (p2(op, w, s_lo, s_hi)) return true;
+          }
           break;
         }
         case 4:                                     // the head window, shared with the previous CTA, comes last
           state = 5;
-          if (lo < hi && defer_head() && p2(op, lo >> 2, lo, hi)) return true;
+          if (deferred && p2(op, lo >> 2, lo, hi)) return true;
           break;
         default:
           return false;
       }
     }
+  }
+};
+
+// The stages of the loader -> tensor-core ring, derived from the operation sequence.  The ring is
+// byte-granular: a stage takes what its tile needs (a 1-group tile a quarter of a 4-group tile), so
+// the bytes in flight do not shrink with the tile.  Placement is a pure function of the sequence;
+// the loaders and the MMA warp compute it independently.
+struct Stage {
+  int kind;            // OP_P1, OP_P2 or OP_PUBLISH (no bytes)
+  bool first, last;    // first / last stage of its operation
+  int k0, n;           // P1: first k-block, k-blocks;  P2: first W_down tile, tiles
+  uint32_t off;        // byte offset in the ring
+  uint32_t len;        // bytes reserved (including what a partial tile's 128-row reads run past its end)
+  uint32_t it, lap;    // running stage index; how often the ring wrapped before this stage
+};
+
+template <int NT>
+struct StageIter {
+  using C = TcCfg<NT>;
+  Walker walk;
+  Op op;
+  int KB, HT, pos, end;
+  bool have_op;
+  uint32_t cur, it, lap;
+  __device__ StageIter(int lo, int hi, int ng, int kb, int ht)
+      : walk(lo, hi, ng, ht, C::kScWindows), KB(kb), HT(ht), pos(0), end(0), have_op(false), cur(0), it(0), lap(0) {}
+  __device__ bool next(Stage& st) {
+    if (!have_op) {
+      if (!walk.next(op)) return false;
+      if (op.kind == OP_PUBLISH) {
+        st.kind = OP_PUBLISH;
+        return true;
+      }
+      have_op = true;
+      pos = op.kind == OP_P1 ? 0 : op.a * HT / 4;
+      end = op.kind == OP_P1 ? KB : op.b * HT / 4;
+      st.first = true;
+    } else {
+      st.first = false;
+    }
+    st.kind = op.kind;
+    st.k0 = pos;
+    st.n = min(C::kKbs, end - pos);
+    pos += C::kKbs;
+    st.last = pos >= end;
+    uint32_t bytes, over;
+    if (op.kind == OP_P1) {
+      bytes = (uint32_t)C::kKbs * (4096u * op.g + C::kBSub);
+      over = (uint32_t)(128 - 32 * op.g) * 128u;
+    } else {
+      bytes = (uint32_t)st.n * kATileBytes;
+      over = 0;
+    }
+    if (cur + bytes + over > (uint32_t)C::kRingBytes) {
+      cur = 0;
+      ++lap;
+    }
+    st.off = cur;
+    st.len = bytes + over;
+    st.lap = lap;
+    st.it = it++;
+    cur += bytes;
+    if (st.last) have_op = false;
+    return true;
   }
 };
 
@@ -293,14 +405,15 @@ k_experts_tc(TcArgs a) {
   using C = TcCfg<NT>;
   constexpr bool RES = C::kRes;
   constexpr int KBS = C::kKbs;
+  constexpr int NB = kRingBars;
   extern __shared__ unsigned char smem_dyn[];
   const Dims d = a.d;
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~uintptr_t(1023));
   unsigned char* act_buf = smem + C::kRingBytes;                                 // [kActBufs][NT][128 B]
   uint64_t* bars = reinterpret_cast<uint64_t*>(act_buf + C::kActBufs * C::kActBytes);
-  uint64_t* bar_full = bars;                                       // [kStages] loaders -> MMA
-  uint64_t* bar_empty = bars + C::kStages;                         // [kStages] MMA -> loaders
-  uint64_t* bar_acc1_full = bars + 2 * C::kStages;                 // [kScWindows]
+  uint64_t* bar_full = bars;                                       // [NB] loaders -> MMA
+  uint64_t* bar_empty = bars + NB;                                 // [NB] MMA -> loaders
+  uint64_t* bar_acc1_full = bars + 2 * NB;                         // [kScWindows]
   uint64_t* bar_acc1_empty = bar_acc1_full + C::kScWindows;        // [1]
   uint64_t* bar_act_full = bar_acc1_empty + 1;                     // [kActBufs]
   uint64_t* bar_act_empty = bar_act_full + C::kActBufs;            // [kActBufs]
@@ -319,7 +432,7 @@ k_experts_tc(TcArgs a) {
   const int WPI = NG / 4;           // windows per work item
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < C::kStages; ++s) {
+    for (int s = 0; s < NB; ++s) {
       mbar_init(smem_u32(bar_full + s), kLoaders * 32);
       mbar_init(smem_u32(bar_empty + s), 1);
     }
@@ -342,17 +455,6 @@ k_experts_tc(TcArgs a) {
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
-  if (RES && warp < kLoaders) {
-    // token rows T..15 of every stage's token tiles stay zero for the whole kernel
-    for (int i = threadIdx.x; i < C::kStages * KBS * (kResidentRows * 8); i += kLoaders * 32) {
-      const int ch = i & 7, r = (i >> 3) % kResidentRows, sub = (i >> 3) / kResidentRows;
-      if (r >= d.T) {
-        const uint32_t dst = smem_u32(smem + (sub / KBS) * C::kStageBytes + C::kABytes + (sub % KBS) * C::kBSub) + sw128(r, ch);
-        asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(dst), "r"(0) : "memory");
-      }
-    }
-    fence_async_smem();
-  }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -369,142 +471,153 @@ k_experts_tc(TcArgs a) {
     constexpr int RSTEP = kLoaders * RPI;   // rows between two instructions of one warp
     const int sub = lane / LPR, kbi = (lane >> 3) % KBS, ch = lane & 7;
     int32_t* my_rows = ld_row + warp * NT;
-    uint32_t it = 0;
-    int tbl_item = -1;
-    bool ok = true;
-    Walker walk(g_lo, g_hi, NG, HT, C::kScWindows);
-    Op op;
-    while (ok && walk.next(op)) {
-      if (op.kind == OP_PUBLISH) continue;
-      const WorkItem item = a.items[op.item];
-      if (op.kind == OP_P1) {
-        const int ncols = RES ? d.T : item.n;
-        if (!RES && op.item != tbl_item) {
-          __syncwarp();
-          for (int r = lane; r < item.n; r += 32) {
-            int row;
-            float wt;
-            slot_row_weight(a.perm[item.begin + r], d.T, d.k, a.topk_w, row, wt);
-            my_rows[r] = row;
-          }
-          __syncwarp();
-          tbl_item = op.item;
+    int tbl_item = -1, in_flight = 0;
+    bool ok = true, have_tail = false;
+    StageIter<NT> head(g_lo, g_hi, NG, KB, HT), tail(g_lo, g_hi, NG, KB, HT);
+    Stage st, ts;
+    size_t wrow[4] = {0, 0, 0, 0};          // first weight row of each group of the current tile
+    int ncols = 0;
+    while (ok && head.next(st)) {
+      if (st.kind == OP_PUBLISH) continue;
+      // make room: the oldest stages in flight are released by the MMA warp in order
+      while (in_flight > 0) {
+        if (!have_tail) {
+          do { tail.next(ts); } while (ts.kind == OP_PUBLISH);
+          have_tail = true;
         }
-        const int blocks = op.g * 2;                                  // 16-row blocks: [group][gate | up]
-        const size_t wrow0 = (size_t)item.e * d.I + (size_t)op.j * kGroupCols;
-        // Row r of the tile = block b (even: gate, odd: up; group b / 2) * 16 + rr.  This lane's rows inside
-        // a block are rr0, rr0 + RSTEP, ...: constant strides, so the copies of one block are independent.
-        const int rr0 = warp * RPI + sub;
-        const size_t rstep = (size_t)RSTEP * d.H;
-        for (int kb0 = 0; kb0 < KB; kb0 += KBS) {
-          const uint32_t s = it % C::kStages, par = (it / C::kStages) & 1;
-          if (!(ok = mbar_wait_warp(smem_u32(bar_empty + s), par ^ 1, abort_flag, a.status, 1))) break;
-          if (kb0 + kbi < KB) {
-            const uint32_t dstA = smem_u32(smem + s * C::kStageBytes) + kbi * kATileBytes;
-            const uint32_t dstB = smem_u32(smem + s * C::kStageBytes + C::kABytes) + kbi * C::kBSub;
-            const int koff = (kb0 + kbi) * 64 + ch * 8;
-            for (int b = 0; b < blocks; ++b) {
-              const __nv_bfloat16* src =
-                  ((b & 1) ? a.w_up : a.w_gate) + (wrow0 + (size_t)(b >> 1) * kGroupCols + rr0) * d.H + koff;
-              const uint32_t dst = dstA + (uint32_t)(b * 16 + rr0) * 128u;
+        const bool conflict = in_flight >= NB || ts.lap + 1 < st.lap || (ts.lap + 1 == st.lap && ts.off < st.off + st.len);
+        if (!conflict) break;
+        if (!(ok = mbar_wait_warp(smem_u32(bar_empty + ts.it % NB), (ts.it / NB) & 1, abort_flag, a.status, 1))) break;
+        have_tail = false;
+        --in_flight;
+      }
+      if (!ok) break;
+      const Op& op = head.op;
+      const uint32_t base = smem_u32(smem) + st.off;
+      if (st.kind == OP_P1) {
+        if (st.first) {
+          const WorkItem item = a.items[op.item];
+          ncols = RES ? d.T : item.n;
+          if (!RES && op.item != tbl_item) {
+            __syncwarp();
+            for (int r = lane; r < item.n; r += 32) {
+              int row;
+              float wt;
+              slot_row_weight(a.perm[item.begin + r], d.T, d.k, a.topk_w, row, wt);
+              my_rows[r] = row;
+            }
+            __syncwarp();
+            tbl_item = op.item;
+          }
 #pragma unroll
-              for (int ii = 0; ii < 16 / RSTEP; ++ii) {
-                const int rr = rr0 + ii * RSTEP;      // (b * 16 + rr) & 7 == rr & 7
-                cp_async16(dst + (uint32_t)(ii * RSTEP) * 128u + (uint32_t)((ch ^ (rr & 7)) << 4), src + ii * rstep);
+          for (int q = 0; q < 4; ++q)
+            wrow[q] = (size_t)item.e * d.I + (size_t)(op.grp[q] - op.item * NG) * kGroupCols;
+        }
+        if (st.k0 + kbi < KB) {
+          // Row r of the tile = 16-row block b (even: gate, odd: up; group b / 2) * 16 + rr.  This lane's rows
+          // inside a block are rr0, rr0 + RSTEP, ...: constant strides, so the copies of one block are independent.
+          const uint32_t sub_bytes = 4096u * op.g;                     // one k-block of the tile
+          const uint32_t dstA = base + kbi * sub_bytes;
+          const uint32_t dstB = base + KBS * sub_bytes + kbi * C::kBSub;
+          const int koff = (st.k0 + kbi) * 64 + ch * 8;
+          const int rr0 = warp * RPI + sub;
+          const size_t rstep = (size_t)RSTEP * d.H;
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            if (q < op.g) {
+#pragma unroll
+              for (int m = 0; m < 2; ++m) {
+                const __nv_bfloat16* src = (m ? a.w_up : a.w_gate) + (wrow[q] + rr0) * d.H + koff;
+                const uint32_t dst = dstA + (uint32_t)((q * 2 + m) * 16 + rr0) * 128u;
+#pragma unroll
+                for (int ii = 0; ii < 16 / RSTEP; ++ii) {
+                  const int rr = rr0 + ii * RSTEP;      // (block * 16 + rr) & 7 == rr & 7
+                  cp_async16(dst + (uint32_t)(ii * RSTEP) * 128u + (uint32_t)((ch ^ (rr & 7)) << 4), src + ii * rstep);
+                }
               }
             }
-            for (int r = rr0; r < ncols; r += RSTEP)
-              cp_async16(dstB + sw128(r, ch), a.x + (size_t)(RES ? r : my_rows[r]) * d.H + koff);
           }
-          cp_async_arrive(smem_u32(bar_full + s));     // the stage is handed over when this lane's copies land
-          ++it;
+          for (int r = rr0; r < ncols; r += RSTEP)
+            cp_async16(dstB + sw128(r, ch), a.x + (size_t)(RES ? r : my_rows[r]) * d.H + koff);
         }
       } else {
+        const WorkItem item = a.items[op.item];
         const int w = op.W - op.item * WPI;
-        const int ht0 = op.a * HT / 4, ht1 = op.b * HT / 4;
         // 4 rows x 128 B per warp instruction; this lane's rows r = r_first + 16 * ii share r & 7
         const int r_first = warp * 4 + (lane >> 3);
         const size_t rstep = (size_t)16 * d.I;
-        for (int t0 = ht0; t0 < ht1; t0 += KBS) {
-          const uint32_t s = it % C::kStages, par = (it / C::kStages) & 1;
-          if (!(ok = mbar_wait_warp(smem_u32(bar_empty + s), par ^ 1, abort_flag, a.status, 2))) break;
-          const int nt = min(KBS, ht1 - t0);
-          for (int i = 0; i < nt; ++i) {
-            const uint32_t dstA = smem_u32(smem + s * C::kStageBytes) + i * kATileBytes + sw128(r_first, ch);
-            const __nv_bfloat16* src =
-                a.w_down + ((size_t)item.e * d.H + (size_t)(t0 + i) * 128 + r_first) * d.I + w * kWindowCols + ch * 8;
+        for (int i = 0; i < st.n; ++i) {
+          const uint32_t dstA = base + i * kATileBytes + sw128(r_first, ch);
+          const __nv_bfloat16* src =
+              a.w_down + ((size_t)item.e * d.H + (size_t)(st.k0 + i) * 128 + r_first) * d.I + w * kWindowCols + ch * 8;
 #pragma unroll
-            for (int ii = 0; ii < 8; ++ii) cp_async16(dstA + (uint32_t)ii * 16u * 128u, src + ii * rstep);
-          }
-          cp_async_arrive(smem_u32(bar_full + s));
-          ++it;
+          for (int ii = 0; ii < 8; ++ii) cp_async16(dstA + (uint32_t)ii * 16u * 128u, src + ii * rstep);
         }
       }
+      cp_async_arrive(smem_u32(bar_full + st.it % NB));     // the stage is handed over when this lane's copies land
+      ++in_flight;
     }
     // everything still in flight lands before shared memory is released (also on abort)
     cp_async_wait_all();
   } else if (warp == kMmaWarp) {
     // ------------------------------ MMA issuer (whole warp converged, elected lane issues) ------------------------------
-    uint32_t it = 0, sc_i = 0, t2 = 0, jc = 0;
+    uint32_t sc_i = 0, t2 = 0, jc = 0, idesc = 0, ab = 0;
+    uint64_t act_desc = 0;
     bool ok = true;
-    Walker walk(g_lo, g_hi, NG, HT, C::kScWindows);
-    Op op;
-    while (ok && walk.next(op)) {
-      if (op.kind == OP_PUBLISH) { ++sc_i; continue; }
-      const WorkItem item = a.items[op.item];
-      const int N = RES ? kResidentRows : ((item.n + 15) & ~15);
-      const uint32_t idesc = make_idesc_bf16(N);
-      if (op.kind == OP_P1) {
-        if (op.tile == 0) {
+    StageIter<NT> si(g_lo, g_hi, NG, KB, HT);
+    Stage st;
+    while (ok && si.next(st)) {
+      if (st.kind == OP_PUBLISH) { ++sc_i; continue; }
+      const Op& op = si.op;
+      const uint32_t base = smem_u32(smem) + st.off;
+      if (st.first) {
+        const WorkItem item = a.items[op.item];
+        idesc = make_idesc_bf16(RES ? kResidentRows : ((item.n + 15) & ~15));
+      }
+      if (st.kind == OP_P1) {
+        if (st.first && op.tile == 0) {
           // the epilogue has read the previous super-chunk's accumulators
           if (!(ok = mbar_wait_warp(smem_u32(bar_acc1_empty), (sc_i & 1) ^ 1, abort_flag, a.status, 3))) break;
           tc_fence_after();
         }
-        const uint32_t acc1 = tmem_base + op.tile * NT;
-        for (int kb0 = 0; kb0 < KB; kb0 += KBS, ++it) {
-          const uint32_t s = it % C::kStages, par = (it / C::kStages) & 1;
-          if (!(ok = mbar_wait_warp(smem_u32(bar_full + s), par, abort_flag, a.status, 4))) break;
-          fence_async_smem();      // the loaders' cp.async writes (generic proxy) before the tensor core's reads
-          tc_fence_after();
-          const uint32_t sa = smem_u32(smem + s * C::kStageBytes);
-          const int n = min(KBS, KB - kb0);
-          for (int i = 0; i < n; ++i) {
-            const uint64_t da = make_kmajor_sw128_desc(sa + i * kATileBytes);
-            const uint64_t db = make_kmajor_sw128_desc(sa + C::kABytes + i * C::kBSub);
-#pragma unroll
-            for (int k4 = 0; k4 < 4; ++k4) tc_mma(acc1, da + 2 * k4, db + 2 * k4, idesc, ((kb0 + i) | k4) != 0);
-          }
-          tc_commit(smem_u32(bar_empty + s));
-        }
-        if (!ok) break;
-        tc_commit(smem_u32(bar_acc1_full + op.tile));
-      } else {
-        const uint32_t ab = jc % C::kActBufs;
-        if (!(ok = mbar_wait_warp(smem_u32(bar_act_full + ab), (jc / C::kActBufs) & 1, abort_flag, a.status, 6))) break;
+        if (!(ok = mbar_wait_warp(smem_u32(bar_full + st.it % NB), (st.it / NB) & 1, abort_flag, a.status, 4))) break;
+        fence_async_smem();      // the loaders' cp.async writes (generic proxy) before the tensor core's reads
         tc_fence_after();
-        const uint64_t act_desc = make_kmajor_sw128_desc(smem_u32(act_buf + ab * C::kActBytes));
-        const int ht0 = op.a * HT / 4, ht1 = op.b * HT / 4;
-        for (int t0 = ht0; ok && t0 < ht1; t0 += KBS, ++it) {
-          const uint32_t s = it % C::kStages, par = (it / C::kStages) & 1;
-          if (!(ok = mbar_wait_warp(smem_u32(bar_full + s), par, abort_flag, a.status, 8))) break;
-          fence_async_smem();
-          const int nt = min(KBS, ht1 - t0);
-          for (int i = 0; i < nt; ++i, ++t2) {
-            const uint32_t b = t2 % C::kAcc2, u = t2 / C::kAcc2;
-            if (!(ok = mbar_wait_warp(smem_u32(bar_acc2_empty + b), (u & 1) ^ 1, abort_flag, a.status, 7))) break;
-            tc_fence_after();
-            const uint64_t da = make_kmajor_sw128_desc(smem_u32(smem + s * C::kStageBytes) + i * kATileBytes);
-            const uint32_t acc2 = tmem_base + (C::kScWindows + b) * NT;
+        const uint32_t acc1 = tmem_base + op.tile * NT;
+        const uint32_t sub_bytes = 4096u * op.g;
+        for (int i = 0; i < st.n; ++i) {
+          const uint64_t da = make_kmajor_sw128_desc(base + i * sub_bytes);
+          const uint64_t db = make_kmajor_sw128_desc(base + KBS * sub_bytes + i * C::kBSub);
 #pragma unroll
-            for (int kk = 0; kk < 4; ++kk) tc_mma(acc2, da + 2 * kk, act_desc + 2 * kk, idesc, kk != 0);
-            tc_commit(smem_u32(bar_acc2_full + b));
-          }
-          if (!ok) break;
-          tc_commit(smem_u32(bar_empty + s));
+          for (int k4 = 0; k4 < 4; ++k4) tc_mma(acc1, da + 2 * k4, db + 2 * k4, idesc, ((st.k0 + i) | k4) != 0);
+        }
+        tc_commit(smem_u32(bar_empty + st.it % NB));
+        if (st.last) tc_commit(smem_u32(bar_acc1_full + op.tile));
+      } else {
+        if (st.first) {
+          ab = jc % C::kActBufs;
+          if (!(ok = mbar_wait_warp(smem_u32(bar_act_full + ab), (jc / C::kActBufs) & 1, abort_flag, a.status, 6))) break;
+          tc_fence_after();
+          act_desc = make_kmajor_sw128_desc(smem_u32(act_buf + ab * C::kActBytes));
+        }
+        if (!(ok = mbar_wait_warp(smem_u32(bar_full + st.it % NB), (st.it / NB) & 1, abort_flag, a.status, 8))) break;
+        fence_async_smem();
+        for (int i = 0; i < st.n; ++i, ++t2) {
+          const uint32_t b = t2 % C::kAcc2, u = t2 / C::kAcc2;
+          if (!(ok = mbar_wait_warp(smem_u32(bar_acc2_empty + b), (u & 1) ^ 1, abort_flag, a.status, 7))) break;
+          tc_fence_after();
+          const uint64_t da = make_kmajor_sw128_desc(base + i * kATileBytes);
+          const uint32_t acc2 = tmem_base + (C::kScWindows + b) * NT;
+#pragma unroll
+          for (int kk = 0; kk < 4; ++kk) tc_mma(acc2, da + 2 * kk, act_desc + 2 * kk, idesc, kk != 0);
+          tc_commit(smem_u32(bar_acc2_full + b));
         }
         if (!ok) break;
-        tc_commit(smem_u32(bar_act_empty + ab));
-        ++jc;
+        tc_commit(smem_u32(bar_empty + st.it % NB));
+        if (st.last) {
+          tc_commit(smem_u32(bar_act_empty + ab));
+          ++jc;
+        }
       }
     }
   } else if (warp == kActWarp) {
@@ -571,8 +684,12 @@ k_experts_tc(TcArgs a) {
         use1 ^= 1u << op.tile;
         tc_fence_after();
         if (q < op.g) {
-          const int col = (op.j + q) * kGroupCols + (lane & 15);     // intermediate column of this lane pair
-          const bool is_gate = lane < 16;                            // lanes 0-15 hold gate rows, 16-31 up rows
+          int grp = op.grp[0];                     // this warp's group
+#pragma unroll
+          for (int i = 1; i < 4; ++i)
+            if (i == q) grp = op.grp[i];
+          const int col = (grp - op.item * NG) * kGroupCols + (lane & 15);   // intermediate column of this lane pair
+          const bool is_gate = lane < 16;                                   // lanes 0-15 hold gate rows, 16-31 up rows
           __nv_bfloat16* dst = a.act_g + (size_t)op.item * NT * d.I + col;
           const uint32_t acc1 = tmem_base + op.tile * NT + lane_off;
           for (int c0 = 0; c0 < ncols; c0 += 8) {
@@ -597,7 +714,7 @@ k_experts_tc(TcArgs a) {
           __syncwarp();
           if (lane == 0) {
             __threadfence();
-            atomicAdd(a.win_flags + op.W, 1);
+            atomicAdd(a.win_flags + (grp >> 2), 1);
           }
         }
       } else if (op.kind == OP_PUBLISH) {
