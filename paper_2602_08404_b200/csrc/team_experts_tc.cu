@@ -27,7 +27,7 @@
 // publish ever waits on another CTA, so the waits cannot form a cycle; the launch is cooperative so
 // that all CTAs are resident, and every wait is bounded.
 //
-// Loads.  Four loader warps fill the ring with cp.async: every warp instruction fetches kKbs * 128
+// Loads.  Eight loader warps fill the ring with cp.async: every warp instruction fetches kKbs * 128
 // contiguous bytes of one weight row (phase 1) or 128-byte row pieces of four rows (phase 2) and
 // scatters them into the K-major, 128-byte-swizzled tiles the tensor core reads; the stage's
 // mbarrier is armed to fire when the copies land (cp.async.mbarrier.arrive), so a loader only ever
@@ -39,19 +39,19 @@
 //              to the expert get weight 0 in the combine.
 //   gather     (N = 16..NT): the loaders gather the item's token rows.
 //
-// Warp roles (384 threads): warps 0-3 = loaders, warp 4 = MMA issuer + TMEM owner (converged warp,
-// one elected lane issues), warp 5 = activation-window loader, warps 8-11 = epilogue (one TMEM lane
+// Warp roles (512 threads): warps 0-7 = loaders, warp 8 = MMA issuer + TMEM owner (converged warp,
+// one elected lane issues), warp 9 = activation-window loader, warps 12-15 = epilogue (one TMEM lane
 // quarter each).  On a wait's expiry the kernel records TEAM_ERR_TIMEOUT, drains and frees its
 // tensor memory.
 #include "team_common.cuh"
 
 namespace team {
 
-constexpr int kTcThreads = 384;
-constexpr int kLoaders = 4;                     // warps 0..3
-constexpr int kMmaWarp = 4;
-constexpr int kActWarp = 5;
-constexpr int kEpiWarp0 = 8;                    // warps 8..11 (warp % 4 = TMEM lane quarter)
+constexpr int kTcThreads = 512;
+constexpr int kLoaders = 8;                     // warps 0..7
+constexpr int kMmaWarp = 8;
+constexpr int kActWarp = 9;
+constexpr int kEpiWarp0 = 12;                   // warps 12..15 (warp % 4 = TMEM lane quarter)
 constexpr int kATileBytes = 128 * 128;          // 128 rows x 64 bf16
 constexpr int kGroupCols = 16;                  // intermediate columns per group (the unit of balance)
 constexpr int kWindowCols = 64;                 // columns per window (one 128-byte swizzle row of W_down)
@@ -75,7 +75,7 @@ struct TcCfg {
   static constexpr int kTmemCols = kTmemUsed <= 128 ? 128 : (kTmemUsed <= 256 ? 256 : 512);
   static constexpr int kNumBars = 2 * kRingBars + kScWindows + 1 + 2 * kActBufs + 2 * kAcc2;
   static constexpr int kBarBytes = ((kNumBars * 8 + 15) / 16) * 16;
-  static constexpr int kTableBytes = 4 * NT * 8 + kLoaders * NT * 4;   // epilogue (row, weight) + loader row tables
+  static constexpr int kTableBytes = 4 * NT * 8 + kLoaders * NT * 4 + kLoaders * kRingBars * 16;   // epilogue (row, weight), loader rows, loader stage queues
   static constexpr int kOtherBytes = 1024 + kActBufs * kActBytes + kBarBytes + kTableBytes + 64;
   static constexpr int kRingBytes = ((kMaxSmemBytes - kOtherBytes) / 1024) * 1024;   // everything that is left
   static constexpr int kSmemBytes = kOtherBytes + kRingBytes;
@@ -190,6 +190,23 @@ __device__ __forceinline__ void tmem_ld8(uint32_t taddr, float (&v)[8]) {
   v[4] = __uint_as_float(r4); v[5] = __uint_as_float(r5); v[6] = __uint_as_float(r6); v[7] = __uint_as_float(r7);
 }
 
+// The same load without the wait: the registers are valid only after tmem_ld_wait on them.
+__device__ __forceinline__ void tmem_ld8_issue(uint32_t taddr, uint32_t (&r)[8]) {
+  asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+               : "r"(taddr));
+}
+// Waits for all tensor-memory loads of this thread; the operands tie the loaded registers to the wait.
+__device__ __forceinline__ void tmem_ld_wait(uint32_t (&a)[8], uint32_t (&b)[8], uint32_t (&c)[8], uint32_t (&d)[8]) {
+  asm volatile("tcgen05.wait::ld.sync.aligned;"
+               : "+r"(a[0]), "+r"(a[1]), "+r"(a[2]), "+r"(a[3]), "+r"(a[4]), "+r"(a[5]), "+r"(a[6]), "+r"(a[7]),
+                 "+r"(b[0]), "+r"(b[1]), "+r"(b[2]), "+r"(b[3]), "+r"(b[4]), "+r"(b[5]), "+r"(b[6]), "+r"(b[7]),
+                 "+r"(c[0]), "+r"(c[1]), "+r"(c[2]), "+r"(c[3]), "+r"(c[4]), "+r"(c[5]), "+r"(c[6]), "+r"(c[7]),
+                 "+r"(d[0]), "+r"(d[1]), "+r"(d[2]), "+r"(d[3]), "+r"(d[4]), "+r"(d[5]), "+r"(d[6]), "+r"(d[7])
+               :
+               : "memory");
+}
+
 __device__ __forceinline__ int ld_acquire(const int32_t* p) {
   int v;
   asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
@@ -241,20 +258,39 @@ struct Op {
 struct Walker {
   int lo, hi, NG, HT, scw;
   int s_lo, s_hi, nH, nT, nM, tail0, mid0, li, ji, tile, state;
+  int item0, base0;     // item of the super-chunk's first group and that item's first group
   bool single, deferred;
   __device__ Walker(int lo_, int hi_, int ng, int ht, int sc_windows)
       : lo(lo_), hi(hi_), NG(ng), HT(ht), scw(sc_windows), s_lo(lo_), s_hi(lo_), nH(0), nT(0), nM(0), tail0(0),
-        mid0(0), li(0), ji(0), tile(0), state(0), single(false), deferred(false) {}
+        mid0(0), li(0), ji(0), tile(0), state(0), item0(lo_ / ng), base0((lo_ / ng) * ng), single(false),
+        deferred(false) {}
+  // item of a group at or after the super-chunk's first group (no division: a super-chunk spans few items)
+  __device__ int item_of(int grp) const {
+    int it = item0, b = base0 + NG;
+    while (grp >= b) {
+      b += NG;
+      ++it;
+    }
+    return it;
+  }
   // phase-1 order of the super-chunk: head part, tail part, middle
   __device__ int group_at(int i) const {
     return i < nH ? s_lo + i : (i < nH + nT ? tail0 + (i - nH) : mid0 + (i - nH - nT));
+  }
+  __device__ int lo_item() const {     // the deferred head job comes after the last super-chunk: count down
+    int it = item0, b = base0;
+    while (lo < b) {                   // never taken unless the walk moved past lo's item
+      b -= NG;
+      --it;
+    }
+    return it;
   }
   __device__ bool p2(Op& op, int w, int from, int to) const {
     op.kind = OP_P2;
     op.W = w;
     op.a = max(from, 4 * w) - 4 * w;
     op.b = min(to, 4 * w + 4) - 4 * w;
-    op.item = (4 * w) / NG;
+    op.item = w == (lo >> 2) ? lo_item() : item_of(4 * w);
     return op.a * HT / 4 < op.b * HT / 4;     // jobs without a tile are skipped
   }
   __device__ bool next(Op& op) {
@@ -264,6 +300,10 @@ struct Walker {
           if (s_hi >= hi) { state = 4; break; }
           s_lo = s_hi;
           s_hi = min(hi, ((s_lo >> 2) + scw) << 2);
+          while (s_lo >= base0 + NG) {              // item of the new first group
+            base0 += NG;
+            ++item0;
+          }
           single = (s_lo == lo && s_hi == hi);
           if (single) {
             nH = (s_lo & 3) ? min(s_hi, (s_lo | 3) + 1) - s_lo : 0;
@@ -286,10 +326,11 @@ struct Walker {
           const int n = nH + nT + nM;
           if (li >= n) { state = 2; break; }
           const int first = group_at(li);
+          const int first_item = item_of(first);
           int g = 1;
-          while (g < 4 && li + g < n && li + g != nH + nT && group_at(li + g) / NG == first / NG) ++g;
+          while (g < 4 && li + g < n && li + g != nH + nT && item_of(group_at(li + g)) == first_item) ++g;
           op.kind = OP_P1;
-          op.item = first / NG;
+          op.item = first_item;
           op.g = g;
 #pragma unroll
           for (int q = 0; q < 4; ++q) op.grp[q] = q < g ? group_at(li + q) : first;
@@ -422,7 +463,8 @@ k_experts_tc(TcArgs a) {
   int32_t* tbl_row = reinterpret_cast<int32_t*>(reinterpret_cast<unsigned char*>(bars) + C::kBarBytes);   // [4][NT]
   float* tbl_wt = reinterpret_cast<float*>(tbl_row + 4 * NT);                                             // [4][NT]
   int32_t* ld_row = reinterpret_cast<int32_t*>(tbl_wt + 4 * NT);                                          // [kLoaders][NT]
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(ld_row + kLoaders * NT);
+  uint4* ld_queue = reinterpret_cast<uint4*>(ld_row + kLoaders * NT);                                     // [kLoaders][kRingBars]
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(ld_queue + kLoaders * kRingBars);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -437,14 +479,14 @@ k_experts_tc(TcArgs a) {
       mbar_init(smem_u32(bar_empty + s), 1);
     }
     for (int i = 0; i < C::kScWindows; ++i) mbar_init(smem_u32(bar_acc1_full + i), 1);
-    mbar_init(smem_u32(bar_acc1_empty), 128);
+    mbar_init(smem_u32(bar_acc1_empty), 4);
     for (int i = 0; i < C::kActBufs; ++i) {
       mbar_init(smem_u32(bar_act_full + i), 32);
       mbar_init(smem_u32(bar_act_empty + i), 1);
     }
     for (int i = 0; i < C::kAcc2; ++i) {
       mbar_init(smem_u32(bar_acc2_full + i), 1);
-      mbar_init(smem_u32(bar_acc2_empty + i), 128);
+      mbar_init(smem_u32(bar_acc2_empty + i), 4);
     }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -471,27 +513,28 @@ k_experts_tc(TcArgs a) {
     constexpr int RSTEP = kLoaders * RPI;   // rows between two instructions of one warp
     const int sub = lane / LPR, kbi = (lane >> 3) % KBS, ch = lane & 7;
     int32_t* my_rows = ld_row + warp * NT;
+    uint4* my_queue = ld_queue + warp * NB;     // (offset, lap, index) of this warp's stages in flight, oldest first
     int tbl_item = -1, in_flight = 0;
-    bool ok = true, have_tail = false;
-    StageIter<NT> head(g_lo, g_hi, NG, KB, HT), tail(g_lo, g_hi, NG, KB, HT);
-    Stage st, ts;
+    uint32_t q_tail = 0;                        // running index of the oldest stage in flight
+    bool ok = true;
+    StageIter<NT> head(g_lo, g_hi, NG, KB, HT);
+    Stage st;
     size_t wrow[4] = {0, 0, 0, 0};          // first weight row of each group of the current tile
     int ncols = 0;
     while (ok && head.next(st)) {
       if (st.kind == OP_PUBLISH) continue;
       // make room: the oldest stages in flight are released by the MMA warp in order
       while (in_flight > 0) {
-        if (!have_tail) {
-          do { tail.next(ts); } while (ts.kind == OP_PUBLISH);
-          have_tail = true;
-        }
-        const bool conflict = in_flight >= NB || ts.lap + 1 < st.lap || (ts.lap + 1 == st.lap && ts.off < st.off + st.len);
+        const uint4 ts = my_queue[q_tail % NB];   // x: offset, y: lap
+        const bool conflict = in_flight >= NB || ts.y + 1 < st.lap || (ts.y + 1 == st.lap && ts.x < st.off + st.len);
         if (!conflict) break;
-        if (!(ok = mbar_wait_warp(smem_u32(bar_empty + ts.it % NB), (ts.it / NB) & 1, abort_flag, a.status, 1))) break;
-        have_tail = false;
+        if (!(ok = mbar_wait_warp(smem_u32(bar_empty + q_tail % NB), (q_tail / NB) & 1, abort_flag, a.status, 1))) break;
+        ++q_tail;
         --in_flight;
       }
       if (!ok) break;
+      if (lane == 0) my_queue[st.it % NB] = make_uint4(st.off, st.lap, 0u, 0u);
+      __syncwarp();
       const Op& op = head.op;
       const uint32_t base = smem_u32(smem) + st.off;
       if (st.kind == OP_P1) {
@@ -543,15 +586,16 @@ k_experts_tc(TcArgs a) {
       } else {
         const WorkItem item = a.items[op.item];
         const int w = op.W - op.item * WPI;
-        // 4 rows x 128 B per warp instruction; this lane's rows r = r_first + 16 * ii share r & 7
+        // 4 rows x 128 B per warp instruction; this lane's rows r = r_first + 4 * kLoaders * ii share r & 7
         const int r_first = warp * 4 + (lane >> 3);
-        const size_t rstep = (size_t)16 * d.I;
+        const size_t rstep = (size_t)(4 * kLoaders) * d.I;
         for (int i = 0; i < st.n; ++i) {
           const uint32_t dstA = base + i * kATileBytes + sw128(r_first, ch);
           const __nv_bfloat16* src =
               a.w_down + ((size_t)item.e * d.H + (size_t)(st.k0 + i) * 128 + r_first) * d.I + w * kWindowCols + ch * 8;
 #pragma unroll
-          for (int ii = 0; ii < 8; ++ii) cp_async16(dstA + (uint32_t)ii * 16u * 128u, src + ii * rstep);
+          for (int ii = 0; ii < 128 / (4 * kLoaders); ++ii)
+            cp_async16(dstA + (uint32_t)(ii * 4 * kLoaders) * 128u, src + ii * rstep);
         }
       }
       cp_async_arrive(smem_u32(bar_full + st.it % NB));     // the stage is handed over when this lane's copies land
@@ -720,7 +764,8 @@ k_experts_tc(TcArgs a) {
       } else if (op.kind == OP_PUBLISH) {
         // the super-chunk's accumulators are free again
         tc_fence_before();
-        mbar_arrive(smem_u32(bar_acc1_empty));
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(bar_acc1_empty));
       } else {
         // ---- down projection tiles: scale by routing weight, add into y ----
         const WorkItem item = a.items[op.item];
@@ -748,7 +793,48 @@ k_experts_tc(TcArgs a) {
           __syncwarp();
           tbl_item = op.item;
         }
-        for (int ht = op.a * HT / 4; ht < op.b * HT / 4; ++ht, ++t2) {
+        const int ht1 = op.b * HT / 4;
+        int ht = op.a * HT / 4;
+        // Few columns: a tile's epilogue is one short tensor-memory load, so up to four tiles are taken per
+        // round (their loads in flight together, one wait) instead of paying the load latency per tile.
+        while (ncols <= 8 && ht < ht1) {
+          const int nb = min(C::kAcc2 < 4 ? C::kAcc2 : 4, ht1 - ht);     // never more than the MMA warp can run ahead
+          uint32_t r[4][8];
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            if (i < nb && ok) {
+              const uint32_t b = (t2 + i) % C::kAcc2, u = (t2 + i) / C::kAcc2;
+              ok = mbar_wait_warp(smem_u32(bar_acc2_full + b), u & 1, abort_flag, a.status, 11);
+              if (ok) {
+                tc_fence_after();
+                tmem_ld8_issue(tmem_base + (C::kScWindows + b) * NT + lane_off, r[i]);
+              }
+            }
+          }
+          if (!ok) break;
+          tmem_ld_wait(r[0], r[1], r[2], r[3]);
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            if (i < nb) {
+              float* ycol = a.y + (ht + i) * 128 + q * 32 + lane;
+#pragma unroll
+              for (int j = 0; j < 8; ++j) {
+                if (j < ncols) {
+                  const float wt = my_wt[j];
+                  if (wt != 0.f) atomicAdd(ycol + (size_t)my_row[j] * d.H, wt * __uint_as_float(r[i][j]));
+                }
+              }
+            }
+          }
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0)
+            for (int i = 0; i < nb; ++i) mbar_arrive(smem_u32(bar_acc2_empty + (t2 + i) % C::kAcc2));
+          ht += nb;
+          t2 += nb;
+        }
+        if (!ok) break;
+        for (; ht < ht1; ++ht, ++t2) {
           const uint32_t b = t2 % C::kAcc2, u = t2 / C::kAcc2;
           ok = mbar_wait_warp(smem_u32(bar_acc2_full + b), u & 1, abort_flag, a.status, 11);
           if (!ok) break;
@@ -768,7 +854,8 @@ k_experts_tc(TcArgs a) {
             }
           }
           tc_fence_before();
-          mbar_arrive(smem_u32(bar_acc2_empty + b));
+          __syncwarp();
+          if (lane == 0) mbar_arrive(smem_u32(bar_acc2_empty + b));
         }
       }
     }
