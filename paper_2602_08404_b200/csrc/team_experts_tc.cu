@@ -104,15 +104,20 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
-// Bounded wait.  Returns false when it gave up (or another thread of the CTA already did).
+// Bounded wait.  Returns false when it gave up (or another thread of the CTA already did).  Every role
+// but the MMA issuer backs off between polls (kSleepNs): spinning warps take issue slots from the
+// warp that feeds the tensor core.
+template <int kSleepNs = 0>
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status,
                                           int where) {
   if (mbar_try(bar, parity)) return true;
   const unsigned long long t0 = clock64();
   for (;;) {
 #pragma unroll 1
-    for (int i = 0; i < 64; ++i)
+    for (int i = 0; i < 64; ++i) {
       if (mbar_try(bar, parity)) return true;
+      if (kSleepNs > 0) __nanosleep(kSleepNs);
+    }
     if (*abort_flag) return false;
     if (clock64() - t0 > kWaitCycles) {
       *abort_flag = 1;
@@ -122,9 +127,10 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
   }
 }
 // The same for a whole converged warp: every lane returns the same answer.
+template <int kSleepNs = 0>
 __device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status,
                                                int where) {
-  return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag, status, where));
+  return __all_sync(0xffffffffu, mbar_wait<kSleepNs>(bar, parity, abort_flag, status, where));
 }
 
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
@@ -528,7 +534,7 @@ k_experts_tc(TcArgs a) {
         const uint4 ts = my_queue[q_tail % NB];   // x: offset, y: lap
         const bool conflict = in_flight >= NB || ts.y + 1 < st.lap || (ts.y + 1 == st.lap && ts.x < st.off + st.len);
         if (!conflict) break;
-        if (!(ok = mbar_wait_warp(smem_u32(bar_empty + q_tail % NB), (q_tail / NB) & 1, abort_flag, a.status, 1))) break;
+        if (!(ok = mbar_wait_warp<64>(smem_u32(bar_empty + q_tail % NB), (q_tail / NB) & 1, abort_flag, a.status, 1))) break;
         ++q_tail;
         --in_flight;
       }
@@ -625,7 +631,8 @@ k_experts_tc(TcArgs a) {
           tc_fence_after();
         }
         if (!(ok = mbar_wait_warp(smem_u32(bar_full + st.it % NB), (st.it / NB) & 1, abort_flag, a.status, 4))) break;
-        fence_async_smem();      // the loaders' cp.async writes (generic proxy) before the tensor core's reads
+        // The barrier fires when the loaders' cp.async copies have landed in shared memory (completion-
+        // triggered arrival), so the tiles are in place for the tensor core without a further proxy fence.
         tc_fence_after();
         const uint32_t acc1 = tmem_base + op.tile * NT;
         const uint32_t sub_bytes = 4096u * op.g;
@@ -645,7 +652,6 @@ k_experts_tc(TcArgs a) {
           act_desc = make_kmajor_sw128_desc(smem_u32(act_buf + ab * C::kActBytes));
         }
         if (!(ok = mbar_wait_warp(smem_u32(bar_full + st.it % NB), (st.it / NB) & 1, abort_flag, a.status, 8))) break;
-        fence_async_smem();
         for (int i = 0; i < st.n; ++i, ++t2) {
           const uint32_t b = t2 % C::kAcc2, u = t2 / C::kAcc2;
           if (!(ok = mbar_wait_warp(smem_u32(bar_acc2_empty + b), (u & 1) ^ 1, abort_flag, a.status, 7))) break;
@@ -674,13 +680,14 @@ k_experts_tc(TcArgs a) {
       if (op.kind != OP_P2) continue;
       const WorkItem item = a.items[op.item];
       const uint32_t ab = jc % C::kActBufs;
-      ok = mbar_wait(smem_u32(bar_act_empty + ab), ((jc / C::kActBufs) & 1) ^ 1, abort_flag, a.status, 14);
+      ok = mbar_wait<64>(smem_u32(bar_act_empty + ab), ((jc / C::kActBufs) & 1) ^ 1, abort_flag, a.status, 14);
       // all four groups of the window published (by this CTA and / or its neighbours)?
       if (ok && lane == 0) {
         const int32_t* flag = a.win_flags + op.W;
         if (ld_acquire(flag) < 4) {
           const unsigned long long t0 = clock64();
           while (ld_acquire(flag) < 4) {
+            __nanosleep(64);
             if (*abort_flag) { ok = false; break; }
             if (clock64() - t0 > kWaitCycles) {
               *abort_flag = 1;
@@ -723,7 +730,7 @@ k_experts_tc(TcArgs a) {
         // ---- SwiGLU: TMEM -> registers -> bf16 activations in the global scratch ----
         const WorkItem item = a.items[op.item];
         const int ncols = RES ? d.T : item.n;
-        ok = mbar_wait_warp(smem_u32(bar_acc1_full + op.tile), (use1 >> op.tile) & 1, abort_flag, a.status, 10);
+        ok = mbar_wait_warp<32>(smem_u32(bar_acc1_full + op.tile), (use1 >> op.tile) & 1, abort_flag, a.status, 10);
         if (!ok) break;
         use1 ^= 1u << op.tile;
         tc_fence_after();
@@ -804,7 +811,7 @@ k_experts_tc(TcArgs a) {
           for (int i = 0; i < 4; ++i) {
             if (i < nb && ok) {
               const uint32_t b = (t2 + i) % C::kAcc2, u = (t2 + i) / C::kAcc2;
-              ok = mbar_wait_warp(smem_u32(bar_acc2_full + b), u & 1, abort_flag, a.status, 11);
+              ok = mbar_wait_warp<32>(smem_u32(bar_acc2_full + b), u & 1, abort_flag, a.status, 11);
               if (ok) {
                 tc_fence_after();
                 tmem_ld8_issue(tmem_base + (C::kScWindows + b) * NT + lane_off, r[i]);
@@ -836,7 +843,7 @@ k_experts_tc(TcArgs a) {
         if (!ok) break;
         for (; ht < ht1; ++ht, ++t2) {
           const uint32_t b = t2 % C::kAcc2, u = t2 / C::kAcc2;
-          ok = mbar_wait_warp(smem_u32(bar_acc2_full + b), u & 1, abort_flag, a.status, 11);
+          ok = mbar_wait_warp<32>(smem_u32(bar_acc2_full + b), u & 1, abort_flag, a.status, 11);
           if (!ok) break;
           tc_fence_after();
           const uint32_t acc2 = tmem_base + (C::kScWindows + b) * NT + lane_off;
