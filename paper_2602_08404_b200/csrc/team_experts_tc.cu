@@ -432,6 +432,9 @@ struct StageIter {
       bytes = (uint32_t)st.n * kATileBytes;
       over = 0;
     }
+    // Large stages sit on a grid of full-stage slots, so that the ring always holds as many of them as
+    // fit (small stages placed before them would otherwise leave the last slot a few KB short).
+    if (2 * bytes > (uint32_t)C::kStageBytes) cur = (cur + C::kStageBytes - 1) / C::kStageBytes * C::kStageBytes;
     if (cur + bytes + over > (uint32_t)C::kRingBytes) {
       cur = 0;
       ++lap;
@@ -507,6 +510,9 @@ k_experts_tc(TcArgs a) {
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  // Everything above overlaps the selection kernel (programmatic dependent launch); its tables are
+  // complete and visible from here on.
+  asm volatile("griddepcontrol.wait;" ::: "memory");
 
   // This CTA's contiguous range of groups.
   const long long n_groups = (long long)(*a.n_items) * NG;
@@ -525,8 +531,18 @@ k_experts_tc(TcArgs a) {
     bool ok = true;
     StageIter<NT> head(g_lo, g_hi, NG, KB, HT);
     Stage st;
-    size_t wrow[4] = {0, 0, 0, 0};          // first weight row of each group of the current tile
+    // Per tile (phase 1) or job (phase 2) this lane's source pointers are formed once; a stage then only
+    // adds its k offset (phase 1) or steps to the next tile (phase 2).
+    const __nv_bfloat16* src1[4][2];        // phase 1: [group][gate, up], this lane's first row and 16-byte piece
+    const __nv_bfloat16* src2 = nullptr;    // phase 2: this lane's first row of the next W_down tile
+    const int rr0 = warp * RPI + sub;       // phase 1: first row inside a 16-row block; the others follow RSTEP apart
+    const uint32_t dst1 = (uint32_t)rr0 * 128u + (uint32_t)((ch ^ (rr0 & 7)) << 4);   // (RSTEP is a multiple of 8: same swizzle)
+    const int r_first = warp * 4 + (lane >> 3);                                       // phase 2: 4 rows x 128 B per instruction
+    const uint32_t dst2 = sw128(r_first, ch);
+    const size_t rstep1 = (size_t)RSTEP * d.H, rstep2 = (size_t)(4 * kLoaders) * d.I, tstep2 = (size_t)128 * d.I;
     int ncols = 0;
+#pragma unroll
+    for (int q = 0; q < 4; ++q) src1[q][0] = src1[q][1] = nullptr;
     while (ok && head.next(st)) {
       if (st.kind == OP_PUBLISH) continue;
       // make room: the oldest stages in flight are released by the MMA warp in order
@@ -558,50 +574,45 @@ k_experts_tc(TcArgs a) {
             __syncwarp();
             tbl_item = op.item;
           }
+          // row r of the tile = 16-row block (2 * group + (0: gate, 1: up)) * 16 + rr
 #pragma unroll
-          for (int q = 0; q < 4; ++q)
-            wrow[q] = (size_t)item.e * d.I + (size_t)(op.grp[q] - op.item * NG) * kGroupCols;
+          for (int q = 0; q < 4; ++q) {
+            const size_t off = ((size_t)item.e * d.I + (size_t)(op.grp[q] - op.item * NG) * kGroupCols + rr0) * d.H +
+                               kbi * 64 + ch * 8;
+            src1[q][0] = a.w_gate + off;
+            src1[q][1] = a.w_up + off;
+          }
         }
         if (st.k0 + kbi < KB) {
-          // Row r of the tile = 16-row block b (even: gate, odd: up; group b / 2) * 16 + rr.  This lane's rows
-          // inside a block are rr0, rr0 + RSTEP, ...: constant strides, so the copies of one block are independent.
           const uint32_t sub_bytes = 4096u * op.g;                     // one k-block of the tile
-          const uint32_t dstA = base + kbi * sub_bytes;
-          const uint32_t dstB = base + KBS * sub_bytes + kbi * C::kBSub;
-          const int koff = (st.k0 + kbi) * 64 + ch * 8;
-          const int rr0 = warp * RPI + sub;
-          const size_t rstep = (size_t)RSTEP * d.H;
+          const uint32_t dstA = base + kbi * sub_bytes + dst1;
+          const int koff = st.k0 * 64;
 #pragma unroll
           for (int q = 0; q < 4; ++q) {
             if (q < op.g) {
 #pragma unroll
               for (int m = 0; m < 2; ++m) {
-                const __nv_bfloat16* src = (m ? a.w_up : a.w_gate) + (wrow[q] + rr0) * d.H + koff;
-                const uint32_t dst = dstA + (uint32_t)((q * 2 + m) * 16 + rr0) * 128u;
 #pragma unroll
-                for (int ii = 0; ii < 16 / RSTEP; ++ii) {
-                  const int rr = rr0 + ii * RSTEP;      // (block * 16 + rr) & 7 == rr & 7
-                  cp_async16(dst + (uint32_t)(ii * RSTEP) * 128u + (uint32_t)((ch ^ (rr & 7)) << 4), src + ii * rstep);
-                }
+                for (int ii = 0; ii < 16 / RSTEP; ++ii)
+                  cp_async16(dstA + (uint32_t)(((q * 2 + m) * 16 + ii * RSTEP) * 128), src1[q][m] + koff + ii * rstep1);
               }
             }
           }
+          const uint32_t dstB = base + KBS * sub_bytes + kbi * C::kBSub;
           for (int r = rr0; r < ncols; r += RSTEP)
-            cp_async16(dstB + sw128(r, ch), a.x + (size_t)(RES ? r : my_rows[r]) * d.H + koff);
+            cp_async16(dstB + sw128(r, ch), a.x + (size_t)(RES ? r : my_rows[r]) * d.H + (koff + kbi * 64 + ch * 8));
         }
       } else {
-        const WorkItem item = a.items[op.item];
-        const int w = op.W - op.item * WPI;
-        // 4 rows x 128 B per warp instruction; this lane's rows r = r_first + 4 * kLoaders * ii share r & 7
-        const int r_first = warp * 4 + (lane >> 3);
-        const size_t rstep = (size_t)(4 * kLoaders) * d.I;
-        for (int i = 0; i < st.n; ++i) {
-          const uint32_t dstA = base + i * kATileBytes + sw128(r_first, ch);
-          const __nv_bfloat16* src =
-              a.w_down + ((size_t)item.e * d.H + (size_t)(st.k0 + i) * 128 + r_first) * d.I + w * kWindowCols + ch * 8;
+        if (st.first) {
+          const WorkItem item = a.items[op.item];
+          src2 = a.w_down + ((size_t)item.e * d.H + (size_t)st.k0 * 128 + r_first) * d.I +
+                 (op.W - op.item * WPI) * kWindowCols + ch * 8;
+        }
+        for (int i = 0; i < st.n; ++i, src2 += tstep2) {
+          const uint32_t dstA = base + i * kATileBytes + dst2;
 #pragma unroll
           for (int ii = 0; ii < 128 / (4 * kLoaders); ++ii)
-            cp_async16(dstA + (uint32_t)(ii * 4 * kLoaders) * 128u, src + ii * rstep);
+            cp_async16(dstA + (uint32_t)(ii * 4 * kLoaders) * 128u, src2 + ii * rstep2);
         }
       }
       cp_async_arrive(smem_u32(bar_full + st.it % NB));     // the stage is handed over when this lane's copies land
@@ -892,14 +903,28 @@ int experts_tc_item_tile(int max_rows) {
 template <int NT>
 static cudaError_t launch_tc(TcArgs args, int grid, cudaStream_t s) {
   // Cooperative: CTAs that share a window wait for each other's activations, so all must be resident.
-  void* params[1] = {&args};
-  return cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(&k_experts_tc<NT>), dim3(grid), dim3(kTcThreads),
-                                     params, (size_t)TcCfg<NT>::kSmemBytes, s);
+  // Programmatic serialization: the CTAs may start their prologue while the selection kernel still runs.
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(grid);
+  cfg.blockDim = dim3(kTcThreads);
+  cfg.dynamicSmemBytes = (size_t)TcCfg<NT>::kSmemBytes;
+  cfg.stream = s;
+  cudaLaunchAttribute attrs[2];
+  attrs[0].id = cudaLaunchAttributeCooperative;
+  attrs[0].val.cooperative = 1;
+  attrs[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attrs[1].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attrs;
+  cfg.numAttrs = 2;
+  return cudaLaunchKernelEx(&cfg, k_experts_tc<NT>, args);
 }
 
 template <int NT>
 static cudaError_t configure_tc() {
-  return cudaFuncSetAttribute(k_experts_tc<NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, TcCfg<NT>::kSmemBytes);
+  cudaError_t e = cudaFuncSetAttribute(k_experts_tc<NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, TcCfg<NT>::kSmemBytes);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(k_experts_tc<NT>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+  return e;
 }
 
 cudaError_t configure_experts_tc(int item_tile) {

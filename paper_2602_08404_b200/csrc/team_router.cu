@@ -20,6 +20,7 @@ __global__ void __launch_bounds__(kExpertsPerCta * 32)
 k_router_logits(const XT* __restrict__ x, const float* __restrict__ w_router, const uint8_t* __restrict__ tok_state,
                 float* __restrict__ logits, float* __restrict__ y_zero, Dims d, int flags) {
   extern __shared__ __align__(16) float s_x[];   // [kRowTile][H]
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the selection kernel may stage its inputs meanwhile
   const int t0 = blockIdx.y * kRowTile;
   const int nt = min(kRowTile, d.T - t0);
   const int tid = threadIdx.x;
@@ -92,6 +93,7 @@ k_router_logits_small(const XT* __restrict__ x, const float* __restrict__ w_rout
                       const uint8_t* __restrict__ tok_state, float* __restrict__ logits, float* __restrict__ y_zero,
                       Dims d, int flags) {
   extern __shared__ __align__(16) float s_x[];   // [T][H] then partial sums
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the selection kernel may stage its inputs meanwhile
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int H = d.H, T = d.T;
   const int e = blockIdx.x * kSmallExperts + warp / kSmallSplit;
@@ -215,18 +217,28 @@ static bool small_router_ok(const Dims& d) {
   return d.T <= kRowTile && d.H % (4 * kSmallSplit) == 0 && d.H / (4 * kSmallSplit) <= 32 * kSmallMaxVec;
 }
 
+// All kernels of the layer ask for the largest shared-memory carve-out, as the expert kernel must:
+// an SM whose carve-out differs from what the next kernel prefers is drained and reconfigured first.
+template <typename K>
+static cudaError_t prepare_kernel(K kernel, int smem) {
+  cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+  return e;
+}
+
 cudaError_t configure_router(int dtype, int hidden) {
   const int smem = kRowTile * hidden * (int)sizeof(float) + 1024;
   cudaError_t e;
   if (dtype == TEAM_DTYPE_F32) {
-    e = cudaFuncSetAttribute(k_router_logits<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-    if (e == cudaSuccess)
-      e = cudaFuncSetAttribute(k_router_logits_small<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    e = prepare_kernel(k_router_logits<float>, smem);
+    if (e == cudaSuccess) e = prepare_kernel(k_router_logits_small<float>, smem);
   } else {
-    e = cudaFuncSetAttribute(k_router_logits<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-    if (e == cudaSuccess)
-      e = cudaFuncSetAttribute(k_router_logits_small<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    e = prepare_kernel(k_router_logits<__nv_bfloat16>, smem);
+    if (e == cudaSuccess) e = prepare_kernel(k_router_logits_small<__nv_bfloat16>, smem);
   }
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(k_router_topk, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
   return e;
 }
 

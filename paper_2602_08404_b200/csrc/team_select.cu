@@ -76,6 +76,8 @@ k_select(const float* __restrict__ logits, StepPtrs st, Workspace ws, RoutePtrs 
   sel_smem_layout(d, &s, smem_raw);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int T = d.T, E = d.E, k = d.k, ns = d.ns, EN = d.E + d.ns;
+  // the expert kernel may be scheduled now: its prologue overlaps this kernel and it waits for this grid's end
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   const int n_words32 = 8;
   RoutePtrs& r = ws.r;
   const int S = T * k;
@@ -375,15 +377,27 @@ k_select(const float* __restrict__ logits, StepPtrs st, Workspace ws, RoutePtrs 
 }
 
 cudaError_t configure_select(Dims max_dims) {
-  return cudaFuncSetAttribute(k_select, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                              (int)select_smem_bytes(max_dims));
+  cudaError_t e = cudaFuncSetAttribute(k_select, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       (int)select_smem_bytes(max_dims));
+  // same carve-out as the expert kernel that follows: no reconfiguration of the SM in between
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(k_select, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+  return e;
 }
 
 cudaError_t launch_select(const float* logits, StepPtrs st, Workspace ws, RoutePtrs ex, Dims d, Policy p,
                           int item_tile, cudaStream_t s) {
-  const size_t smem = select_smem_bytes(d);
-  k_select<<<1, kSelThreads, smem, s>>>(logits, st, ws, ex, d, p, item_tile, 0);
-  return cudaGetLastError();
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(1);
+  cfg.blockDim = dim3(kSelThreads);
+  cfg.dynamicSmemBytes = select_smem_bytes(d);
+  cfg.stream = s;
+  cudaLaunchAttribute attr;
+  attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;   // staging the step state overlaps the router kernel
+  attr.val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = &attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, k_select, logits, st, ws, ex, d, p, item_tile, 1);
 }
 
 }  // namespace team
