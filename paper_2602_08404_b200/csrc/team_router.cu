@@ -7,6 +7,8 @@
 //                    The same launch zeroes the output rows the expert kernel will accumulate into.
 //  k_router_topk   : one warp per row: softmax over all experts, plain top-k by warp shuffles,
 //                    renormalised weights, decision margin (team_route's outputs).
+#include <mutex>
+
 #include "team_common.cuh"
 #include "team_topk.cuh"
 
@@ -227,9 +229,19 @@ static cudaError_t prepare_kernel(K kernel, int smem) {
   return e;
 }
 
+// The opt-in is a per-device property of the kernel, shared by every context (and by the context-free
+// entry point): it is only ever raised, so that preparing for a small hidden size cannot take away
+// what a larger one needs.
 cudaError_t configure_router(int dtype, int hidden) {
+  static std::mutex mu;
+  static int prepared[64][2] = {};   // [device][dtype]: shared-memory bytes opted in so far
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
   const int smem = kRowTile * hidden * (int)sizeof(float) + 1024;
-  cudaError_t e;
+  const int di = dtype == TEAM_DTYPE_F32 ? 0 : 1;
+  std::lock_guard<std::mutex> lock(mu);
+  if (dev >= 0 && dev < 64 && prepared[dev][di] >= smem) return cudaSuccess;
   if (dtype == TEAM_DTYPE_F32) {
     e = prepare_kernel(k_router_logits<float>, smem);
     if (e == cudaSuccess) e = prepare_kernel(k_router_logits_small<float>, smem);
@@ -239,6 +251,7 @@ cudaError_t configure_router(int dtype, int hidden) {
   }
   if (e == cudaSuccess)
     e = cudaFuncSetAttribute(k_router_topk, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+  if (e == cudaSuccess && dev >= 0 && dev < 64) prepared[dev][di] = smem;
   return e;
 }
 

@@ -6,6 +6,8 @@
 //
 // Layout contract: rows with equal (group, branch) are contiguous (one decoding block, at most
 // TEAM_MAX_BLOCK rows), so the "distance to a decoded token" test of Eq. 4 only walks a row's own run.
+#include <mutex>
+
 #include "team_common.cuh"
 #include "team_topk.cuh"
 
@@ -376,12 +378,21 @@ k_select(const float* __restrict__ logits, StepPtrs st, Workspace ws, RoutePtrs 
   }
 }
 
+// The opt-in is per device and shared by all contexts: it is only ever raised.
 cudaError_t configure_select(Dims max_dims) {
-  cudaError_t e = cudaFuncSetAttribute(k_select, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       (int)select_smem_bytes(max_dims));
+  static std::mutex mu;
+  static int prepared[64] = {};
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  const int smem = (int)select_smem_bytes(max_dims);
+  std::lock_guard<std::mutex> lock(mu);
+  if (dev >= 0 && dev < 64 && prepared[dev] >= smem && prepared[dev] > 0) return cudaSuccess;
+  e = cudaFuncSetAttribute(k_select, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
   // same carve-out as the expert kernel that follows: no reconfiguration of the SM in between
   if (e == cudaSuccess)
     e = cudaFuncSetAttribute(k_select, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+  if (e == cudaSuccess && dev >= 0 && dev < 64) prepared[dev] = smem;
   return e;
 }
 
