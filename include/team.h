@@ -64,7 +64,8 @@ enum {
   TEAM_ERR_SHAPE = -2,   /* configuration the kernels do not support                   */
   TEAM_ERR_CUDA = -3,    /* CUDA runtime / driver error (see team_last_cuda_error)     */
   TEAM_ERR_TIMEOUT = -4, /* device status: a bounded wait expired                      */
-  TEAM_ERR_STATE = -5    /* device status: row layout contract broken / index range    */
+  TEAM_ERR_STATE = -5,   /* device status: row layout contract broken / index range    */
+  TEAM_ERR_CAPACITY = -6 /* more rows than a fixed-size scratch area holds               */
 };
 
 enum { TEAM_TOK_MASKED = 0, TEAM_TOK_NEW = 1, TEAM_TOK_CACHED = 2 };   /* team_step_state.tok_state */
@@ -78,6 +79,7 @@ enum { TEAM_DTYPE_F32 = 0, TEAM_DTYPE_BF16 = 1 };
 #define TEAM_MAX_ROWS 2048     /* rows per call                        */
 #define TEAM_MAX_GROUPS 1024
 #define TEAM_MAX_BLOCK 64      /* rows of one (group, branch)          */
+#define TEAM_STATIC_ROUTE_MAX_ROWS 256   /* rows per team_route_static call */
 
 typedef struct {
   int32_t hidden;      /* H; multiple of 128 for bf16, of 4 for fp32                     */
@@ -156,6 +158,36 @@ int team_set_policy(team_ctx *ctx, const team_config *cfg);
  * renormalised weights and the decision margin.  x: [T, H] row-major, dtype per
  * config.  Logits stay in the context for team_select_experts. */
 int team_route(team_ctx *ctx, const void *x, const team_step_state *st, team_routing *out, void *stream);
+
+/* The router step without any allocation.  (The paper has no counterpart; this is a deployment
+ * variant of team_route.)
+ *
+ * Who needs it: code that runs where device allocation is off limits -- a serving loop whose device
+ * memory is planned up front and frozen, a plug-in called from inside another framework's stream
+ * callback or capture region, a latency-critical path that must not hit the allocator's implicit
+ * device synchronisation, or a process whose memory pool is owned by someone else.  Such callers
+ * cannot create a team_ctx, because team_create allocates the workspace that holds the logits.
+ *
+ * What it does: the same two router kernels as team_route (fp32 logits, softmax, plain top-k with
+ * renormalised weights, decision margin; cached rows skipped when TEAM_F_DCD is set), with the logits
+ * kept in a fixed scratch array that is part of the library image: TEAM_STATIC_ROUTE_MAX_ROWS x
+ * TEAM_MAX_EXPERTS floats = 256 KiB on every GPU that loads the library, held until the process
+ * exits.  No context is involved: shapes, dtype and policy come from `cfg` (hidden, n_experts, top_k,
+ * dtype, flags, norm_topk are read; the rest is ignored), x [T, H] and w_router [E, H] fp32 are
+ * caller-owned device memory, `st->tok_state` must be set, and `out` receives probs / topk_idx /
+ * topk_w / margin exactly as team_route writes them (NULL members are skipped).
+ *
+ * Limits and caveats:
+ *   - st->n_rows > TEAM_STATIC_ROUTE_MAX_ROWS returns TEAM_ERR_CAPACITY and launches nothing.
+ *   - The call never calls cudaMalloc / cudaFree or any allocating routine.  The first call on a
+ *     device looks up the scratch array's device address and opts the kernels in to their shared
+ *     memory; make that first call outside any stream capture.
+ *   - All calls on a device share the one scratch array, which keeps the previous call's contents
+ *     (nothing in it needs clearing: every row that is read is rewritten first).  Two calls whose
+ *     kernels overlap on the GPU (different streams) race on it; keep them stream-ordered.
+ * Errors: TEAM_ERR_ARG, TEAM_ERR_SHAPE, TEAM_ERR_CAPACITY, TEAM_ERR_CUDA. */
+int team_route_static(const team_config *cfg, const void *x, const void *w_router, const team_step_state *st,
+                      team_routing *out, void *stream);
 
 /* TEAM selection (Eq. 4, Algorithm 1 steps 1-3) and dispatch tables, from the
  * logits left by the preceding team_route on the same context, stream and rows. */

@@ -15,13 +15,15 @@ _PKG = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_PKG, "libteam_b200.so")
 
 TEAM_OK, TEAM_ERR_ARG, TEAM_ERR_SHAPE, TEAM_ERR_CUDA, TEAM_ERR_TIMEOUT, TEAM_ERR_STATE = 0, -1, -2, -3, -4, -5
+TEAM_ERR_CAPACITY = -6
+TEAM_STATIC_ROUTE_MAX_ROWS = 256
 TEAM_TOK_MASKED, TEAM_TOK_NEW, TEAM_TOK_CACHED = 0, 1, 2
 TEAM_CLS_SKIP, TEAM_CLS_FIRST, TEAM_CLS_COLD = 0, 1, 2
 TEAM_F_DCD, TEAM_F_LAC = 1, 2
 TEAM_DTYPE_F32, TEAM_DTYPE_BF16 = 0, 1
 
 EXPORTS = ["team_create", "team_destroy", "team_set_weights", "team_set_policy", "team_route",
-           "team_select_experts", "team_moe_forward", "team_residual_add", "team_read_status",
+           "team_route_static", "team_select_experts", "team_moe_forward", "team_residual_add", "team_read_status",
            "team_last_launch_count", "team_expert_timing", "team_debug_force_simt", "team_strerror",
            "team_last_cuda_error", "team_version"]
 
@@ -66,6 +68,8 @@ def lib():
         L.team_set_weights.argtypes = [vp, ctypes.POINTER(team_weights)]
         L.team_set_policy.argtypes = [vp, ctypes.POINTER(team_config)]
         L.team_route.argtypes = [vp, vp, ctypes.POINTER(team_step_state), ctypes.POINTER(team_routing), vp]
+        L.team_route_static.argtypes = [ctypes.POINTER(team_config), vp, vp, ctypes.POINTER(team_step_state),
+                                        ctypes.POINTER(team_routing), vp]
         L.team_select_experts.argtypes = [vp, ctypes.POINTER(team_step_state), ctypes.POINTER(team_routing), vp]
         L.team_moe_forward.argtypes = [vp, vp, ctypes.POINTER(team_step_state), ctypes.POINTER(team_routing), vp, vp]
         L.team_residual_add.argtypes = [vp, vp, vp, i32, vp]
@@ -150,6 +154,14 @@ def _routing(out):
 def team_route(ctx, x, st, out):
     r = _routing(out)
     _check(lib().team_route(ctx, _ptr(x), ctypes.byref(_state(st)), ctypes.byref(r), _stream()), ctx)
+
+
+def team_route_static(cfg, x, w_router, st, out):
+    """Router step with no context and no allocation (fixed scratch inside the library); returns the status code
+    instead of raising so that callers can test the capacity limit."""
+    r = _routing(out)
+    return lib().team_route_static(ctypes.byref(cfg), _ptr(x), _ptr(w_router), ctypes.byref(_state(st)), ctypes.byref(r),
+                                   _stream())
 
 
 def team_select_experts(ctx, st, out):

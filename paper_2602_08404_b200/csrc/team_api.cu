@@ -112,6 +112,7 @@ const char* team_strerror(int code) {
     case TEAM_ERR_CUDA: return "CUDA error";
     case TEAM_ERR_TIMEOUT: return "device wait expired";
     case TEAM_ERR_STATE: return "row layout contract broken or index out of range";
+    case TEAM_ERR_CAPACITY: return "more rows than the fixed-size scratch area holds";
     default: return "unknown error";
   }
 }
