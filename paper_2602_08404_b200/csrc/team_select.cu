@@ -93,6 +93,12 @@ k_select(const float* __restrict__ logits, StepPtrs st, Workspace ws, RoutePtrs 
   for (int i = tid; i < nw * EN; i += kSelThreads) s.hist[i] = 0;
   // per-window publication counters of the expert kernel start every step from zero
   for (int i = tid; i < ws.n_flags; i += kSelThreads) ws.win_flags[i] = 0;
+  float conf_r[TEAM_MAX_ROWS / kSelThreads];     // confidences of the rows this thread classifies, fetched with the rest
+#pragma unroll
+  for (int i = 0; i < TEAM_MAX_ROWS / kSelThreads; ++i) {
+    const int t = tid + i * kSelThreads;
+    conf_r[i] = t < T ? st.conf[t] : 0.f;
+  }
   for (int t = tid; t < T; t += kSelThreads) {
     int g = st.group[t], b = st.branch[t];
     if (g < 0 || g >= d.G || b < 0 || b > 255) {
@@ -124,7 +130,7 @@ k_select(const float* __restrict__ logits, StepPtrs st, Workspace ws, RoutePtrs 
     } else {
       const int key = s.key[t], mypos = s.pos[t];
       const int lim = p.inclusive ? p.L_hot : p.L_hot - 1;   // |pos - j| <= lim
-      bool hot = st.conf[t] > p.tau_hot;
+      bool hot = conf_r[t / kSelThreads] > p.tau_hot;
       if (p.prefix_decoded && mypos + 1 <= lim) hot = true;
       for (int u = t - 1; !hot && u >= 0 && s.key[u] == key; --u) {
         if (t - u > TEAM_MAX_BLOCK) { set_status(ws.status, TEAM_ERR_STATE, 2); break; }

@@ -18,48 +18,57 @@ struct TopkResult {
   float top;      // all lanes: largest candidate logit
 };
 
+// Order-preserving map from a float to an unsigned key (larger float <-> larger key; -inf maps below
+// every finite value), so that the warp-wide maximum is one redux instruction.
+__device__ __forceinline__ uint32_t float_key(float f) {
+  const uint32_t u = __float_as_uint(f + 0.0f);   // -0 and +0 compare equal: both take +0's key
+  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+__device__ __forceinline__ float key_float(uint32_t k) {
+  return __uint_as_float((k & 0x80000000u) ? (k & 0x7fffffffu) : ~k);
+}
+
 // v[i] is the logit of expert i*32+lane, or -inf if that expert is not a candidate
-// (beyond E, or outside the allowed set).  v is consumed.
+// (beyond E, or outside the allowed set).  v is consumed.  Each of the k+1 rounds takes the
+// warp-wide maximum key and then the lowest expert id among the lanes that hold it.
 __device__ __forceinline__ TopkResult warp_topk(float (&v)[kMaxPerLane], int k, int lane) {
   TopkResult r;
   r.idx = -1;
   r.val = kNegInf;
   r.top = kNegInf;
+  r.margin = __builtin_huge_valf();
   float last = kNegInf;
+  const uint32_t key_neg_inf = float_key(kNegInf);
   for (int j = 0; j <= k; ++j) {
-    float bv = kNegInf;
+    uint32_t bk = key_neg_inf;
     int bi = 0x7fffffff;
 #pragma unroll
     for (int i = 0; i < kMaxPerLane; ++i) {
       // ascending expert id within the lane, strict '>' keeps the lower id on ties
-      if (v[i] > bv) {
-        bv = v[i];
+      const uint32_t ki = float_key(v[i]);
+      if (ki > bk) {
+        bk = ki;
         bi = i * 32 + lane;
       }
     }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-      float ov = __shfl_xor_sync(0xffffffffu, bv, o);
-      int oi = __shfl_xor_sync(0xffffffffu, bi, o);
-      if (ov > bv || (ov == bv && oi < bi)) {
-        bv = ov;
-        bi = oi;
-      }
-    }
+    const uint32_t wk = __reduce_max_sync(0xffffffffu, bk);
+    const int wi = (int)__reduce_min_sync(0xffffffffu, (bk == wk && wk != key_neg_inf) ? (uint32_t)bi : 0x7fffffffu);
+    const bool none = wk == key_neg_inf;
+    const float bv = none ? kNegInf : key_float(wk);
     if (j == 0) r.top = bv;
     if (j < k) {
       if (lane == j) {
-        r.idx = (bv == kNegInf) ? -1 : bi;
+        r.idx = none ? -1 : wi;
         r.val = bv;
       }
       last = bv;
-      if (bv != kNegInf && (bi & 31) == lane) {
+      if (!none && (wi & 31) == lane) {
 #pragma unroll
         for (int i = 0; i < kMaxPerLane; ++i)
-          if (i == (bi >> 5)) v[i] = kNegInf;
+          if (i == (wi >> 5)) v[i] = kNegInf;
       }
     } else {
-      r.margin = (bv == kNegInf) ? __builtin_huge_valf() : last - bv;
+      r.margin = none ? __builtin_huge_valf() : last - bv;
     }
   }
   return r;
