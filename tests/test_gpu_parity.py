@@ -67,3 +67,66 @@ def test_c4_batch_sweep(seqs, weights_cache):
     P.run_schedule(shape, weights_cache(shape), steps, 3)
     if seqs <= 4:
         P.run_schedule(shape, weights_cache(shape), steps, 0)
+
+
+def _run_stack(shape, n_layers, flags, weights_cache):
+    """MoE-only stack (config 5's structure): x <- x + layer(x) on computed rows, layer after layer, step after step.
+
+    Every layer is checked teacher-forced (the oracle gets the activations the GPU stack actually fed into that
+    layer, which are exact in the storage type), so a near-tie early in the stack cannot cascade; the stack's final
+    activations are compared with the oracle's own stack as well.
+    """
+    import dataclasses
+    layers_w = [W.make_weights(dataclasses.replace(shape, seed=shape.seed + 100 * l)) for l in range(n_layers)]
+    steps = W.make_schedule(shape)
+    ocfg = P.oracle_config(shape, flags)
+    layers = [P.Layer(shape, w, flags) for w in layers_w]
+    dc = P.dtype_code(shape)
+    T = steps[0]["x"].shape[0]
+    round_fn = (lambda a: W.round_to_bf16(np.asarray(a, dtype=np.float32)).astype(np.float64)) if shape.dtype == "bf16" \
+        else (lambda a: np.asarray(a, dtype=np.float32).astype(np.float64))
+    try:
+        for si, step in enumerate(steps):
+            x_dev = B.to_device(step["x"], dc)
+            st = B.state_to_device(step)
+            y_dev = torch.zeros((T, shape.hidden), dtype=torch.float32, device="cuda")
+            all_exact = True
+            for li, layer in enumerate(layers):
+                x_in = x_dev.float().cpu().numpy()
+                out = B.alloc_routing(layer.cfg, T)
+                y_before = y_dev.cpu().numpy()
+                B.team_moe_forward(layer.ctx, x_dev, st, out, y_dev)
+                B.team_residual_add(layer.ctx, x_dev, y_dev, T)
+                code, detail = B.team_read_status(layer.ctx)
+                assert code == B.TEAM_OK, (code, detail)
+                got = B.routing_to_host(out)
+                y_ref, ref = O.moe_forward(ocfg, layers_w[li], x_in, step["tok_state"], step["conf"], step["pos"],
+                                           step["group"], step["branch"], y_prev=y_before)
+                what = f"{shape.name} stack step={si} layer={li}"
+                exact = P.compare_routing(ocfg, ref, got, step["group"], what)
+                all_exact = all_exact and exact
+                if exact:
+                    P.compare_y(shape, y_ref, y_dev.cpu().numpy(), ref["tok_class"], y_before, what)
+                    # the residual add: fp32 add, stored in the activation type
+                    comp = ref["tok_class"] != O.CLS_SKIP
+                    want = x_in.astype(np.float64).copy()
+                    want[comp] = round_fn(x_in[comp].astype(np.float32) + y_dev.cpu().numpy()[comp])
+                    np.testing.assert_array_equal(x_dev.float().cpu().numpy().astype(np.float64), want, err_msg=what)
+            if all_exact:
+                x_ref, _ = O.stack_forward(ocfg, layers_w, step["x"], step["tok_state"], step["conf"], step["pos"],
+                                           step["group"], step["branch"], round_fn=round_fn)
+                x_got = x_dev.float().cpu().numpy()
+                tol = (P.TOL_BF16 if shape.dtype == "bf16" else P.TOL_F32) * np.abs(x_ref).max()
+                assert np.abs(x_got - x_ref).max() <= tol * n_layers, f"{shape.name} stack step={si} end to end"
+    finally:
+        for layer in layers:
+            layer.close()
+
+
+@pytest.mark.parametrize("flags", [0, 3])
+def test_c5_stack_small_shape(flags, weights_cache):
+    _run_stack(W.MINI_WRAP, 8, flags, weights_cache)
+
+
+def test_c5_stack_sdar_shape_two_layers(weights_cache):
+    _run_stack(W.C2, 2, 3, weights_cache)
