@@ -24,6 +24,7 @@ struct team_ctx {
   int item_tile;
   int last_launches;
   int force_simt;
+  bool stream_path;   // few rows: the weight-streaming expert kernel instead of the tensor-memory one
   void* simt_act;   // diagnostic fp32-FMA path on bf16 weights: activation scratch
   char cuda_err[256];
   // expert-kernel timing
@@ -148,7 +149,9 @@ int team_create(const team_config* cfg, team_ctx** out) {
   ctx->item_tile = pick_item_tile(*cfg);
   e = team::configure_router(cfg->dtype, cfg->hidden);
   if (e == cudaSuccess) e = team::configure_select(dims_of(*cfg, cfg->max_rows));
+  ctx->stream_path = cfg->dtype == TEAM_DTYPE_BF16 && team::experts_stream_supported(cfg->max_rows, cfg->hidden, cfg->inter);
   if (e == cudaSuccess && cfg->dtype == TEAM_DTYPE_BF16) e = team::configure_experts_tc(ctx->item_tile);
+  if (e == cudaSuccess && ctx->stream_path) e = team::configure_experts_stream(cfg->hidden);
   if (e != cudaSuccess) {
     delete ctx;
     return TEAM_ERR_CUDA;
@@ -314,7 +317,10 @@ int team_moe_forward(team_ctx* ctx, const void* x, const team_step_state* st, te
     cudaEventRecord(ev0, s);
   }
   if (tc) {
-    e = team::launch_experts_tc(ctx->item_tile, x, ctx->w.w_gate, ctx->w.w_up, ctx->w.w_down, ctx->ws, y, d, ctx->n_sms, s);
+    if (ctx->stream_path)
+      e = team::launch_experts_stream(x, ctx->w.w_gate, ctx->w.w_up, ctx->w.w_down, ctx->ws, y, d, ctx->n_sms, s);
+    else
+      e = team::launch_experts_tc(ctx->item_tile, x, ctx->w.w_gate, ctx->w.w_up, ctx->w.w_down, ctx->ws, y, d, ctx->n_sms, s);
     if (e != cudaSuccess) return fail_cuda(ctx, e, "expert kernel");
     ++ctx->last_launches;
   } else {

@@ -72,6 +72,11 @@ MINI_WRAP = Shape("mini_wrap_bf16", 768, 64, 4, 192, 0, "bf16", 16, 4, 3, 1, 2, 
                   seqs=2, branches=2, seed=13)
 
 
+# Few rows, many activated experts with a wide intermediate dimension and a shared expert: in vanilla
+# mode every CTA of a 148-SM grid gets more column groups than one pass of the few-rows expert kernel
+# holds, so its range spans several passes and windows are shared between neighbouring CTAs.
+STREAM_MULTI = Shape("stream_multi_bf16", 1024, 48, 8, 1024, 1, "bf16", 8, 4, 2, 1, 2, 0.7, seed=14)
+
 def round_to_bf16(a):
     """Round fp32 values to the nearest bf16-representable value (ties to even); returns fp32."""
     a = np.ascontiguousarray(a, dtype=np.float32)

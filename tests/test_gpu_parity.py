@@ -52,6 +52,16 @@ def test_c2_sdar_shape(flags, weights_cache):
         assert [s["rows"] for s in stats] == [4, 4, 3, 2]
 
 
+@pytest.mark.parametrize("flags", [0, 1, 3])
+def test_few_rows_kernel_multi_pass_ranges_and_shared_expert(flags, weights_cache):
+    shape = W.STREAM_MULTI
+    stats = P.run_schedule(shape, weights_cache(shape), W.make_schedule(shape), flags)
+    assert len(stats) == 4
+    if flags == 0:
+        # enough activated experts that a CTA's range of column groups exceeds one pass (8 groups)
+        assert max(s["n_active"] for s in stats) * (shape.inter // 16) > 8 * 148
+
+
 @pytest.mark.parametrize("flags", [0, 3])
 def test_c3_llada_shape_with_shared_expert(flags, weights_cache):
     stats = P.run_schedule(W.C3, weights_cache(W.C3), W.make_schedule(W.C3), flags)
