@@ -190,19 +190,20 @@ def main():
 
     # R independent layers, generated on the device (seeded); layer 0 also goes to the host for the oracle leg
     gen = torch.Generator(device=dev)
-    layers = []
+    layers, packed = [], []
     for r in range(R):
         gen.manual_seed(1000 + r)
         wr = (torch.randn((E, H), generator=gen, device=dev, dtype=torch.float32) * 0.02).contiguous()
         wg, wu, wd = [(torch.randn(s, generator=gen, device=dev, dtype=torch.float32) * 0.02).to(torch.bfloat16)
                       for s in ((E, I, H), (E, I, H), (E, H, I))]
-        layers.append((wr, wg, wu, wd))
+        layers.append((wr, wg, wu, wd if r == 0 else None))
+        packed.append(B.team_pack_w_down(wd))      # the layout the library reads; row-major kept for the oracle leg
     cfg = B.make_config(H, E, k, I, 0, max_rows=T, max_groups=1, dtype=B.TEAM_DTYPE_BF16, flags=args.flags,
                         tau_hot=shape.tau_hot, L_hot=shape.L_hot)
     ctxs = []
     for r in range(R):
         c = B.team_create(cfg)
-        B.team_set_weights(c, *layers[r])
+        B.team_set_weights(c, *layers[r][:3], packed[r])
         ctxs.append(c)
 
     x_dev = [B.to_device(s["x"], B.TEAM_DTYPE_BF16, dev) for s in steps_host]

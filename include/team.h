@@ -104,7 +104,8 @@ typedef struct {
   const void *w_router; /* fp32 [E, H] row-major                                          */
   const void *w_gate;   /* [E + n_shared, I, H] row-major, dtype per config               */
   const void *w_up;     /* [E + n_shared, I, H]                                           */
-  const void *w_down;   /* [E + n_shared, H, I]                                           */
+  const void *w_down;   /* [E + n_shared, I/16, H, 16]: Eq. 1's W_down [H, I] of every expert
+                           stored in slabs of 16 columns, as team_pack_w_down() writes it */
 } team_weights;
 
 /* State carried from the previous denoising step (Algorithm 1 inputs D, M; Eq. 4). */
@@ -148,6 +149,19 @@ int team_destroy(team_ctx *ctx);
  * takes effect for calls issued afterwards (pointers are passed by value at
  * launch). */
 int team_set_weights(team_ctx *ctx, const team_weights *w);
+
+/* Convert down-projection weights from row-major [n_experts_total, H, I] (src)
+ * to the slab layout [n_experts_total, I/16, H, 16] (dst) that team_weights.w_down
+ * expects: element (e, h, c) moves to (((e * I/16 + c/16) * H + h) * 16 + c%16).
+ * The expert kernels give each group of 16 intermediate columns to one CTA
+ * (Eq. 1's down projection, summed over groups); in this layout the 16 columns
+ * of all H rows are one contiguous block.  Done once per layer when weights are
+ * loaded; needs no context.  src and dst are device pointers, 16-byte aligned,
+ * of the same size, not overlapping; both stay owned by the caller.  inter must
+ * be a multiple of 16.  Asynchronous on `stream`.
+ * Errors: TEAM_ERR_ARG, TEAM_ERR_SHAPE, TEAM_ERR_CUDA. */
+int team_pack_w_down(const void *src, void *dst, int n_experts_total, int hidden,
+                     int inter, int dtype, void *stream);
 
 /* Change flags / tau_hot / L_hot / hot_dist_inclusive / prefix_decoded /
  * norm_topk of an existing context (shapes and dtype must be unchanged). */

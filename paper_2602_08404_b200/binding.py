@@ -23,7 +23,7 @@ TEAM_F_DCD, TEAM_F_LAC = 1, 2
 TEAM_DTYPE_F32, TEAM_DTYPE_BF16 = 0, 1
 
 EXPORTS = ["team_create", "team_destroy", "team_set_weights", "team_set_policy", "team_route",
-           "team_route_static", "team_select_experts", "team_moe_forward", "team_residual_add", "team_read_status",
+           "team_route_static", "team_pack_w_down", "team_select_experts", "team_moe_forward", "team_residual_add", "team_read_status",
            "team_last_launch_count", "team_expert_timing", "team_debug_force_simt", "team_strerror",
            "team_last_cuda_error", "team_version"]
 
@@ -68,6 +68,7 @@ def lib():
         L.team_set_weights.argtypes = [vp, ctypes.POINTER(team_weights)]
         L.team_set_policy.argtypes = [vp, ctypes.POINTER(team_config)]
         L.team_route.argtypes = [vp, vp, ctypes.POINTER(team_step_state), ctypes.POINTER(team_routing), vp]
+        L.team_pack_w_down.argtypes = [vp, vp, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int, vp]
         L.team_route_static.argtypes = [ctypes.POINTER(team_config), vp, vp, ctypes.POINTER(team_step_state),
                                         ctypes.POINTER(team_routing), vp]
         L.team_select_experts.argtypes = [vp, ctypes.POINTER(team_step_state), ctypes.POINTER(team_routing), vp]
@@ -134,6 +135,16 @@ def team_destroy(ctx):
 def team_set_weights(ctx, w_router, w_gate, w_up, w_down):
     w = team_weights(_ptr(w_router), _ptr(w_gate), _ptr(w_up), _ptr(w_down))
     _check(lib().team_set_weights(ctx, ctypes.byref(w)), ctx)
+
+
+def team_pack_w_down(w_down):
+    """Row-major [n_experts_total, H, I] device tensor -> new tensor in the slab layout team_set_weights expects."""
+    n, H, I = w_down.shape
+    dtype = TEAM_DTYPE_BF16 if w_down.dtype == torch.bfloat16 else TEAM_DTYPE_F32
+    src = w_down.contiguous()
+    dst = torch.empty_like(src)
+    _check(lib().team_pack_w_down(_ptr(src), _ptr(dst), n, H, I, dtype, _stream()))
+    return dst
 
 
 def team_set_policy(ctx, cfg):

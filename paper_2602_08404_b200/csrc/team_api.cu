@@ -61,7 +61,7 @@ int check_config(const team_config* c) {
   if (c->max_rows <= 0 || c->max_rows > TEAM_MAX_ROWS) return TEAM_ERR_SHAPE;
   if (c->max_groups <= 0 || c->max_groups > TEAM_MAX_GROUPS) return TEAM_ERR_SHAPE;
   if (c->dtype == TEAM_DTYPE_F32) {
-    if (c->hidden % 4 || c->inter % 4) return TEAM_ERR_SHAPE;
+    if (c->hidden % 4 || c->inter % 16) return TEAM_ERR_SHAPE;
   } else if (c->dtype == TEAM_DTYPE_BF16) {
     if (c->hidden % 128 || c->inter % 64) return TEAM_ERR_SHAPE;
   } else {

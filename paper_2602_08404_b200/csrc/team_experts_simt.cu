@@ -104,10 +104,11 @@ k_down(const WT* __restrict__ w_down, const float* __restrict__ act, const int32
       w = 1.f;
     }
     if (e < 0) continue;
-    const WT* wr = w_down + ((size_t)e * d.H + h) * d.I;
+    // W_down is stored in slabs of 16 columns: element (e, h, c) sits at (((e * I/16 + c/16) * H + h) * 16 + c%16)
+    const WT* wr = w_down + ((size_t)e * (d.I / 16) * d.H + h) * 16;
     const float* ar = act + (size_t)slot * d.I;
     float acc = 0.f;
-    for (int c = lane; c < d.I; c += 32) acc = fmaf(to_f32(wr[c]), ar[c], acc);
+    for (int c = lane; c < d.I; c += 32) acc = fmaf(to_f32(wr[(size_t)(c >> 4) * d.H * 16 + (c & 15)]), ar[c], acc);
     out = fmaf(w, warp_sum(acc), out);
   }
   if (lane == 0) y[(size_t)t * d.H + h] = out;

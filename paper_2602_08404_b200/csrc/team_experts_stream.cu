@@ -1,31 +1,29 @@
 // Expert kernel for the few-rows regime (T <= 8 rows, bf16 weights): a weight-streaming kernel.
 //
-// With a handful of rows the SwiGLU experts are a matrix-vector problem: ~1 MB of weights per SM and
-// a few hundred kFLOP.  Staging tiles for the tensor-memory path costs more in hand-offs between
+// With a handful of rows the SwiGLU experts (Eq. 1) are a matrix-vector problem: ~1 MB of weights per
+// SM and a few hundred kFLOP.  Staging tiles for the tensor-memory path costs more in hand-offs between
 // warps than the math is worth, so here every warp is its own pipeline: it copies 2 KB chunks of
-// weights (16 rows x 128 bytes) from HBM into a private ring in shared memory with asynchronous
-// copies, several chunks ahead, and multiplies each chunk with the token rows using warp-level mma
-// (m16n8k16: 16 weight rows x 8 tokens).  No warp ever waits for another one inside a phase; one
-// block-wide barrier per pass separates the gate/up phase from the down phase.
+// weights from HBM into a private ring in shared memory with asynchronous copies, several chunks
+// ahead, and multiplies each chunk with the token rows using warp-level mma (m16n8k16: 16 weight rows
+// x 8 tokens).  No warp waits for another one inside a phase, and no CTA ever waits for another CTA.
 //
-// The work partition is the expert kernel's: the intermediate dimension of every activated expert is
-// cut into groups of 16 columns; a group costs 16 gate rows + 16 up rows of W (phase 1) and a quarter
-// of the W_down tiles of its 64-column window (phase 2); the global list of groups is cut into one
-// contiguous range per CTA.  Windows cut by a range boundary are shared by neighbouring CTAs through
-// the activation scratch in global memory and one counter per window (cooperative launch, bounded
-// waits; a CTA's head window comes last when its range spans several passes, so waits cannot form a
-// cycle).
+// Work partition: the intermediate dimension of every activated expert is cut into groups of 16
+// columns, the global list of groups into one contiguous range per CTA.  A group is self-contained:
+// its 16 gate rows and 16 up rows of W give 16 activations per token (phase 1), and those multiply
+// the group's slab of W_down, 16 columns of all H rows, stored contiguously ([I/16][H][16]), into a
+// partial y that is added to the output with fp32 reductions (phase 2).  Groups are handled in passes
+// of up to 8:
 //
 //   phase 1   warp = (gate | up tile of 16 rows) x (one of 8 slices of the hidden dimension), for every
-//             group of the pass in turn; partial sums of a slice go to shared memory.
-//   barrier   sum the 8 slices, a = silu(gate) * up, round to bf16, publish to the scratch, count.
-//   phase 2   per window and owned tile range: warps take 16-row units of W_down (128 bytes per row),
-//             read the window's activations from the scratch (L2), scale by the routing weight and
-//             add into y with fp32 reductions.  Fully owned windows go first, shared ones after, so
-//             that the neighbours' activations have arrived by the time they are needed.
+//             group of the pass in turn; chunk = 16 rows x 128 bytes; partial sums of a slice go to
+//             shared memory.
+//   barrier   sum the 8 slices, a = silu(gate) * up, round to bf16, keep in shared memory.
+//   phase 2   warp = H/16 consecutive output rows, for every group of the pass in turn; chunk = 64
+//             slab rows x 32 bytes; the accumulators stay in registers across the groups of one
+//             expert and are scaled by the routing weights and added to y when the expert changes.
 //
-// A warp's copies run ahead across the barrier: while the slices are being summed, the first W_down
-// units of phase 2 are already on their way.
+// A warp's copies run ahead across the barrier: while the slices are being summed, its first slab
+// chunks of phase 2 are already on their way.
 #include "team_common.cuh"
 
 namespace team {
@@ -34,25 +32,21 @@ constexpr int kStThreads = 512;
 constexpr int kStWarps = 16;
 constexpr int kStSlices = 8;                    // slices of the hidden dimension in phase 1
 constexpr int kStRows = 8;                      // token rows (n of the mma)
-constexpr int kStScWindows = 2;                 // windows per pass
-constexpr int kStScGroups = kStScWindows * 4;   // groups whose partial sums fit in shared memory
-constexpr int kStChunkBytes = 2048;             // 16 rows x 128 bytes
-constexpr int kStRedBytes = kStScGroups * kStSlices * 2 * 16 * kStRows * 4;
-constexpr unsigned long long kStWaitCycles = 2000000000ull;   // ~1 s
+constexpr int kStPassGroups = 8;                // groups whose partial sums fit in shared memory
+constexpr int kStSlots = 4;                     // chunks per warp ring
+constexpr int kStChunkBytes = 2048;
+constexpr int kStRedBytes = kStPassGroups * kStSlices * 2 * 16 * kStRows * 4;
 
 struct StArgs {
   const __nv_bfloat16* x;       // [T, H]
   const __nv_bfloat16* w_gate;  // [E + ns, I, H]
   const __nv_bfloat16* w_up;
-  const __nv_bfloat16* w_down;  // [E + ns, H, I]
+  const __nv_bfloat16* w_down;  // [E + ns, I/16, H, 16]
   const int32_t* perm;
   const float* topk_w;
   const WorkItem* items;
   const int32_t* n_items;
-  __nv_bfloat16* act_g;         // [items][16][I]
-  int32_t* win_flags;           // [items * I/64]
   float* y;                     // [T, H]
-  int32_t* status;
   Dims d;
 };
 
@@ -78,16 +72,6 @@ __device__ __forceinline__ uint4 st_ldg_stream(const void* p) {
                : "l"(p));
   return v;
 }
-__device__ __forceinline__ uint32_t st_ldg_l2(const void* p) {      // data written by other CTAs during this launch
-  uint32_t v;
-  asm volatile("ld.global.cg.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
-  return v;
-}
-__device__ __forceinline__ int st_ld_acquire(const int32_t* p) {
-  int v;
-  asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
-  return v;
-}
 // d += A(16x16, rows g / g+8) * B(16x8), bf16 inputs, fp32 accumulate
 __device__ __forceinline__ void st_mma(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
   asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
@@ -96,33 +80,31 @@ __device__ __forceinline__ void st_mma(float (&d)[4], const uint32_t (&a)[4], ui
 }
 
 // shared memory: token rows | partial sums [group][slice][gate, up][16 rows][8 tokens] | per-warp rings
-__host__ __device__ inline int stream_ring_slots(int H) { return H <= 2048 ? 4 : 3; }
 __host__ __device__ inline size_t stream_smem_bytes(int H) {
-  return (size_t)kStRows * H * 2 + kStRedBytes + (size_t)kStWarps * stream_ring_slots(H) * kStChunkBytes;
+  return (size_t)kStRows * H * 2 + kStRedBytes + (size_t)kStWarps * kStSlots * kStChunkBytes;
 }
 
-// Phase-2 job: the CTA's groups [a, b) of window W (global window index) own the W_down row tiles
-// [a*HT/4, b*HT/4) of that window; a 16-row unit of them is what one warp handles at a time.
-struct StJob {
-  int W, a, b;
-};
-
-template <int SLOTS>
+// CPG: 64-row chunks of a W_down slab per warp and group (H = CPG * 1024)
+template <int CPG>
 __global__ void __launch_bounds__(kStThreads, 1) k_experts_stream(StArgs a) {
   extern __shared__ __align__(128) unsigned char st_smem[];
-  __shared__ int s_item[kStScGroups], s_col[kStScGroups];
+  __shared__ __align__(16) __nv_bfloat16 s_act[kStPassGroups][kStRows][16];    // a = silu(gate) * up of the pass
+  __shared__ float s_w[kStPassGroups][kStRows];                                // routing weight of token n for group q's expert
+  __shared__ int s_item[kStPassGroups];
+  constexpr int SLOTS = kStSlots;
+  constexpr int H = CPG * 1024, HW = H / kStWarps;      // output rows per warp in phase 2
+  constexpr int KS = H / kStSlices, NCH = KS / 64;      // phase 1: elements per slice, 64-wide chunks per slice
   const Dims d = a.d;
-  const int H = d.H, I = d.I, T = d.T;
+  const int I = d.I, T = d.T;
   unsigned char* xs = st_smem;                                                    // [8][H] bf16, 16-byte pieces swizzled
   float* red = reinterpret_cast<float*>(st_smem + (size_t)kStRows * H * 2);      // [group][slice][2][16][8]
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int g = lane >> 2, c = lane & 3;        // fragment row (and token of the B fragment), k / token pair
-  const int NG = I / 16, WPI = NG / 4, HT = H / 128;
-  const int KS = H / kStSlices, NCH = KS / 64;  // elements per slice, 64-wide chunks per slice
+  const int NG = I / 16;
 
   // ---- token rows into shared memory (an input of the call: may overlap the selection kernel) ----
   {
-    const int per_row = H / 8;
+    constexpr int per_row = H / 8;
     for (int idx = tid; idx < kStRows * per_row; idx += kStThreads) {
       const int n = idx / per_row, ci = idx - n * per_row;
       uint4 v = make_uint4(0u, 0u, 0u, 0u);
@@ -135,114 +117,95 @@ __global__ void __launch_bounds__(kStThreads, 1) k_experts_stream(StArgs a) {
 
   const long long n_groups = (long long)(*a.n_items) * NG;
   const int g_lo = (int)(n_groups * blockIdx.x / gridDim.x), g_hi = (int)(n_groups * (blockIdx.x + 1) / gridDim.x);
-  const bool multi = g_hi > (((g_lo >> 2) + kStScWindows) << 2);   // more than one pass
-  bool ok = true;
 
   // ---- this warp's ring and its fixed lane roles ----
   const uint32_t ring = st_smem_u32(st_smem + (size_t)kStRows * H * 2 + kStRedBytes + (size_t)warp * SLOTS * kStChunkBytes);
-  const int cp_row = lane >> 3, cp_piece = lane & 7;                 // copies: rows cp_row + 4j, one 16-byte piece
+  // phase-1 chunk: 16 rows x 128 bytes; lane copies one 16-byte piece of rows cp_row + 4j; piece p of row r sits at p ^ (r & 7)
+  const int cp_row = lane >> 3, cp_piece = lane & 7;
   const uint32_t cp_off0 = cp_row * 128 + ((cp_piece ^ cp_row) << 4);          // rows cp_row, cp_row + 8 (+1024)
   const uint32_t cp_off1 = (cp_row + 4) * 128 + ((cp_piece ^ (cp_row + 4)) << 4);
-  const int a_row = (lane & 7) + ((lane >> 3) & 1) * 8, a_hi = lane >> 4;      // ldmatrix: A tile row, low / high k half
-  const uint32_t a_base = a_row * 128;
-  const int a_swz = a_row & 7;
-  const int b_tok = lane & 7, b_m = lane >> 3;                                 // ldmatrix: token row, k piece
+  // phase-2 chunk: 64 slab rows x 32 bytes, contiguous in memory; lane copies pieces lane + 32j; half p of row r sits at p ^ bit 2 of r
+  const uint32_t cq_off = (lane >> 1) * 32 + (((lane & 1) ^ ((lane >> 3) & 1)) << 4);
+  // ldmatrix lane roles: A tile row and k half (low / high 8), B token row and k piece
+  const int a_row = (lane & 7) + ((lane >> 3) & 1) * 8, a_hi = lane >> 4;
+  const uint32_t a1_base = a_row * 128;
+  const int a1_swz = a_row & 7;
+  const uint32_t a2_off = a_row * 32 + ((a_hi ^ ((a_row >> 2) & 1)) << 4);
+  const int b_tok = lane & 7, b_m = lane >> 3;
   const uint32_t xs_lane = st_smem_u32(xs) + (uint32_t)b_tok * H * 2;
   const int tile = warp & 1, ks = warp >> 1;     // phase 1: this warp's 16-row tile (gate | up) and hidden slice
   const __nv_bfloat16* wmat = tile ? a.w_up : a.w_gate;
 
-  // One pass: phase 1 over groups [s_lo, s_hi) (may be empty), then the phase-2 jobs.
-  auto run_pass = [&](int s_lo, int s_hi, const StJob* jobs, int nj) {
+  for (int s_lo = g_lo, s_hi; s_lo < g_hi; s_lo = s_hi) {
+    s_hi = min(g_hi, s_lo + kStPassGroups);
     const int ng = s_hi - s_lo;
-    // ---- group table: lane q holds expert and first column of group q ----
-    int my_e = 0, my_col = 0;
+    // ---- group table: lane q holds item, expert and position of group q ----
+    int my_item = -1, my_e = 0, my_gi = 0;
     if (lane < ng) {
       const int grp = s_lo + lane;
-      const int item = grp / NG;
-      my_e = a.items[item].e;
-      my_col = (grp - item * NG) * 16;
-      if (warp == 0) {
-        s_item[lane] = item;
-        s_col[lane] = my_col;
-      }
+      my_item = grp / NG;
+      my_e = a.items[my_item].e;
+      my_gi = grp - my_item * NG;
     }
-    // ---- job table: expert of each phase-2 job ----
-    int je[kStScWindows] = {};
-#pragma unroll
-    for (int jj = 0; jj < kStScWindows; ++jj)
-      if (jj < nj) je[jj] = a.items[(4 * jobs[jj].W) / NG].e;
-    const int n1 = ng * NCH;
-    // ---- issue side: phase-1 chunks, then phase-2 units, then empty groups ----
-    auto n_units = [&](int jj) { const StJob& j = jobs[jj]; return (j.b * HT / 4 - j.a * HT / 4) * 8; };
-    auto first_valid = [&](int& jj, int& u) {
-      while (jj < nj && u >= n_units(jj)) { ++jj; u = warp; }
-    };
+    // ---- issue side: phase-1 chunks, then phase-2 chunks, then empty groups ----
+    const int n1 = ng * NCH, n2 = ng * CPG;
     int n_issued = 0, iq = 0, icc = 0;
-    const __nv_bfloat16* p1_src = nullptr;
-    int ij = 0, iu = warp;
-    first_valid(ij, iu);
+    const __nv_bfloat16* i_src = nullptr;
     auto issue_one = [&]() {
       const uint32_t dst = ring + (uint32_t)(n_issued % SLOTS) * kStChunkBytes;
-      const __nv_bfloat16* src = nullptr;
-      size_t stride = 0;
       if (n_issued < n1) {
         if (icc == 0) {
-          const int e = __shfl_sync(0xffffffffu, my_e, iq), col = __shfl_sync(0xffffffffu, my_col, iq);
-          p1_src = wmat + ((size_t)e * I + col) * H + (size_t)ks * KS;
+          const int e = __shfl_sync(0xffffffffu, my_e, iq), gi = __shfl_sync(0xffffffffu, my_gi, iq);
+          i_src = wmat + ((size_t)e * I + gi * 16 + cp_row) * H + ks * KS + cp_piece * 8;
         }
-        src = p1_src + icc * 64;
-        stride = H;
-        if (++icc == NCH) { icc = 0; ++iq; }
-      } else if (ij < nj) {
-        const StJob& j = jobs[ij];
-        const int item = (4 * j.W) / NG, w = j.W - item * WPI;
-        int e = je[0];
-#pragma unroll
-        for (int jj = 1; jj < kStScWindows; ++jj)
-          if (jj == ij) e = je[jj];
-        const int h0 = (j.a * HT / 4) * 128 + iu * 16;
-        src = a.w_down + ((size_t)e * H + h0) * I + w * 64;
-        stride = I;
-        iu += kStWarps;
-        first_valid(ij, iu);
-      }
-      if (src != nullptr) {
-        const __nv_bfloat16* p = src + (size_t)cp_row * stride + cp_piece * 8;
+        const __nv_bfloat16* p = i_src + icc * 64;
         st_cp16(dst + cp_off0, p);
-        st_cp16(dst + cp_off1, p + 4 * stride);
-        st_cp16(dst + cp_off0 + 1024, p + 8 * stride);
-        st_cp16(dst + cp_off1 + 1024, p + 12 * stride);
+        st_cp16(dst + cp_off1, p + 4 * (size_t)H);
+        st_cp16(dst + cp_off0 + 1024, p + 8 * (size_t)H);
+        st_cp16(dst + cp_off1 + 1024, p + 12 * (size_t)H);
+        if (++icc == NCH) {
+          icc = 0;
+          if (++iq == ng) iq = 0;      // phase 2 walks the groups again
+        }
+      } else if (n_issued < n1 + n2) {
+        if (icc == 0) {
+          const int e = __shfl_sync(0xffffffffu, my_e, iq), gi = __shfl_sync(0xffffffffu, my_gi, iq);
+          i_src = a.w_down + (((size_t)e * NG + gi) * H + warp * HW) * 16 + lane * 8;
+        }
+        const __nv_bfloat16* p = i_src + icc * 1024;
+        st_cp16(dst + cq_off, p);
+        st_cp16(dst + cq_off + 512, p + 256);
+        st_cp16(dst + cq_off + 1024, p + 512);
+        st_cp16(dst + cq_off + 1536, p + 768);
+        if (++icc == CPG) {
+          icc = 0;
+          ++iq;
+        }
       }
       st_commit();
       ++n_issued;
     };
-    // A fragments of k16 step s of the chunk in a slot
-    auto load_a = [&](uint32_t slot, int s, uint32_t (&af)[4]) {
-      st_ldmatrix4(slot + a_base + (uint32_t)(((2 * s + a_hi) ^ a_swz) << 4), af);
-    };
 #pragma unroll
     for (int b = 0; b < SLOTS - 1; ++b) issue_one();
-    // ---- routing weights of this thread's two tokens (2c, 2c + 1) for each job's expert ----
-    float jwA[kStScWindows] = {}, jwB[kStScWindows] = {};
-#pragma unroll
-    for (int jj = 0; jj < kStScWindows; ++jj) {
-      if (jj < nj) {
-        const WorkItem it = a.items[(4 * jobs[jj].W) / NG];
-        int row = -1;
-        float wt = 0.f;
-        if (lane < it.n) slot_row_weight(a.perm[it.begin + lane], T, d.k, a.topk_w, row, wt);
-#pragma unroll
-        for (int r = 0; r < kStRows; ++r) {
-          const int rr = __shfl_sync(0xffffffffu, row, r);
-          const float ww = __shfl_sync(0xffffffffu, wt, r);
-          if (rr == 2 * c) jwA[jj] = ww;
-          if (rr == 2 * c + 1) jwB[jj] = ww;
-        }
+
+    // ---- routing weights of the pass's experts, per group and token (read in phase 2, after the barriers) ----
+    if (warp < ng) {
+      const int item = __shfl_sync(0xffffffffu, my_item, warp);
+      const WorkItem it = a.items[item];
+      if (lane < kStRows) s_w[warp][lane] = 0.f;
+      if (lane == 0) s_item[warp] = item;
+      __syncwarp();
+      if (lane < it.n) {
+        int row;
+        float wt;
+        slot_row_weight(a.perm[it.begin + lane], T, d.k, a.topk_w, row, wt);
+        s_w[warp][row] = wt;
       }
     }
+
+    // ---- phase 1 ----
     int t = 0;     // chunks consumed in this pass
-    if (ng > 0) {
-      // ---- phase 1 ----
+    {
       float acc[4] = {0.f, 0.f, 0.f, 0.f};
       int q = 0, cc = 0;
       for (; t < n1; ++t) {
@@ -255,13 +218,13 @@ __global__ void __launch_bounds__(kStThreads, 1) k_experts_stream(StArgs a) {
         st_ldmatrix4(xs_lane + (uint32_t)((p0 + (b_m ^ b_tok)) << 4), bf0);
         st_ldmatrix4(xs_lane + (uint32_t)((p0 + ((4 + b_m) ^ b_tok)) << 4), bf1);
         uint32_t af[4];
-        load_a(slot, 0, af);
+        st_ldmatrix4(slot + a1_base + (uint32_t)(((0 + a_hi) ^ a1_swz) << 4), af);
         st_mma(acc, af, bf0[0], bf0[1]);
-        load_a(slot, 1, af);
+        st_ldmatrix4(slot + a1_base + (uint32_t)(((2 + a_hi) ^ a1_swz) << 4), af);
         st_mma(acc, af, bf0[2], bf0[3]);
-        load_a(slot, 2, af);
+        st_ldmatrix4(slot + a1_base + (uint32_t)(((4 + a_hi) ^ a1_swz) << 4), af);
         st_mma(acc, af, bf1[0], bf1[1]);
-        load_a(slot, 3, af);
+        st_ldmatrix4(slot + a1_base + (uint32_t)(((6 + a_hi) ^ a1_swz) << 4), af);
         st_mma(acc, af, bf1[2], bf1[3]);
         __syncwarp();                                           // the slot may be overwritten from here on
         if (++cc == NCH) {
@@ -273,162 +236,75 @@ __global__ void __launch_bounds__(kStThreads, 1) k_experts_stream(StArgs a) {
           ++q;
         }
       }
-      __syncthreads();
-      // ---- sum the slices, SwiGLU, publish ----
-      for (int idx = tid; idx < ng * 16 * kStRows; idx += kStThreads) {
-        const int qq = idx >> 7, r = (idx >> 3) & 15, n = idx & 7;
-        float gs = 0.f, us = 0.f;
-#pragma unroll
-        for (int s = 0; s < kStSlices; ++s) {
-          const float* base = red + ((size_t)((qq * kStSlices + s) * 2) * 16) * kStRows + r * kStRows + n;
-          gs += base[0];
-          us += base[16 * kStRows];
-        }
-        if (n < T)
-          a.act_g[((size_t)s_item[qq] * 16 + n) * I + s_col[qq] + r] = __float2bfloat16_rn(gs / (1.f + expf(-gs)) * us);
-      }
-      __syncthreads();
-      if (tid < kStScWindows) {
-        const int w = (s_lo >> 2) + tid;
-        if (w <= ((s_hi - 1) >> 2)) {
-          __threadfence();      // the CTA's activations are visible device-wide before the count moves
-          atomicAdd(a.win_flags + w, min(s_hi, 4 * w + 4) - max(s_lo, 4 * w));
-        }
-      }
     }
+    __syncthreads();
+    // ---- sum the slices, SwiGLU ----
+    for (int idx = tid; idx < ng * 16 * kStRows; idx += kStThreads) {
+      const int qq = idx >> 7, r = (idx >> 3) & 15, n = idx & 7;
+      float gs = 0.f, us = 0.f;
+#pragma unroll
+      for (int s = 0; s < kStSlices; ++s) {
+        const float* base = red + ((size_t)((qq * kStSlices + s) * 2) * 16) * kStRows + r * kStRows + n;
+        gs += base[0];
+        us += base[16 * kStRows];
+      }
+      s_act[qq][n][r] = __float2bfloat16_rn(gs / (1.f + expf(-gs)) * us);     // rows n >= T are zero (x is)
+    }
+    __syncthreads();
     // ---- phase 2 ----
-    // Activations of a job's window as B fragments, once all four groups are published.  Without
-    // `block` a window that is not complete yet is left for later.
-    uint32_t bfr[kStScWindows][4][2] = {};
-    bool ready[kStScWindows] = {};
-    auto prep = [&](int jj, bool block) {
-      const StJob& j = jobs[jj];
-      bool have = j.a == 0 && j.b == 4;        // all four groups are this CTA's own
-      if (!have) {
-        int seen = 0;
-        if (lane == 0) {
-          const unsigned long long t0 = clock64();
-          while ((seen = st_ld_acquire(a.win_flags + j.W)) < 4 && block) {
-            __nanosleep(64);
-            if (clock64() - t0 > kStWaitCycles) {
-              set_status(a.status, TEAM_ERR_TIMEOUT, 21);
-              break;
+    {
+      float acc[CPG * 4][4];
+#pragma unroll
+      for (int u = 0; u < CPG * 4; ++u) acc[u][0] = acc[u][1] = acc[u][2] = acc[u][3] = 0.f;
+      for (int q = 0; q < ng; ++q) {
+        const uint32_t b0 = *reinterpret_cast<const uint32_t*>(&s_act[q][g][2 * c]);
+        const uint32_t b1 = *reinterpret_cast<const uint32_t*>(&s_act[q][g][8 + 2 * c]);
+#pragma unroll
+        for (int ch = 0; ch < CPG; ++ch, ++t) {
+          issue_one();
+          st_wait_group<SLOTS - 1>();
+          __syncwarp();
+          const uint32_t slot = ring + (uint32_t)(t % SLOTS) * kStChunkBytes;
+#pragma unroll
+          for (int u = 0; u < 4; ++u) {
+            uint32_t af[4];
+            st_ldmatrix4(slot + u * 512 + a2_off, af);
+            st_mma(acc[ch * 4 + u], af, b0, b1);
+          }
+          __syncwarp();
+        }
+        // the expert's groups in this pass are summed: scale by the routing weights and add to y
+        if (q == ng - 1 || s_item[q + 1] != s_item[q]) {
+          const float wA = s_w[q][2 * c], wB = s_w[q][2 * c + 1];
+          float* y0 = a.y + (size_t)(2 * c) * H + warp * HW + g;
+#pragma unroll
+          for (int u = 0; u < CPG * 4; ++u) {
+            if (wA != 0.f) {
+              atomicAdd(y0 + u * 16, wA * acc[u][0]);
+              atomicAdd(y0 + u * 16 + 8, wA * acc[u][2]);
             }
+            if (wB != 0.f) {
+              atomicAdd(y0 + H + u * 16, wB * acc[u][1]);
+              atomicAdd(y0 + H + u * 16 + 8, wB * acc[u][3]);
+            }
+            acc[u][0] = acc[u][1] = acc[u][2] = acc[u][3] = 0.f;
           }
         }
-        seen = __shfl_sync(0xffffffffu, seen, 0);
-        have = seen >= 4;
-        if (block && !have) ok = false;
       }
-      if (have) {
-        const int item = (4 * j.W) / NG, w = j.W - item * WPI;
-        const __nv_bfloat16* ap = a.act_g + ((size_t)item * 16 + g) * I + w * 64 + 2 * c;
-#pragma unroll
-        for (int s = 0; s < 4; ++s) {
-          bfr[jj][s][0] = st_ldg_l2(ap + s * 16);
-          bfr[jj][s][1] = st_ldg_l2(ap + s * 16 + 8);
-        }
-        ready[jj] = true;
-      }
-    };
-#pragma unroll
-    for (int jj = 0; jj < kStScWindows; ++jj)
-      if (jj < nj && ok) prep(jj, false);
-    int cj = 0, cu = warp, cur_job = -1;
-    first_valid(cj, cu);
-    uint32_t cur[4][2] = {};
-    float wA = 0.f, wB = 0.f;
-    for (; cj < nj; ++t) {
-      issue_one();
-      st_wait_group<SLOTS - 1>();
-      __syncwarp();
-      if (cj != cur_job && ok) {
-#pragma unroll
-        for (int jj = 0; jj < kStScWindows; ++jj) {
-          if (jj == cj) {
-            if (!ready[jj]) prep(jj, true);
-#pragma unroll
-            for (int s = 0; s < 4; ++s) {
-              cur[s][0] = bfr[jj][s][0];
-              cur[s][1] = bfr[jj][s][1];
-            }
-            wA = jwA[jj];
-            wB = jwB[jj];
-          }
-        }
-        cur_job = cj;
-      }
-      if (ok) {      // after a wait ran out the warp only drains its copies
-        const uint32_t slot = ring + (uint32_t)(t % SLOTS) * kStChunkBytes;
-        float acc[4] = {0.f, 0.f, 0.f, 0.f};
-        uint32_t af[4];
-#pragma unroll
-        for (int s = 0; s < 4; ++s) {
-          load_a(slot, s, af);
-          st_mma(acc, af, cur[s][0], cur[s][1]);
-        }
-        const int h = (jobs[cj].a * HT / 4) * 128 + cu * 16 + g;
-        float* y0 = a.y + (size_t)(2 * c) * H + h;
-        if (wA != 0.f) {
-          atomicAdd(y0, wA * acc[0]);
-          atomicAdd(y0 + 8, wA * acc[2]);
-        }
-        if (wB != 0.f) {
-          atomicAdd(y0 + H, wB * acc[1]);
-          atomicAdd(y0 + H + 8, wB * acc[3]);
-        }
-      }
-      __syncwarp();
-      cu += kStWarps;
-      first_valid(cj, cu);
     }
     st_wait_group<0>();     // only empty groups can be pending here
-    __syncwarp();
-  };
-
-  // ---- passes: fully owned windows first, shared ones after; a multi-pass range keeps its head window for last ----
-  for (int s_lo = g_lo, s_hi; s_lo < g_hi; s_lo = s_hi) {
-    s_hi = min(g_hi, ((s_lo >> 2) + kStScWindows) << 2);
-    StJob jobs[kStScWindows];
-    int nj = 0;
-#pragma unroll
-    for (int pass = 0; pass < 2; ++pass) {
-#pragma unroll
-      for (int k = 0; k < kStScWindows; ++k) {
-        const int w = (s_lo >> 2) + k;
-        if (w <= ((s_hi - 1) >> 2)) {
-          const int ja = max(s_lo, 4 * w) - 4 * w, jb = min(s_hi, 4 * w + 4) - 4 * w;
-          const bool full = ja == 0 && jb == 4;
-          const bool deferred = multi && w == (g_lo >> 2) && (g_lo & 3) != 0;
-          if (full == (pass == 0) && !deferred && ja * HT / 4 < jb * HT / 4) {
-            jobs[nj].W = w;
-            jobs[nj].a = ja;
-            jobs[nj].b = jb;
-            ++nj;
-          }
-        }
-      }
-    }
-    run_pass(s_lo, s_hi, jobs, nj);
-  }
-  if (multi && (g_lo & 3) != 0) {
-    StJob job;
-    job.W = g_lo >> 2;
-    job.a = g_lo & 3;
-    job.b = min(g_hi, 4 * job.W + 4) - 4 * job.W;
-    if (job.a * HT / 4 < job.b * HT / 4) run_pass(g_lo, g_lo, &job, 1);
+    __syncthreads();        // s_act, s_w and the partial sums are free for the next pass
   }
 }
 
 bool experts_stream_supported(int max_rows, int hidden, int inter) {
-  return max_rows <= kStRows && hidden % (kStSlices * 64) == 0 && hidden <= 4096 && inter % 64 == 0;
+  return max_rows <= kStRows && (hidden == 1024 || hidden == 2048) && inter % 16 == 0;
 }
 
 cudaError_t configure_experts_stream(int hidden) {
-  const void* fn = stream_ring_slots(hidden) == 4 ? reinterpret_cast<const void*>(&k_experts_stream<4>)
-                                                  : reinterpret_cast<const void*>(&k_experts_stream<3>);
-  cudaError_t e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       (int)stream_smem_bytes(stream_ring_slots(hidden) == 4 ? 2048 : 4096));
+  const void* fn = hidden == 1024 ? reinterpret_cast<const void*>(&k_experts_stream<1>)
+                                  : reinterpret_cast<const void*>(&k_experts_stream<2>);
+  cudaError_t e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)stream_smem_bytes(hidden));
   if (e == cudaSuccess) e = cudaFuncSetAttribute(fn, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
   return e;
 }
@@ -444,27 +320,20 @@ cudaError_t launch_experts_stream(const void* x, const void* w_gate, const void*
   a.topk_w = ws.r.topk_w;
   a.items = ws.items;
   a.n_items = ws.n_items;
-  a.act_g = ws.act_g;
-  a.win_flags = ws.win_flags;
   a.y = y;
-  a.status = ws.status;
   a.d = d;
-  // Cooperative: CTAs that share a window wait for each other's activations, so all must be resident.
   // Programmatic serialization: staging the token rows overlaps the selection kernel.
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(grid);
   cfg.blockDim = dim3(kStThreads);
   cfg.dynamicSmemBytes = stream_smem_bytes(d.H);
   cfg.stream = s;
-  cudaLaunchAttribute attrs[2];
-  attrs[0].id = cudaLaunchAttributeCooperative;
-  attrs[0].val.cooperative = 1;
-  attrs[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  attrs[1].val.programmaticStreamSerializationAllowed = 1;
+  cudaLaunchAttribute attrs[1];
+  attrs[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attrs[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attrs;
-  cfg.numAttrs = 2;
-  return stream_ring_slots(d.H) == 4 ? cudaLaunchKernelEx(&cfg, k_experts_stream<4>, a)
-                                     : cudaLaunchKernelEx(&cfg, k_experts_stream<3>, a);
+  cfg.numAttrs = 1;
+  return d.H == 1024 ? cudaLaunchKernelEx(&cfg, k_experts_stream<1>, a) : cudaLaunchKernelEx(&cfg, k_experts_stream<2>, a);
 }
 
 }  // namespace team

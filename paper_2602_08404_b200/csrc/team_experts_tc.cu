@@ -229,7 +229,7 @@ struct TcArgs {
   const __nv_bfloat16* x;       // [T, H]
   const __nv_bfloat16* w_gate;  // [E + ns, I, H]
   const __nv_bfloat16* w_up;    // [E + ns, I, H]
-  const __nv_bfloat16* w_down;  // [E + ns, H, I]
+  const __nv_bfloat16* w_down;  // [E + ns, I/16, H, 16]
   const int32_t* perm;          // slot ids grouped by expert
   const float* topk_w;          // [T, k]
   const WorkItem* items;
@@ -537,9 +537,12 @@ k_experts_tc(TcArgs a) {
     const __nv_bfloat16* src2 = nullptr;    // phase 2: this lane's first row of the next W_down tile
     const int rr0 = warp * RPI + sub;       // phase 1: first row inside a 16-row block; the others follow RSTEP apart
     const uint32_t dst1 = (uint32_t)rr0 * 128u + (uint32_t)((ch ^ (rr0 & 7)) << 4);   // (RSTEP is a multiple of 8: same swizzle)
-    const int r_first = warp * 4 + (lane >> 3);                                       // phase 2: 4 rows x 128 B per instruction
-    const uint32_t dst2 = sw128(r_first, ch);
-    const size_t rstep1 = (size_t)RSTEP * d.H, rstep2 = (size_t)(4 * kLoaders) * d.I, tstep2 = (size_t)128 * d.I;
+    // phase 2: W_down is stored in slabs of 16 columns ([I/16][H][16]); a window's 128-byte tile row is
+    // gathered from four slabs.  Per instruction a warp copies 4 rows x 32 bytes from each of them.
+    const int r_first = warp * 4 + ((lane & 7) >> 1);
+    const int ch2 = (lane >> 3) * 2 + (lane & 1);                                     // 16-byte piece of the tile row
+    const uint32_t dst2 = sw128(r_first, ch2);
+    const size_t rstep1 = (size_t)RSTEP * d.H, rstep2 = (size_t)(4 * kLoaders) * 16, tstep2 = (size_t)128 * 16;
     int ncols = 0;
 #pragma unroll
     for (int q = 0; q < 4; ++q) src1[q][0] = src1[q][1] = nullptr;
@@ -605,8 +608,8 @@ k_experts_tc(TcArgs a) {
       } else {
         if (st.first) {
           const WorkItem item = a.items[op.item];
-          src2 = a.w_down + ((size_t)item.e * d.H + (size_t)st.k0 * 128 + r_first) * d.I +
-                 (op.W - op.item * WPI) * kWindowCols + ch * 8;
+          src2 = a.w_down + (((size_t)item.e * NG + (op.W - op.item * WPI) * 4 + (ch2 >> 1)) * d.H +
+                             (size_t)st.k0 * 128 + r_first) * 16 + (ch2 & 1) * 8;
         }
         for (int i = 0; i < st.n; ++i, src2 += tstep2) {
           const uint32_t dstA = base + i * kATileBytes + dst2;

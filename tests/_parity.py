@@ -35,7 +35,7 @@ class Layer:
         self.ctx = B.team_create(self.cfg)
         dc = dtype_code(shape)
         self.w = [torch.as_tensor(weights["w_router"]).cuda().contiguous(), B.to_device(weights["w_gate"], dc),
-                  B.to_device(weights["w_up"], dc), B.to_device(weights["w_down"], dc)]
+                  B.to_device(weights["w_up"], dc), B.team_pack_w_down(B.to_device(weights["w_down"], dc))]
         B.team_set_weights(self.ctx, *self.w)
 
     def close(self):

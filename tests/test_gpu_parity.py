@@ -25,6 +25,18 @@ def weights_cache():
     return get
 
 
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16], ids=["f32", "bf16"])
+def test_pack_w_down_is_the_stated_permutation(dtype):
+    n, H, I = 3, 40, 48
+    gen = torch.Generator().manual_seed(5)
+    src = torch.randn((n, H, I), generator=gen).to(dtype)
+    expected = src.view(n, H, I // 16, 16).permute(0, 2, 1, 3).contiguous()       # [n, I/16, H, 16]
+    got = B.team_pack_w_down(src.cuda())
+    torch.cuda.synchronize()
+    assert got.shape == src.shape and got.dtype == dtype
+    assert torch.equal(got.cpu().view(n, I // 16, H, 16), expected)
+
+
 @pytest.mark.parametrize("flags", ALL_FLAGS)
 def test_c1_tiny_fp32_all_steps(flags, weights_cache):
     stats = P.run_schedule(W.C1, weights_cache(W.C1), W.make_schedule(W.C1), flags)

@@ -49,6 +49,13 @@ def test_argument_checks_need_no_device(library):
     assert library.team_create(ctypes.byref(bad), ctypes.byref(ctx)) == B.TEAM_ERR_SHAPE
     assert library.team_destroy(None) == B.TEAM_ERR_ARG
     assert library.team_moe_forward(None, None, None, None, None, None) == B.TEAM_ERR_ARG
+    # weight packing: arguments are validated before anything touches the device
+    p, q = ctypes.c_void_p(0x1000), ctypes.c_void_p(0x2000)
+    assert library.team_pack_w_down(None, q, 1, 128, 64, B.TEAM_DTYPE_BF16, None) == B.TEAM_ERR_ARG
+    assert library.team_pack_w_down(p, p, 1, 128, 64, B.TEAM_DTYPE_BF16, None) == B.TEAM_ERR_ARG          # in place
+    assert library.team_pack_w_down(ctypes.c_void_p(0x1008), q, 1, 128, 64, B.TEAM_DTYPE_BF16, None) == B.TEAM_ERR_ARG
+    assert library.team_pack_w_down(p, q, 1, 128, 72, B.TEAM_DTYPE_BF16, None) == B.TEAM_ERR_SHAPE       # 72 % 16
+    assert library.team_pack_w_down(p, q, 1, 128, 64, 7, None) == B.TEAM_ERR_SHAPE                       # dtype
 
 
 def test_no_cpu_fallback(library):

@@ -37,7 +37,7 @@ def _route_both(shape, step, flags):
     ctx = B.team_create(cfg)
     try:
         B.team_set_weights(ctx, w_router, B.to_device(weights["w_gate"], dc), B.to_device(weights["w_up"], dc),
-                           B.to_device(weights["w_down"], dc))
+                           B.team_pack_w_down(B.to_device(weights["w_down"], dc)))
         ref = B.alloc_routing(cfg, T)
         B.team_route(ctx, x, st, ref)
         torch.cuda.synchronize()
