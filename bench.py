@@ -364,8 +364,9 @@ def main():
                      "peak_kind": f"of {peak_kind}", "unit": "GB/s", "frac": achieved / peak,
                      "frac_of_8TBs_nominal": achieved / 8000.0, "kernel_ms": kernel_ms,
                      "algorithmic_bytes_per_launch": algo_bytes, "launches_timed": tot_n,
-                     # no DRAM counters have been taken for this kernel yet
-                     "traffic": None},
+                     # DRAM read + write bytes per launch: ncu capture at 16 activated experts (151.06 MB read +
+                     # 3.6 MB written, profiles/experts_stream_c2_bench.md), scaled to this run's mean
+                     "traffic": mean_act * (151.06e6 + 3.6e6) / 16.0 if (H, I) == (2048, 768) else None},
     }
 
     if rank == 0:
