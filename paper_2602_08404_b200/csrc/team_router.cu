@@ -205,7 +205,7 @@ k_router_topk(const float* __restrict__ logits, const uint8_t* __restrict__ tok_
       if (e < d.E) out.probs[(size_t)t * d.E + e] = expf(v[i] - row_max) / denom;
     }
   }
-  TopkResult r = warp_topk(v, d.k, lane);
+  TopkResult r = warp_topk(v, d.k, lane, (d.E + 31) / 32);
   const float w = routing_weight(r, d.k, lane, row_max, denom, p.norm_topk);
   if (lane < d.k) {
     if (out.topk_idx) out.topk_idx[t * d.k + lane] = r.idx;

@@ -17,6 +17,7 @@ constexpr int kSelThreads = 1024;
 constexpr int kSelWarps = kSelThreads / 32;
 
 constexpr int kIdxInSmemMax = 8192;   // routed slots kept in shared memory between the rounds and the dispatch
+constexpr int kSmallSlots = 128;      // up to here every expert's thread counts and places its slots by itself
 
 struct SelSmem {
   // carved from dynamic shared memory in this order
@@ -26,6 +27,7 @@ struct SelSmem {
   int32_t* key;        // [T] group*256 + branch
   int32_t* pos;        // [T]
   int32_t* warp_cnt;   // [kSelWarps + 1]
+  int32_t* scan_tot;   // [3][kSelWarps] per-warp totals of the scan over experts: slots, work items, active experts
   int32_t* idx;        // [min(T*k, kIdxInSmemMax)]
   uint8_t* state;      // [T]
   uint8_t* cls;        // [T]
@@ -47,6 +49,7 @@ __host__ __device__ inline size_t sel_smem_layout(Dims d, SelSmem* s, unsigned c
   size_t a_key = take((size_t)d.T * 4);
   size_t a_pos = take((size_t)d.T * 4);
   size_t a_wc = take((size_t)(kSelWarps + 1) * 4);
+  size_t a_st = take((size_t)3 * kSelWarps * 4);
   size_t a_idx = take((size_t)n_idx * 4);
   size_t a_state = take((size_t)d.T);
   size_t a_cls = take((size_t)d.T);
@@ -58,6 +61,7 @@ __host__ __device__ inline size_t sel_smem_layout(Dims d, SelSmem* s, unsigned c
     s->key = reinterpret_cast<int32_t*>(base + a_key);
     s->pos = reinterpret_cast<int32_t*>(base + a_pos);
     s->warp_cnt = reinterpret_cast<int32_t*>(base + a_wc);
+    s->scan_tot = reinterpret_cast<int32_t*>(base + a_st);
     s->idx = n_idx ? reinterpret_cast<int32_t*>(base + a_idx) : nullptr;
     s->state = base + a_state;
     s->cls = base + a_cls;
@@ -110,13 +114,6 @@ k_select(const float* __restrict__ logits, StepPtrs st, Workspace ws, RoutePtrs 
     s.pos[t] = st.pos[t];
     s.state[t] = st.tok_state[t];
   }
-  // The logits come from the preceding kernel of the stream.
-  if (wait_prior) asm volatile("griddepcontrol.wait;" ::: "memory");
-  // With at most one row per warp the row's logits are fetched now and stay in registers through
-  // both routing rounds.
-  float keep[kMaxPerLane];
-  float keep_max = 0.f, keep_denom = 1.f;
-  if (one_row_per_warp && warp < T) load_row(logits + (size_t)warp * E, E, lane, keep, keep_max, keep_denom);
   __syncthreads();
 
   // ---- Eq. 4: classification --------------------------------------------------------------
@@ -150,6 +147,15 @@ k_select(const float* __restrict__ logits, StepPtrs st, Workspace ws, RoutePtrs 
   // rewrites rows it classified itself, so the next barrier is the one after round 1's reads.)
   for (int t = tid; t < T; t += kSelThreads)
     if (s.cls[t] == TEAM_CLS_COLD && !s.has_first[s.key[t] >> 8]) s.cls[t] = TEAM_CLS_FIRST;
+
+  // Everything above depends on the step state only (inputs of the call) and overlaps the preceding
+  // kernel of the stream; the logits come from that kernel.
+  if (wait_prior) asm volatile("griddepcontrol.wait;" ::: "memory");
+  // With at most one row per warp the row's logits are fetched now and stay in registers through
+  // both routing rounds.
+  float keep[kMaxPerLane];
+  float keep_max = 0.f, keep_denom = 1.f;
+  if (one_row_per_warp && warp < T) load_row(logits + (size_t)warp * E, E, lane, keep, keep_max, keep_denom);
   __syncthreads();
 
   // ---- Algorithm 1, round 1 (free top-k) then round 2 (top-k inside E_A) -------------------
@@ -196,7 +202,7 @@ k_select(const float* __restrict__ logits, StepPtrs st, Workspace ws, RoutePtrs 
         for (int i = 0; i < kMaxPerLane; ++i)
           if (!((s.mask[g * n_words32 + i] >> lane) & 1u)) v[i] = kNegInf;
       }
-      TopkResult tr = warp_topk(v, k, lane);
+      TopkResult tr = warp_topk(v, k, lane, (E + 31) / 32);
       const float w = routing_weight(tr, k, lane, row_max, denom, p.norm_topk);
       if (lane < k) {
         if (s.idx) s.idx[t * k + lane] = tr.idx;
@@ -232,17 +238,23 @@ k_select(const float* __restrict__ logits, StepPtrs st, Workspace ws, RoutePtrs 
   }
 
   // ---- dispatch: stable counting sort of slots by expert ------------------------------------
-  // Routed slots t*k+j are walked in ascending order, warp w < nw owning a contiguous range, so the
-  // rank of a slot inside its expert is (slots of that expert in earlier warps) + (earlier in this warp).
+  // Small steps (at most kSmallSlots routed slots): expert e's thread counts its slots by walking the
+  // slot list in shared memory and, after the scan, walks it again to place them (ascending slot id).
+  // Larger steps: routed slots t*k+j are walked in ascending order, warp w < nw owning a contiguous
+  // range, so the rank of a slot inside its expert is (slots of that expert in earlier warps) +
+  // (earlier in this warp).
+  const bool small = s.idx != nullptr && S <= kSmallSlots;
   const int per_warp = ((S + nw - 1) / nw + 31) & ~31;
   const int lo = min(S, warp * per_warp), hi = warp < nw ? min(S, lo + per_warp) : lo;
   int32_t* my_hist = s.hist + (warp < nw ? warp : 0) * EN;
-  for (int base = lo; base < hi; base += 32) {
-    const int slot = base + lane;
-    const int e = (slot < hi) ? idx_src[slot] : -1;
-    const unsigned peers = __match_any_sync(0xffffffffu, e);
-    if (e >= 0 && (__ffs(peers) - 1) == lane) my_hist[e] += __popc(peers);
-    __syncwarp();
+  if (!small) {
+    for (int base = lo; base < hi; base += 32) {
+      const int slot = base + lane;
+      const int e = (slot < hi) ? idx_src[slot] : -1;
+      const unsigned peers = __match_any_sync(0xffffffffu, e);
+      if (e >= 0 && (__ffs(peers) - 1) == lane) my_hist[e] += __popc(peers);
+      __syncwarp();
+    }
   }
   // number of computed rows; shared experts take every one of them
   {
@@ -260,124 +272,155 @@ k_select(const float* __restrict__ logits, StepPtrs st, Workspace ws, RoutePtrs 
     const int used = min(kSelWarps, (T + 31) / 32);
     for (int w = 0; w < used; ++w) n_rows_active += s.warp_cnt[w];
   }
-  // per expert: turn per-warp counts into per-warp starting ranks, total into off[e+1]
-  for (int e = tid; e < EN; e += kSelThreads) {
-    int run = 0;
+  // ---- per-expert counts, then a scan over experts by ceil(EN / 32) warps ----------------------
+  const int nwe = (EN + 31) / 32;            // EN <= 260: at most 9 warps, expert e = tid
+  int c = 0, tiles = 0, incl_c = 0, incl_t = 0, arank = 0;
+  unsigned act_b = 0;
+  if (warp < nwe) {
+    const int e = tid;
     if (e < E) {
-      for (int w = 0; w < nw; ++w) {
-        const int c = s.hist[w * EN + e];
-        s.hist[w * EN + e] = run;
-        run += c;
+      if (small) {
+        for (int i = 0; i < S; ++i) c += (s.idx[i] == e);
+      } else {
+        // turn per-warp counts into per-warp starting ranks
+        for (int w = 0; w < nw; ++w) {
+          const int cw = s.hist[w * EN + e];
+          s.hist[w * EN + e] = c;
+          c += cw;
+        }
       }
-    } else {
-      run = n_rows_active;
+    } else if (e < EN) {
+      c = n_rows_active;
     }
-    s.off[e + 1] = run;   // counts for now
+    tiles = (c + item_tile - 1) / item_tile;      // work items: ceil(c / item_tile) per expert
+    incl_c = c;
+    incl_t = tiles;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int n1 = __shfl_up_sync(0xffffffffu, incl_c, o), n2 = __shfl_up_sync(0xffffffffu, incl_t, o);
+      if (lane >= o) {
+        incl_c += n1;
+        incl_t += n2;
+      }
+    }
+    act_b = __ballot_sync(0xffffffffu, c > 0);
+    arank = __popc(act_b & ((1u << lane) - 1));
+    if (lane == 31) {
+      s.scan_tot[warp] = incl_c;
+      s.scan_tot[kSelWarps + warp] = incl_t;
+      s.scan_tot[2 * kSelWarps + warp] = __popc(act_b);
+    }
   }
-  if (tid == 0) s.off[0] = 0;
   __syncthreads();
-  // exclusive scan over experts (EN <= 260) by warp 0; also active list and work items
-  if (warp == 0) {
-    int carry = 0, n_act = 0, n_items = 0;
-    for (int base = 0; base < EN; base += 32) {
-      const int e = base + lane;
-      const int c = (e < EN) ? s.off[e + 1] : 0;
-      int incl = c;
-#pragma unroll
-      for (int o = 1; o < 32; o <<= 1) {
-        const int n = __shfl_up_sync(0xffffffffu, incl, o);
-        if (lane >= o) incl += n;
-      }
-      const int excl = carry + incl - c;
-      // active list
-      const unsigned act = __ballot_sync(0xffffffffu, c > 0);
-      const int arank = n_act + __popc(act & ((1u << lane) - 1));
-      // work items: ceil(c / item_tile) per expert
-      const int tiles = (c + item_tile - 1) / item_tile;
-      int tincl = tiles;
-#pragma unroll
-      for (int o = 1; o < 32; o <<= 1) {
-        const int n = __shfl_up_sync(0xffffffffu, tincl, o);
-        if (lane >= o) tincl += n;
-      }
-      const int tbase = n_items + tincl - tiles;
-      if (e < EN) {
-        r.expert_count[e] = c;
-        r.expert_offset[e] = excl;
-        if (ex.expert_count) ex.expert_count[e] = c;
-        if (ex.expert_offset) ex.expert_offset[e] = excl;
-        if (c > 0) {
-          r.active[arank] = e;
-          if (ex.active) ex.active[arank] = e;
-          for (int i = 0; i < tiles; ++i) {
-            WorkItem it;
-            it.e = e;
-            it.begin = excl + i * item_tile;
-            it.n = min(item_tile, c - i * item_tile);
-            it.pad = 0;
-            ws.items[tbase + i] = it;
+  int total = 0;
+  for (int w = 0; w < nwe; ++w) total += s.scan_tot[w];
+  if (warp < nwe) {
+    const int e = tid;
+    int pc = 0, pt = 0, pa = 0;
+    for (int w = 0; w < warp; ++w) {
+      pc += s.scan_tot[w];
+      pt += s.scan_tot[kSelWarps + w];
+      pa += s.scan_tot[2 * kSelWarps + w];
+    }
+    const int excl = pc + incl_c - c, tbase = pt + incl_t - tiles;
+    arank += pa;
+    if (e < EN) {
+      r.expert_count[e] = c;
+      r.expert_offset[e] = excl;
+      if (ex.expert_count) ex.expert_count[e] = c;
+      if (ex.expert_offset) ex.expert_offset[e] = excl;
+      if (!small) s.off[e] = excl;
+      if (c > 0) {
+        r.active[arank] = e;
+        if (ex.active) ex.active[arank] = e;
+        for (int i = 0; i < tiles; ++i) {
+          WorkItem it;
+          it.e = e;
+          it.begin = excl + i * item_tile;
+          it.n = min(item_tile, c - i * item_tile);
+          it.pad = 0;
+          ws.items[tbase + i] = it;
+        }
+        if (small) {
+          // place this expert's slots: routed ones by ascending slot id, a shared expert's by ascending row
+          int at = excl;
+          if (e < E) {
+            for (int i = 0; i < S; ++i) {
+              if (s.idx[i] == e) {
+                r.perm[at] = i;
+                if (ex.perm) ex.perm[at] = i;
+                ++at;
+              }
+            }
+          } else {
+            for (int t = 0; t < T; ++t) {
+              if (s.cls[t] != TEAM_CLS_SKIP) {
+                const int slot = T * k + (e - E) * T + t;
+                r.perm[at] = slot;
+                if (ex.perm) ex.perm[at] = slot;
+                ++at;
+              }
+            }
           }
         }
       }
-      __syncwarp();
-      if (e < EN) s.off[e] = excl;
-      carry += __shfl_sync(0xffffffffu, incl, 31);
-      n_act += __popc(act);
-      n_items += __shfl_sync(0xffffffffu, tincl, 31);
     }
-    // inactive tail of the active list
-    for (int i = n_act + lane; i < EN; i += 32) {
-      r.active[i] = -1;
-      if (ex.active) ex.active[i] = -1;
-    }
-    if (lane == 0) {
-      s.off[EN] = carry;
-      r.expert_offset[EN] = carry;
-      if (ex.expert_offset) ex.expert_offset[EN] = carry;
-      *r.n_active = n_act;
-      *r.n_rows_active = n_rows_active;
-      *ws.n_items = n_items;
-      if (ex.n_active) *ex.n_active = n_act;
-      if (ex.n_rows_active) *ex.n_rows_active = n_rows_active;
-    }
-  }
-  __syncthreads();
-  // second walk: place the routed slots
-  for (int base = lo; base < hi; base += 32) {
-    const int slot = base + lane;
-    const int e = (slot < hi) ? idx_src[slot] : -1;
-    const unsigned peers = __match_any_sync(0xffffffffu, e);
-    if (e >= 0) {
-      const int rank = my_hist[e] + __popc(peers & ((1u << lane) - 1));
-      const int at = s.off[e] + rank;
-      r.perm[at] = slot;
-      if (ex.perm) ex.perm[at] = slot;
-    }
-    __syncwarp();
-    if (e >= 0 && (__ffs(peers) - 1) == lane) my_hist[e] += __popc(peers);
-    __syncwarp();
-  }
-  // shared experts: slot T*k + s*T + t for every active row t, ascending t.
-  if (ns > 0 && warp == kSelWarps - 1) {
-    int run = 0;
-    for (int base = 0; base < T; base += 32) {
-      const int t = base + lane;
-      const bool a = t < T && s.cls[t] != TEAM_CLS_SKIP;
-      const unsigned b = __ballot_sync(0xffffffffu, a);
-      if (a) {
-        const int rank = run + __popc(b & ((1u << lane) - 1));
-        for (int sh = 0; sh < ns; ++sh) {
-          const int at = s.off[E + sh] + rank;
-          const int slot = T * k + sh * T + t;
-          r.perm[at] = slot;
-          if (ex.perm) ex.perm[at] = slot;
-        }
+    if (warp == nwe - 1) {
+      // inactive tail of the active list, and the totals
+      const int n_act = pa + __popc(act_b), n_items = pt + __shfl_sync(0xffffffffu, incl_t, 31);
+      for (int i = n_act + lane; i < EN; i += 32) {
+        r.active[i] = -1;
+        if (ex.active) ex.active[i] = -1;
       }
-      run += __popc(b);
+      if (lane == 0) {
+        r.expert_offset[EN] = total;
+        if (ex.expert_offset) ex.expert_offset[EN] = total;
+        *r.n_active = n_act;
+        *r.n_rows_active = n_rows_active;
+        *ws.n_items = n_items;
+        if (ex.n_active) *ex.n_active = n_act;
+        if (ex.n_rows_active) *ex.n_rows_active = n_rows_active;
+      }
+    }
+  }
+  if (!small) {
+    __syncthreads();
+    // second walk: place the routed slots
+    for (int base = lo; base < hi; base += 32) {
+      const int slot = base + lane;
+      const int e = (slot < hi) ? idx_src[slot] : -1;
+      const unsigned peers = __match_any_sync(0xffffffffu, e);
+      if (e >= 0) {
+        const int rank = my_hist[e] + __popc(peers & ((1u << lane) - 1));
+        const int at = s.off[e] + rank;
+        r.perm[at] = slot;
+        if (ex.perm) ex.perm[at] = slot;
+      }
+      __syncwarp();
+      if (e >= 0 && (__ffs(peers) - 1) == lane) my_hist[e] += __popc(peers);
+      __syncwarp();
+    }
+    // shared experts: slot T*k + s*T + t for every active row t, ascending t.
+    if (ns > 0 && warp == kSelWarps - 1) {
+      int run = 0;
+      for (int base = 0; base < T; base += 32) {
+        const int t = base + lane;
+        const bool a = t < T && s.cls[t] != TEAM_CLS_SKIP;
+        const unsigned b = __ballot_sync(0xffffffffu, a);
+        if (a) {
+          const int rank = run + __popc(b & ((1u << lane) - 1));
+          for (int sh = 0; sh < ns; ++sh) {
+            const int at = s.off[E + sh] + rank;
+            const int slot = T * k + sh * T + t;
+            r.perm[at] = slot;
+            if (ex.perm) ex.perm[at] = slot;
+          }
+        }
+        run += __popc(b);
+      }
     }
   }
   // unused tail of perm
-  const int total = s.off[EN];
   for (int i = total + tid; i < T * (k + ns); i += kSelThreads) {
     r.perm[i] = -1;
     if (ex.perm) ex.perm[i] = -1;

@@ -29,9 +29,10 @@ __device__ __forceinline__ float key_float(uint32_t k) {
 }
 
 // v[i] is the logit of expert i*32+lane, or -inf if that expert is not a candidate
-// (beyond E, or outside the allowed set).  v is consumed.  Each of the k+1 rounds takes the
-// warp-wide maximum key and then the lowest expert id among the lanes that hold it.
-__device__ __forceinline__ TopkResult warp_topk(float (&v)[kMaxPerLane], int k, int lane) {
+// (beyond E, or outside the allowed set); only the first ne = ceil(E / 32) entries are looked at.
+// The logits are turned into keys once.  Each of the k+1 rounds takes the warp-wide maximum key and
+// then the lowest expert id among the lanes that hold it, and retires that key.
+__device__ __forceinline__ TopkResult warp_topk(const float (&v)[kMaxPerLane], int k, int lane, int ne = kMaxPerLane) {
   TopkResult r;
   r.idx = -1;
   r.val = kNegInf;
@@ -39,21 +40,24 @@ __device__ __forceinline__ TopkResult warp_topk(float (&v)[kMaxPerLane], int k, 
   r.margin = __builtin_huge_valf();
   float last = kNegInf;
   const uint32_t key_neg_inf = float_key(kNegInf);
+  uint32_t key[kMaxPerLane];
+#pragma unroll
+  for (int i = 0; i < kMaxPerLane; ++i) key[i] = i < ne ? float_key(v[i]) : key_neg_inf;
   for (int j = 0; j <= k; ++j) {
     uint32_t bk = key_neg_inf;
-    int bi = 0x7fffffff;
+    int bi = 0;
 #pragma unroll
     for (int i = 0; i < kMaxPerLane; ++i) {
+      if (i >= ne) break;
       // ascending expert id within the lane, strict '>' keeps the lower id on ties
-      const uint32_t ki = float_key(v[i]);
-      if (ki > bk) {
-        bk = ki;
-        bi = i * 32 + lane;
+      if (key[i] > bk) {
+        bk = key[i];
+        bi = i;
       }
     }
     const uint32_t wk = __reduce_max_sync(0xffffffffu, bk);
-    const int wi = (int)__reduce_min_sync(0xffffffffu, (bk == wk && wk != key_neg_inf) ? (uint32_t)bi : 0x7fffffffu);
     const bool none = wk == key_neg_inf;
+    const int wi = (int)__reduce_min_sync(0xffffffffu, (bk == wk && !none) ? (uint32_t)(bi * 32 + lane) : 0x7fffffffu);
     const float bv = none ? kNegInf : key_float(wk);
     if (j == 0) r.top = bv;
     if (j < k) {
@@ -65,7 +69,7 @@ __device__ __forceinline__ TopkResult warp_topk(float (&v)[kMaxPerLane], int k, 
       if (!none && (wi & 31) == lane) {
 #pragma unroll
         for (int i = 0; i < kMaxPerLane; ++i)
-          if (i == (wi >> 5)) v[i] = kNegInf;
+          if (i == (wi >> 5)) key[i] = key_neg_inf;
       }
     } else {
       r.margin = none ? __builtin_huge_valf() : last - bv;
