@@ -165,6 +165,7 @@ def main():
     import torch
     import torch.distributed as dist
     from paper_2602_08404_b200 import binding as B
+    from paper_2602_08404_b200 import replicas as R_
     from paper_2602_08404_b200 import build as build_mod
     from paper_2602_08404_b200 import workloads as W
 
@@ -281,10 +282,7 @@ def main():
         barrier()
         ms = e0.elapsed_time(e1)
         ms_per_step = ms / issued
-        if world > 1:
-            t = torch.tensor([ms_per_step], device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms_per_step = float(t.item())
+        ms_per_step = R_.max_over_ranks(ms_per_step, dev)
 
         # ---- expert-kernel duration (CUDA events around every launch, on the launching stream) -------
         for c in ctxs:
@@ -331,10 +329,7 @@ def main():
             e2e_step(i)
         barrier()
         e2e_ms_per_step = (time.perf_counter() - t0) * 1e3 / n_e2e
-        if world > 1:
-            t = torch.tensor([e2e_ms_per_step], device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            e2e_ms_per_step = float(t.item())
+        e2e_ms_per_step = R_.max_over_ranks(e2e_ms_per_step, dev)
     clocks = sampler.summary()
 
     # ---- accounting ------------------------------------------------------------------------------
@@ -343,7 +338,7 @@ def main():
     algo_bytes = mean_act * bytes_per_expert                      # activated-expert weight bytes per launch
     peak, peak_kind = measured_peaks()
     achieved = algo_bytes / (kernel_ms * 1e-3) / 1e9
-    value = world * T / (ms_per_step * 1e-3)
+    value = R_.whole_job_rate(T, ms_per_step)
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
@@ -354,11 +349,11 @@ def main():
                    "l2": f"inputs larger than L2: weights rotate over {R} layers ({R * E * bytes_per_expert / 1e9:.1f} GB)",
                    "cuda_graph": graph is not None, "steps_issued": issued, "parallelism": f"replicas x{world}"},
         "clocks": clocks,
-        "e2e": {"value": world * T / (e2e_ms_per_step * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+        "e2e": {"value": R_.whole_job_rate(T, e2e_ms_per_step), "unit": UNIT, "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms_per_step, "steps": n_e2e},
         "gpu_launches": launches_per_step * issued,
-        "activated_experts_per_s": world * mean_act / (ms_per_step * 1e-3),
-        "rows_computed_per_s": world * mean_rows / (ms_per_step * 1e-3),
+        "activated_experts_per_s": R_.whole_job_rate(mean_act, ms_per_step),
+        "rows_computed_per_s": R_.whole_job_rate(mean_rows, ms_per_step),
         "step_hbm_frac": (algo_bytes + 4 * E * H) / (ms_per_step * 1e-3) / 1e9 / peak,
         "roofline": {"bound": "hbm", "kernel": "k_experts_stream", "achieved": achieved, "peak": peak,
                      "peak_kind": f"of {peak_kind}", "unit": "GB/s", "frac": achieved / peak,

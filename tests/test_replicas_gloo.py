@@ -1,0 +1,67 @@
+"""The N > 1 path of the measurement on CPU: two gloo ranks, no GPU.
+
+The hot path does not shard: N GPUs run N independent replicas, and the only collective work is the
+barrier and the maximum over the ranks' times.  The test runs that bookkeeping with world_size 2 and
+checks the whole-job rate against the definition (units of all ranks / slowest rank's time); it also
+checks that the reference arm stays silent on ranks other than 0.
+"""
+import json
+import os
+import subprocess
+import sys
+
+import torch
+import torch.distributed as dist
+import torch.multiprocessing as mp
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _worker(rank, world, port, out):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    sys.path.insert(0, ROOT)
+    from paper_2602_08404_b200 import replicas as R
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        R.barrier()
+        local_ms = 0.040 + 0.010 * rank              # rank 1 is the slow one
+        ms = R.max_over_ranks(local_ms)
+        rate = R.whole_job_rate(4, ms)               # 4 rows per rank and step
+        out.put((rank, R.world_size(), ms, rate))
+        R.barrier()
+    finally:
+        dist.destroy_process_group()
+
+
+def test_two_replicas_rate_is_all_units_over_the_slowest_time():
+    ctx = mp.get_context("spawn")
+    out = ctx.Queue()
+    port = 29500 + os.getpid() % 2000
+    procs = [ctx.Process(target=_worker, args=(r, 2, port, out)) for r in range(2)]
+    for p in procs:
+        p.start()
+    got = sorted(out.get(timeout=120) for _ in procs)
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    for rank, world, ms, rate in got:
+        assert world == 2
+        assert abs(ms - 0.050) < 1e-12                            # the maximum, on every rank
+        assert abs(rate - 2 * 4 / 0.050e-3) < 1e-6                # 8 rows per step over 50 us
+
+
+def test_single_process_needs_no_process_group():
+    sys.path.insert(0, ROOT)
+    from paper_2602_08404_b200 import replicas as R
+    assert R.world_size() == 1
+    assert R.max_over_ranks(0.25) == 0.25
+    assert R.whole_job_rate(4, 0.04) == 4 / 0.04e-3
+    R.barrier()
+
+
+def test_reference_arm_prints_nothing_on_other_ranks():
+    env = dict(os.environ, RANK="1", WORLD_SIZE="2", LOCAL_RANK="1", MASTER_ADDR="127.0.0.1", MASTER_PORT="29999")
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--steps", "2", "--warmup", "1"],
+                       env=env, capture_output=True, text=True, timeout=300)
+    assert r.returncode == 0
+    assert r.stdout.strip() == ""
