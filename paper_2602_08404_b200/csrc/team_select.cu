@@ -222,14 +222,14 @@ k_select(const float* __restrict__ logits, StepPtrs st, Workspace ws, RoutePtrs 
   }
   const int32_t* idx_src = s.idx ? s.idx : r.topk_idx;
 
-  // ---- exports that need no further work ---------------------------------------------------
-  for (int t = tid; t < T; t += kSelThreads) {
+  // ---- exports that need no further work: by the upper half of the CTA, beside the dispatch below ----
+  for (int t = tid - kSelThreads / 2; t >= 0 && t < T; t += kSelThreads / 2) {
     r.tok_class[t] = s.cls[t];
     if (ex.tok_class) ex.tok_class[t] = s.cls[t];
   }
   {
     const int n_words64 = (E + 63) / 64;
-    for (int i = tid; i < d.G * n_words64; i += kSelThreads) {
+    for (int i = tid - kSelThreads / 2; i >= 0 && i < d.G * n_words64; i += kSelThreads / 2) {
       const int g = i / n_words64, wd = i % n_words64;
       const uint64_t m = (uint64_t)s.mask[g * n_words32 + 2 * wd] | ((uint64_t)s.mask[g * n_words32 + 2 * wd + 1] << 32);
       r.group_mask[i] = m;
@@ -257,7 +257,11 @@ k_select(const float* __restrict__ logits, StepPtrs st, Workspace ws, RoutePtrs 
     }
   }
   // number of computed rows; shared experts take every one of them
-  {
+  int n_rows_active = 0;
+  if (T <= 32) {
+    // every warp counts for itself: nothing to exchange
+    n_rows_active = __popc(__ballot_sync(0xffffffffu, lane < T && s.cls[lane] != TEAM_CLS_SKIP));
+  } else {
     int c = 0;
     for (int base = warp * 32; base < T; base += kSelThreads) {
       const int t = base + lane;
@@ -266,9 +270,8 @@ k_select(const float* __restrict__ logits, StepPtrs st, Workspace ws, RoutePtrs 
     }
     if (lane == 0) s.warp_cnt[warp] = c;
   }
-  __syncthreads();
-  int n_rows_active = 0;
-  {
+  if (!small || T > 32) __syncthreads();      // per-warp histograms and row counts are complete
+  if (T > 32) {
     const int used = min(kSelWarps, (T + 31) / 32);
     for (int w = 0; w < used; ++w) n_rows_active += s.warp_cnt[w];
   }
@@ -276,11 +279,27 @@ k_select(const float* __restrict__ logits, StepPtrs st, Workspace ws, RoutePtrs 
   const int nwe = (EN + 31) / 32;            // EN <= 260: at most 9 warps, expert e = tid
   int c = 0, tiles = 0, incl_c = 0, incl_t = 0, arank = 0;
   unsigned act_b = 0;
+  uint32_t mine[kSmallSlots / 32] = {};
   if (warp < nwe) {
     const int e = tid;
     if (e < E) {
       if (small) {
-        for (int i = 0; i < S; ++i) c += (s.idx[i] == e);
+        // which of the (at most kSmallSlots) slots chose this expert: one bit per slot
+#pragma unroll
+        for (int q = 0; q < kSmallSlots / 32; ++q) {
+          if (q * 32 < S) {
+#pragma unroll
+            for (int i = 0; i < 32; i += 4) {
+              const int at = q * 32 + i;
+              if (at < S) {
+                const int4 v = *reinterpret_cast<const int4*>(s.idx + at);      // the array is padded to 16 bytes
+                mine[q] |= (uint32_t)(v.x == e) << i | (uint32_t)(v.y == e && at + 1 < S) << (i + 1) |
+                           (uint32_t)(v.z == e && at + 2 < S) << (i + 2) | (uint32_t)(v.w == e && at + 3 < S) << (i + 3);
+              }
+            }
+            c += __popc(mine[q]);
+          }
+        }
       } else {
         // turn per-warp counts into per-warp starting ranks
         for (int w = 0; w < nw; ++w) {
@@ -345,10 +364,12 @@ k_select(const float* __restrict__ logits, StepPtrs st, Workspace ws, RoutePtrs 
           // place this expert's slots: routed ones by ascending slot id, a shared expert's by ascending row
           int at = excl;
           if (e < E) {
-            for (int i = 0; i < S; ++i) {
-              if (s.idx[i] == e) {
-                r.perm[at] = i;
-                if (ex.perm) ex.perm[at] = i;
+#pragma unroll
+            for (int q = 0; q < kSmallSlots / 32; ++q) {
+              for (uint32_t m = mine[q]; m != 0; m &= m - 1) {
+                const int slot = q * 32 + __ffs(m) - 1;
+                r.perm[at] = slot;
+                if (ex.perm) ex.perm[at] = slot;
                 ++at;
               }
             }
