@@ -51,8 +51,15 @@ struct StArgs {
 };
 
 __device__ __forceinline__ uint32_t st_smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ void st_cp16(uint32_t dst, const void* src) {
-  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+// Weights are read once per step: they are marked evict-first in L2 so that streaming them does not push out
+// what the step's small kernels reuse from one step to the next (router weights, tables, code).
+__device__ __forceinline__ uint64_t st_stream_policy() {
+  uint64_t pol;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+  return pol;
+}
+__device__ __forceinline__ void st_cp16(uint32_t dst, const void* src, uint64_t pol) {
+  asm volatile("cp.async.cg.shared.global.L2::cache_hint [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "l"(pol) : "memory");
 }
 __device__ __forceinline__ void st_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int N>
@@ -135,6 +142,7 @@ __global__ void __launch_bounds__(kStThreads, 1) k_experts_stream(StArgs a) {
   const uint32_t xs_lane = st_smem_u32(xs) + (uint32_t)b_tok * H * 2;
   const int tile = warp & 1, ks = warp >> 1;     // phase 1: this warp's 16-row tile (gate | up) and hidden slice
   const __nv_bfloat16* wmat = tile ? a.w_up : a.w_gate;
+  const uint64_t pol = st_stream_policy();
 
   for (int s_lo = g_lo, s_hi; s_lo < g_hi; s_lo = s_hi) {
     s_hi = min(g_hi, s_lo + kStPassGroups);
@@ -159,10 +167,10 @@ __global__ void __launch_bounds__(kStThreads, 1) k_experts_stream(StArgs a) {
           i_src = wmat + ((size_t)e * I + gi * 16 + cp_row) * H + ks * KS + cp_piece * 8;
         }
         const __nv_bfloat16* p = i_src + icc * 64;
-        st_cp16(dst + cp_off0, p);
-        st_cp16(dst + cp_off1, p + 4 * (size_t)H);
-        st_cp16(dst + cp_off0 + 1024, p + 8 * (size_t)H);
-        st_cp16(dst + cp_off1 + 1024, p + 12 * (size_t)H);
+        st_cp16(dst + cp_off0, p, pol);
+        st_cp16(dst + cp_off1, p + 4 * (size_t)H, pol);
+        st_cp16(dst + cp_off0 + 1024, p + 8 * (size_t)H, pol);
+        st_cp16(dst + cp_off1 + 1024, p + 12 * (size_t)H, pol);
         if (++icc == NCH) {
           icc = 0;
           if (++iq == ng) iq = 0;      // phase 2 walks the groups again
@@ -173,10 +181,10 @@ __global__ void __launch_bounds__(kStThreads, 1) k_experts_stream(StArgs a) {
           i_src = a.w_down + (((size_t)e * NG + gi) * H + warp * HW) * 16 + lane * 8;
         }
         const __nv_bfloat16* p = i_src + icc * 1024;
-        st_cp16(dst + cq_off, p);
-        st_cp16(dst + cq_off + 512, p + 256);
-        st_cp16(dst + cq_off + 1024, p + 512);
-        st_cp16(dst + cq_off + 1536, p + 768);
+        st_cp16(dst + cq_off, p, pol);
+        st_cp16(dst + cq_off + 512, p + 256, pol);
+        st_cp16(dst + cq_off + 1024, p + 512, pol);
+        st_cp16(dst + cq_off + 1536, p + 768, pol);
         if (++icc == CPG) {
           icc = 0;
           ++iq;
