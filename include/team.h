@@ -214,6 +214,22 @@ int team_select_experts(team_ctx *ctx, const team_step_state *st, team_routing *
 int team_moe_forward(team_ctx *ctx, const void *x, const team_step_state *st, team_routing *out,
                      float *y, void *stream);
 
+/* The same layer step for callers whose buffers live in HOST memory (pageable
+ * or pinned): x_host [T, H] in the config's dtype, the five arrays of st_host
+ * as host pointers, y_host fp32 [T, H].  The call packs the inputs into a pinned
+ * staging block owned by the context, moves them to the device with one copy,
+ * runs team_moe_forward on `stream`, copies y back and synchronises the stream
+ * before it returns, so y_host is valid on return.  Rows with class
+ * TEAM_CLS_SKIP receive what the previous call on this context left in the
+ * context's device-side y (zero before the first call): use one context per
+ * layer to get "the previous step's output" there.  `out`, if given, holds
+ * DEVICE pointers as in team_moe_forward.  The first call on a context allocates
+ * the staging block (device and pinned host, (6 H + 17) bytes per row of
+ * max_rows for bf16); team_destroy frees it.  Not reentrant per context.
+ * Errors: as team_moe_forward. */
+int team_moe_forward_host(team_ctx *ctx, const void *x_host, const team_step_state *st_host,
+                          team_routing *out, float *y_host, void *stream);
+
 /* Stack glue for a MoE-only multi-layer model: x[t,:] <- x[t,:] + y[t,:] for
  * every row computed by the preceding team_moe_forward (fp32 add, stored in
  * x's dtype, round to nearest even). */

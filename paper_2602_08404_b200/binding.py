@@ -23,7 +23,7 @@ TEAM_F_DCD, TEAM_F_LAC = 1, 2
 TEAM_DTYPE_F32, TEAM_DTYPE_BF16 = 0, 1
 
 EXPORTS = ["team_create", "team_destroy", "team_set_weights", "team_set_policy", "team_route",
-           "team_route_static", "team_pack_w_down", "team_select_experts", "team_moe_forward", "team_residual_add", "team_read_status",
+           "team_route_static", "team_pack_w_down", "team_select_experts", "team_moe_forward", "team_moe_forward_host", "team_residual_add", "team_read_status",
            "team_last_launch_count", "team_expert_timing", "team_debug_force_simt", "team_strerror",
            "team_last_cuda_error", "team_version"]
 
@@ -73,6 +73,7 @@ def lib():
                                         ctypes.POINTER(team_routing), vp]
         L.team_select_experts.argtypes = [vp, ctypes.POINTER(team_step_state), ctypes.POINTER(team_routing), vp]
         L.team_moe_forward.argtypes = [vp, vp, ctypes.POINTER(team_step_state), ctypes.POINTER(team_routing), vp, vp]
+        L.team_moe_forward_host.argtypes = [vp, vp, ctypes.POINTER(team_step_state), ctypes.POINTER(team_routing), vp, vp]
         L.team_residual_add.argtypes = [vp, vp, vp, i32, vp]
         L.team_read_status.argtypes = [vp, vp, ctypes.POINTER(i32)]
         L.team_last_launch_count.argtypes = [vp]
@@ -184,6 +185,21 @@ def team_moe_forward(ctx, x, st, out, y):
     r = _routing(out)
     _check(lib().team_moe_forward(ctx, _ptr(x), ctypes.byref(_state(st)), ctypes.byref(r) if r is not None else None, _ptr(y),
                                   _stream()), ctx)
+
+
+def _hptr(t):
+    if t.is_cuda or not t.is_contiguous():
+        raise TeamError("expected a contiguous CPU tensor")
+    return ctypes.c_void_p(t.data_ptr())
+
+
+def team_moe_forward_host(ctx, x_host, st_host, out, y_host):
+    """x_host, the step state and y_host are CPU tensors; `out` (optional) holds device tensors. Blocks until y_host is filled."""
+    st = team_step_state(int(st_host["tok_state"].shape[0]), _hptr(st_host["tok_state"]), _hptr(st_host["conf"]),
+                         _hptr(st_host["pos"]), _hptr(st_host["group"]), _hptr(st_host["branch"]))
+    r = _routing(out)
+    _check(lib().team_moe_forward_host(ctx, _hptr(x_host), ctypes.byref(st), ctypes.byref(r) if r is not None else None,
+                                       _hptr(y_host), _stream()), ctx)
 
 
 def team_residual_add(ctx, x, y, n_rows):

@@ -26,6 +26,10 @@ struct team_ctx {
   int force_simt;
   bool stream_path;   // few rows: the weight-streaming expert kernel instead of the tensor-memory one
   void* simt_act;   // diagnostic fp32-FMA path on bf16 weights: activation scratch
+  // team_moe_forward_host: one device block and its pinned host mirror, [inputs | y]
+  unsigned char* hs_dev;
+  unsigned char* hs_pin;
+  size_t hs_in_bytes, hs_y_off, hs_bytes;
   char cuda_err[256];
   // expert-kernel timing
   bool timing;
@@ -137,6 +141,8 @@ int team_create(const team_config* cfg, team_ctx** out) {
   ctx->last_launches = 0;
   ctx->force_simt = 0;
   ctx->simt_act = nullptr;
+  ctx->hs_dev = nullptr;
+  ctx->hs_pin = nullptr;
   ctx->cuda_err[0] = 0;
   ctx->timing = false;
   ctx->ev_used = 0;
@@ -214,6 +220,8 @@ int team_destroy(team_ctx* ctx) {
   for (cudaEvent_t e : ctx->ev) cudaEventDestroy(e);
   cudaFree(ctx->ws_base);
   if (ctx->simt_act) cudaFree(ctx->simt_act);
+  if (ctx->hs_dev) cudaFree(ctx->hs_dev);
+  if (ctx->hs_pin) cudaFreeHost(ctx->hs_pin);
   delete ctx;
   return TEAM_OK;
 }
@@ -329,6 +337,60 @@ int team_moe_forward(team_ctx* ctx, const void* x, const team_step_state* st, te
     ctx->last_launches += 2;
   }
   if (ev1) cudaEventRecord(ev1, s);
+  return TEAM_OK;
+}
+
+int team_moe_forward_host(team_ctx* ctx, const void* x_host, const team_step_state* st_host, team_routing* out,
+                          float* y_host, void* stream) {
+  int rc = check_state(ctx, st_host);
+  if (rc != TEAM_OK) return rc;
+  if (x_host == nullptr || y_host == nullptr || !ctx->has_weights) return TEAM_ERR_ARG;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const size_t Tm = ctx->cfg.max_rows, H = ctx->cfg.hidden, elt = ctx->cfg.dtype == TEAM_DTYPE_F32 ? 4 : 2;
+  auto up = [](size_t v) { return (v + 255) & ~size_t(255); };
+  // layout of the staging block (sized for max_rows): x | tok_state | conf | pos | group | branch | y
+  const size_t o_x = 0, o_ts = up(Tm * H * elt), o_conf = o_ts + up(Tm), o_pos = o_conf + up(Tm * 4),
+               o_grp = o_pos + up(Tm * 4), o_br = o_grp + up(Tm * 4), o_y = o_br + up(Tm * 4);
+  if (ctx->hs_dev == nullptr) {
+    ctx->hs_in_bytes = o_y;
+    ctx->hs_y_off = o_y;
+    ctx->hs_bytes = o_y + up(Tm * H * 4);
+    cudaError_t e = cudaMalloc(reinterpret_cast<void**>(&ctx->hs_dev), ctx->hs_bytes);
+    if (e == cudaSuccess) e = cudaMemsetAsync(ctx->hs_dev, 0, ctx->hs_bytes, s);
+    if (e == cudaSuccess) e = cudaMallocHost(reinterpret_cast<void**>(&ctx->hs_pin), ctx->hs_bytes);
+    if (e != cudaSuccess) {
+      if (ctx->hs_dev) cudaFree(ctx->hs_dev);
+      ctx->hs_dev = nullptr;
+      return fail_cuda(ctx, e, "host staging");
+    }
+    memset(ctx->hs_pin, 0, ctx->hs_bytes);
+  }
+  const size_t T = st_host->n_rows;
+  unsigned char* hp = ctx->hs_pin;
+  memcpy(hp + o_x, x_host, T * H * elt);
+  memcpy(hp + o_ts, st_host->tok_state, T);
+  memcpy(hp + o_conf, st_host->conf, T * 4);
+  memcpy(hp + o_pos, st_host->pos, T * 4);
+  memcpy(hp + o_grp, st_host->group, T * 4);
+  memcpy(hp + o_br, st_host->branch, T * 4);
+  // one copy in: with few rows the block is small and a single transfer beats six
+  const size_t in_bytes = ctx->hs_in_bytes;
+  cudaError_t e = cudaMemcpyAsync(ctx->hs_dev, hp, in_bytes, cudaMemcpyHostToDevice, s);
+  if (e != cudaSuccess) return fail_cuda(ctx, e, "copy in");
+  unsigned char* dp = ctx->hs_dev;
+  team_step_state st = *st_host;
+  st.tok_state = dp + o_ts;
+  st.conf = reinterpret_cast<const float*>(dp + o_conf);
+  st.pos = reinterpret_cast<const int32_t*>(dp + o_pos);
+  st.group = reinterpret_cast<const int32_t*>(dp + o_grp);
+  st.branch = reinterpret_cast<const int32_t*>(dp + o_br);
+  float* y_dev = reinterpret_cast<float*>(dp + ctx->hs_y_off);
+  rc = team_moe_forward(ctx, dp + o_x, &st, out, y_dev, stream);
+  if (rc != TEAM_OK) return rc;
+  e = cudaMemcpyAsync(hp + ctx->hs_y_off, y_dev, T * H * 4, cudaMemcpyDeviceToHost, s);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+  if (e != cudaSuccess) return fail_cuda(ctx, e, "copy out");
+  memcpy(y_host, hp + ctx->hs_y_off, T * H * 4);
   return TEAM_OK;
 }
 

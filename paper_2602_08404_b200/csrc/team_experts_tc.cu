@@ -136,6 +136,16 @@ __device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, vo
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
 }
+// Weight copies: read once per step, so marked evict-first in L2 (the step's small kernels keep their
+// working set there: router weights, tables, code).
+__device__ __forceinline__ uint64_t stream_policy() {
+  uint64_t pol;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+  return pol;
+}
+__device__ __forceinline__ void cp_async16_stream(uint32_t dst, const void* src, uint64_t pol) {
+  asm volatile("cp.async.cg.shared.global.L2::cache_hint [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "l"(pol) : "memory");
+}
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 __device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
 // The barrier receives one arrival from this thread once all of its earlier cp.async copies have landed.
@@ -539,6 +549,7 @@ k_experts_tc(TcArgs a) {
     const uint32_t dst1 = (uint32_t)rr0 * 128u + (uint32_t)((ch ^ (rr0 & 7)) << 4);   // (RSTEP is a multiple of 8: same swizzle)
     // phase 2: W_down is stored in slabs of 16 columns ([I/16][H][16]); a window's 128-byte tile row is
     // gathered from four slabs.  Per instruction a warp copies 4 rows x 32 bytes from each of them.
+    const uint64_t pol = stream_policy();
     const int r_first = warp * 4 + ((lane & 7) >> 1);
     const int ch2 = (lane >> 3) * 2 + (lane & 1);                                     // 16-byte piece of the tile row
     const uint32_t dst2 = sw128(r_first, ch2);
@@ -597,7 +608,7 @@ k_experts_tc(TcArgs a) {
               for (int m = 0; m < 2; ++m) {
 #pragma unroll
                 for (int ii = 0; ii < 16 / RSTEP; ++ii)
-                  cp_async16(dstA + (uint32_t)(((q * 2 + m) * 16 + ii * RSTEP) * 128), src1[q][m] + koff + ii * rstep1);
+                  cp_async16_stream(dstA + (uint32_t)(((q * 2 + m) * 16 + ii * RSTEP) * 128), src1[q][m] + koff + ii * rstep1, pol);
               }
             }
           }
@@ -615,7 +626,7 @@ k_experts_tc(TcArgs a) {
           const uint32_t dstA = base + i * kATileBytes + dst2;
 #pragma unroll
           for (int ii = 0; ii < 128 / (4 * kLoaders); ++ii)
-            cp_async16(dstA + (uint32_t)(ii * 4 * kLoaders) * 128u, src2 + ii * rstep2);
+            cp_async16_stream(dstA + (uint32_t)(ii * 4 * kLoaders) * 128u, src2 + ii * rstep2, pol);
         }
       }
       cp_async_arrive(smem_u32(bar_full + st.it % NB));     // the stage is handed over when this lane's copies land

@@ -152,3 +152,30 @@ def test_c5_stack_small_shape(flags, weights_cache):
 
 def test_c5_stack_sdar_shape_two_layers(weights_cache):
     _run_stack(W.C2, 2, 3, weights_cache)
+
+
+def test_host_buffer_entry_point_matches_device_entry_point(weights_cache):
+    """team_moe_forward_host on a whole schedule: same y as team_moe_forward, skipped rows keeping the previous step's."""
+    shape, flags = W.C2, 3
+    steps = W.make_schedule(shape)
+    layer_a, layer_b = P.Layer(shape, weights_cache(shape), flags), P.Layer(shape, weights_cache(shape), flags)
+    try:
+        T, H = shape.rows, shape.hidden
+        y_dev = torch.zeros((T, H), dtype=torch.float32, device="cuda")
+        y_host = torch.full((T, H), 7.0, dtype=torch.float32)
+        for step in steps:
+            x_host = torch.as_tensor(step["x"]).to(torch.bfloat16)
+            st_host = {"tok_state": torch.as_tensor(step["tok_state"].astype(np.uint8)),
+                       "conf": torch.as_tensor(step["conf"].astype(np.float32)),
+                       "pos": torch.as_tensor(step["pos"].astype(np.int32)),
+                       "group": torch.as_tensor(step["group"].astype(np.int32)),
+                       "branch": torch.as_tensor(step["branch"].astype(np.int32))}
+            B.team_moe_forward(layer_a.ctx, x_host.cuda(), B.state_to_device(step), None, y_dev)
+            B.team_moe_forward_host(layer_b.ctx, x_host, st_host, None, y_host)
+            ref = y_dev.cpu()
+            # fp32 reductions arrive in a different order from launch to launch: equal to rounding of the sums
+            assert torch.allclose(y_host, ref, rtol=0, atol=1e-5 * float(ref.abs().max()))
+        assert B.team_read_status(layer_b.ctx)[0] == 0
+    finally:
+        layer_a.close()
+        layer_b.close()
