@@ -45,6 +45,9 @@ def parse_args():
     ap.add_argument("--flags", type=int, default=TEAM_FLAGS, help="0 vanilla, 1 DCD, 3 DCD|LAC")
     ap.add_argument("--no-graph", action="store_true", help="issue every step as separate calls (no CUDA graph)")
     ap.add_argument("--cpu-seconds", type=float, default=15.0, help="budget of the oracle baseline leg")
+    ap.add_argument("--workload", default="c2", choices=["c2", "c3", "c4"],
+                    help="c2: the headline step (default); c3: 256 experts + shared, block 32; c4: c2 shape, --seqs x 4 branches x 4")
+    ap.add_argument("--seqs", type=int, default=1, help="sequences of the c4 batch sweep")
     return ap.parse_args()
 
 
@@ -183,9 +186,13 @@ def main():
         dist.barrier()
     dev = torch.device("cuda", local_rank)
 
-    shape = W.C2
+    shape = {"c2": W.C2, "c3": W.C3, "c4": W.c4(args.seqs)}[args.workload]
     T, H, E, k, I = shape.rows, shape.hidden, shape.n_experts, shape.top_k, shape.inter
-    steps_host = W.make_schedule(shape)                      # 4 denoising steps, seeded
+    ns = shape.n_shared
+    workload = WORKLOAD if args.workload == "c2" else (
+        f"{shape.name}: H{H} E{E}{'+%d shared' % ns if ns else ''} top{k} I{I} bf16, {shape.seqs} seq x {shape.branches} "
+        f"branches x block {shape.block} = {T} rows, {shape.n_steps} denoising steps, flags {args.flags}")
+    steps_host = W.make_schedule(shape)                      # the scripted denoising steps, seeded
     n_sched = len(steps_host)
     R = args.layers
 
@@ -196,10 +203,10 @@ def main():
         gen.manual_seed(1000 + r)
         wr = (torch.randn((E, H), generator=gen, device=dev, dtype=torch.float32) * 0.02).contiguous()
         wg, wu, wd = [(torch.randn(s, generator=gen, device=dev, dtype=torch.float32) * 0.02).to(torch.bfloat16)
-                      for s in ((E, I, H), (E, I, H), (E, H, I))]
+                      for s in ((E + ns, I, H), (E + ns, I, H), (E + ns, H, I))]
         layers.append((wr, wg, wu, wd if r == 0 else None))
         packed.append(B.team_pack_w_down(wd))      # the layout the library reads; row-major kept for the oracle leg
-    cfg = B.make_config(H, E, k, I, 0, max_rows=T, max_groups=1, dtype=B.TEAM_DTYPE_BF16, flags=args.flags,
+    cfg = B.make_config(H, E, k, I, ns, max_rows=T, max_groups=shape.seqs, dtype=B.TEAM_DTYPE_BF16, flags=args.flags,
                         tau_hot=shape.tau_hot, L_hot=shape.L_hot)
     ctxs = []
     for r in range(R):
@@ -335,12 +342,13 @@ def main():
     peak, peak_kind = measured_peaks()
     achieved = algo_bytes / (kernel_ms * 1e-3) / 1e9
     value = R_.whole_job_rate(T, ms_per_step)
+    stream_kernel = T <= 8 and H in (1024, 2048)
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": WORKLOAD, "flags": args.flags, "rows_presented": T, "rows_computed_mean": mean_rows,
+        "config": {"workload": workload, "flags": args.flags, "rows_presented": T, "rows_computed_mean": mean_rows,
                    "activated_experts_mean": mean_act, "layers_cycled": R,
                    "l2": f"inputs larger than L2: weights rotate over {R} layers ({R * E * bytes_per_expert / 1e9:.1f} GB)",
                    "cuda_graph": graph is not None, "steps_issued": issued, "parallelism": f"replicas x{world}"},
@@ -351,13 +359,15 @@ def main():
         "activated_experts_per_s": R_.whole_job_rate(mean_act, ms_per_step),
         "rows_computed_per_s": R_.whole_job_rate(mean_rows, ms_per_step),
         "step_hbm_frac": (algo_bytes + 4 * E * H) / (ms_per_step * 1e-3) / 1e9 / peak,
-        "roofline": {"bound": "hbm", "kernel": "k_experts_stream", "achieved": achieved, "peak": peak,
+        "roofline": {"bound": "hbm", "kernel": "k_experts_stream" if stream_kernel else "k_experts_tc", "achieved": achieved, "peak": peak,
                      "peak_kind": f"of {peak_kind}", "unit": "GB/s", "frac": achieved / peak,
                      "frac_of_8TBs_nominal": achieved / 8000.0, "kernel_ms": kernel_ms,
                      "algorithmic_bytes_per_launch": algo_bytes, "launches_timed": tot_n,
                      # DRAM read + write bytes per launch: ncu capture at 16 activated experts (151.06 MB read +
                      # 3.6 MB written, profiles/experts_stream_c2_bench.md), scaled to this run's mean
-                     "traffic": mean_act * (151.06e6 + 3.6e6) / 16.0 if (H, I) == (2048, 768) else None},
+                     "traffic": mean_act * (151.06e6 + 3.6e6) / 16.0 if args.workload == "c2" else None,
+                     # the same launches as a contraction: 6 H I flops per token-slot (routed and shared)
+                     "tensor_tflops": mean_rows * (k + ns) * 6.0 * H * I / (kernel_ms * 1e-3) / 1e12},
     }
 
     if rank == 0:
