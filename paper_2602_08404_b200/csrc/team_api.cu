@@ -153,11 +153,13 @@ int team_create(const team_config* cfg, team_ctx** out) {
     return TEAM_ERR_CUDA;
   }
   ctx->item_tile = pick_item_tile(*cfg);
+  ctx->stream_path = cfg->dtype == TEAM_DTYPE_BF16 && team::experts_stream_supported(cfg->max_rows, cfg->hidden, cfg->inter);
+  // the few-rows kernel's gather mode takes work items of 8 token-slots
+  if (ctx->stream_path && team::experts_stream_gathers(cfg->max_rows)) ctx->item_tile = team::experts_stream_item_tile();
   e = team::configure_router(cfg->dtype, cfg->hidden);
   if (e == cudaSuccess) e = team::configure_select(dims_of(*cfg, cfg->max_rows));
-  ctx->stream_path = cfg->dtype == TEAM_DTYPE_BF16 && team::experts_stream_supported(cfg->max_rows, cfg->hidden, cfg->inter);
-  if (e == cudaSuccess && cfg->dtype == TEAM_DTYPE_BF16) e = team::configure_experts_tc(ctx->item_tile);
-  if (e == cudaSuccess && ctx->stream_path) e = team::configure_experts_stream(cfg->hidden);
+  if (e == cudaSuccess && cfg->dtype == TEAM_DTYPE_BF16 && !ctx->stream_path) e = team::configure_experts_tc(ctx->item_tile);
+  if (e == cudaSuccess && ctx->stream_path) e = team::configure_experts_stream(cfg->hidden, cfg->max_rows);
   if (e != cudaSuccess) {
     delete ctx;
     return TEAM_ERR_CUDA;
@@ -174,7 +176,7 @@ int team_create(const team_config* cfg, team_ctx** out) {
   const size_t o_logits = take(T * E * 4), o_idx = take(T * k * 4), o_w = take(T * k * 4), o_margin = take(T * 4);
   const size_t o_cls = take(T), o_gm = take((size_t)cfg->max_groups * ((E + 63) / 64) * 8);
   const size_t o_cnt = take(EN * 4), o_off = take((EN + 1) * 4), o_perm = take(S * 4), o_act_list = take(EN * 4);
-  const size_t o_scal = take(64), o_items = take((EN + S / 16 + 2) * sizeof(team::WorkItem));
+  const size_t o_scal = take(64), o_items = take((EN + S / 8 + 2) * sizeof(team::WorkItem));
   const size_t o_act = take(cfg->dtype == TEAM_DTYPE_F32 ? S * cfg->inter * 4 : 256);
   const bool bf16 = cfg->dtype == TEAM_DTYPE_BF16;
   const size_t max_items = EN + S / ctx->item_tile + 2;
@@ -326,7 +328,8 @@ int team_moe_forward(team_ctx* ctx, const void* x, const team_step_state* st, te
   }
   if (tc) {
     if (ctx->stream_path)
-      e = team::launch_experts_stream(x, ctx->w.w_gate, ctx->w.w_up, ctx->w.w_down, ctx->ws, y, d, ctx->n_sms, s);
+      e = team::launch_experts_stream(x, ctx->w.w_gate, ctx->w.w_up, ctx->w.w_down, ctx->ws, y, d, ctx->cfg.max_rows,
+                                      ctx->n_sms, s);
     else
       e = team::launch_experts_tc(ctx->item_tile, x, ctx->w.w_gate, ctx->w.w_up, ctx->w.w_down, ctx->ws, y, d, ctx->n_sms, s);
     if (e != cudaSuccess) return fail_cuda(ctx, e, "expert kernel");

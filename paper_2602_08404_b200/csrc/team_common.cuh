@@ -99,9 +99,11 @@ cudaError_t configure_select(Dims max_dims);
 cudaError_t configure_experts_tc(int item_tile);
 int experts_tc_item_tile(int max_rows);
 bool experts_stream_supported(int max_rows, int hidden, int inter);
-cudaError_t configure_experts_stream(int hidden);
+bool experts_stream_gathers(int max_rows);
+int experts_stream_item_tile();
+cudaError_t configure_experts_stream(int hidden, int max_rows);
 cudaError_t launch_experts_stream(const void* x, const void* w_gate, const void* w_up, const void* w_down, Workspace ws,
-                                  float* y, Dims d, int grid, cudaStream_t s);
+                                  float* y, Dims d, int max_rows, int grid, cudaStream_t s);
 cudaError_t launch_router_logits(const void* x, int dtype, const float* w_router, const uint8_t* tok_state,
                                  float* logits, float* y_zero, Dims d, int flags, cudaStream_t s);
 cudaError_t launch_router_topk(const float* logits, const uint8_t* tok_state, RoutePtrs out, Dims d, Policy p,

@@ -91,13 +91,19 @@ __host__ __device__ inline size_t stream_smem_bytes(int H) {
   return (size_t)kStRows * H * 2 + kStRedBytes + (size_t)kStWarps * kStSlots * kStChunkBytes;
 }
 
-// CPG: 64-row chunks of a W_down slab per warp and group (H = CPG * 1024)
-template <int CPG>
+// CPG: 64-row chunks of a W_down slab per warp and group (H = CPG * 1024).
+// GATHER = false: the call has at most 8 rows; all of them are the mma's token columns for every expert, and a
+//                 row that did not choose the expert gets weight 0.
+// GATHER = true:  any number of rows; work items of at most 8 token-slots of one expert (built by the selection
+//                 kernel); a pass stays inside one item and the item's rows are gathered into shared memory.
+template <int CPG, bool GATHER>
 __global__ void __launch_bounds__(kStThreads, 1) k_experts_stream(StArgs a) {
   extern __shared__ __align__(128) unsigned char st_smem[];
   __shared__ __align__(16) __nv_bfloat16 s_act[kStPassGroups][kStRows][16];    // a = silu(gate) * up of the pass
   __shared__ float s_w[kStPassGroups][kStRows];                                // routing weight of token n for group q's expert
   __shared__ int s_item[kStPassGroups];
+  __shared__ int s_row[kStRows];        // gather: output row of token column n (-1: unused column)
+  __shared__ float s_wt[kStRows];       // gather: its routing weight
   constexpr int SLOTS = kStSlots;
   constexpr int H = CPG * 1024, HW = H / kStWarps;      // output rows per warp in phase 2
   constexpr int KS = H / kStSlices, NCH = KS / 64;      // phase 1: elements per slice, 64-wide chunks per slice
@@ -110,8 +116,8 @@ __global__ void __launch_bounds__(kStThreads, 1) k_experts_stream(StArgs a) {
   const int NG = I / 16;
 
   // ---- token rows into shared memory (an input of the call: may overlap the selection kernel) ----
-  {
-    constexpr int per_row = H / 8;
+  constexpr int per_row = H / 8;
+  if (!GATHER) {
     for (int idx = tid; idx < kStRows * per_row; idx += kStThreads) {
       const int n = idx / per_row, ci = idx - n * per_row;
       uint4 v = make_uint4(0u, 0u, 0u, 0u);
@@ -144,8 +150,11 @@ __global__ void __launch_bounds__(kStThreads, 1) k_experts_stream(StArgs a) {
   const __nv_bfloat16* wmat = tile ? a.w_up : a.w_gate;
   const uint64_t pol = st_stream_policy();
 
+  int cur_item = -1;
   for (int s_lo = g_lo, s_hi; s_lo < g_hi; s_lo = s_hi) {
     s_hi = min(g_hi, s_lo + kStPassGroups);
+    const int item0 = s_lo / NG;
+    if (GATHER) s_hi = min(s_hi, (item0 + 1) * NG);      // a pass stays inside one work item
     const int ng = s_hi - s_lo;
     // ---- group table: lane q holds item, expert and position of group q ----
     int my_item = -1, my_e = 0, my_gi = 0;
@@ -196,8 +205,32 @@ __global__ void __launch_bounds__(kStThreads, 1) k_experts_stream(StArgs a) {
 #pragma unroll
     for (int b = 0; b < SLOTS - 1; ++b) issue_one();
 
-    // ---- routing weights of the pass's experts, per group and token (read in phase 2, after the barriers) ----
-    if (warp < ng) {
+    if (GATHER) {
+      // ---- a new work item: its rows and weights, then its token rows into shared memory (the first weight
+      //      chunks are already on their way) ----
+      if (warp == 0 && lane < ng) s_item[lane] = item0;
+      if (item0 != cur_item) {
+        if (warp == 0 && lane < kStRows) {
+          const WorkItem it = a.items[item0];
+          int row = -1;
+          float wt = 0.f;
+          if (lane < it.n) slot_row_weight(a.perm[it.begin + lane], T, d.k, a.topk_w, row, wt);
+          s_row[lane] = row;
+          s_wt[lane] = wt;
+        }
+        __syncthreads();
+        for (int idx = tid; idx < kStRows * per_row; idx += kStThreads) {
+          const int n = idx / per_row, ci = idx - n * per_row;
+          const int row = s_row[n];
+          uint4 v = make_uint4(0u, 0u, 0u, 0u);
+          if (row >= 0) v = st_ldg_stream(a.x + (size_t)row * H + ci * 8);
+          *reinterpret_cast<uint4*>(xs + (size_t)n * H * 2 + ((ci ^ n) << 4)) = v;
+        }
+        __syncthreads();
+        cur_item = item0;
+      }
+    } else if (warp < ng) {
+      // ---- routing weights of the pass's experts, per group and token (read in phase 2, after the barriers) ----
       const int item = __shfl_sync(0xffffffffu, my_item, warp);
       const WorkItem it = a.items[item];
       if (lane < kStRows) s_w[warp][lane] = 0.f;
@@ -283,17 +316,20 @@ __global__ void __launch_bounds__(kStThreads, 1) k_experts_stream(StArgs a) {
         }
         // the expert's groups in this pass are summed: scale by the routing weights and add to y
         if (q == ng - 1 || s_item[q + 1] != s_item[q]) {
-          const float wA = s_w[q][2 * c], wB = s_w[q][2 * c + 1];
-          float* y0 = a.y + (size_t)(2 * c) * H + warp * HW + g;
+          const float wA = GATHER ? s_wt[2 * c] : s_w[q][2 * c], wB = GATHER ? s_wt[2 * c + 1] : s_w[q][2 * c + 1];
+          const int rA = GATHER ? s_row[2 * c] : 2 * c, rB = GATHER ? s_row[2 * c + 1] : 2 * c + 1;
+          float* y0 = a.y + warp * HW + g;
+          float* yA = y0 + (size_t)max(rA, 0) * H;
+          float* yB = y0 + (size_t)max(rB, 0) * H;
 #pragma unroll
           for (int u = 0; u < CPG * 4; ++u) {
             if (wA != 0.f) {
-              atomicAdd(y0 + u * 16, wA * acc[u][0]);
-              atomicAdd(y0 + u * 16 + 8, wA * acc[u][2]);
+              atomicAdd(yA + u * 16, wA * acc[u][0]);
+              atomicAdd(yA + u * 16 + 8, wA * acc[u][2]);
             }
             if (wB != 0.f) {
-              atomicAdd(y0 + H + u * 16, wB * acc[u][1]);
-              atomicAdd(y0 + H + u * 16 + 8, wB * acc[u][3]);
+              atomicAdd(yB + u * 16, wB * acc[u][1]);
+              atomicAdd(yB + u * 16 + 8, wB * acc[u][3]);
             }
             acc[u][0] = acc[u][1] = acc[u][2] = acc[u][3] = 0.f;
           }
@@ -305,20 +341,31 @@ __global__ void __launch_bounds__(kStThreads, 1) k_experts_stream(StArgs a) {
   }
 }
 
+// Few rows: all rows resident.  Up to kStGatherMaxRows rows: items of 8 token-slots, rows gathered per item
+// (an expert with more than 8 slots is streamed once per item, which beyond that size costs more than the
+// tensor-memory kernel's larger tiles).
+constexpr int kStGatherMaxRows = 512;
 bool experts_stream_supported(int max_rows, int hidden, int inter) {
-  return max_rows <= kStRows && (hidden == 1024 || hidden == 2048) && inter % 16 == 0;
+  return max_rows <= kStGatherMaxRows && (hidden == 1024 || hidden == 2048) && inter % 16 == 0;
+}
+bool experts_stream_gathers(int max_rows) { return max_rows > kStRows; }
+int experts_stream_item_tile() { return kStRows; }
+
+static const void* stream_kernel(int hidden, bool gather) {
+  if (hidden == 1024)
+    return gather ? reinterpret_cast<const void*>(&k_experts_stream<1, true>) : reinterpret_cast<const void*>(&k_experts_stream<1, false>);
+  return gather ? reinterpret_cast<const void*>(&k_experts_stream<2, true>) : reinterpret_cast<const void*>(&k_experts_stream<2, false>);
 }
 
-cudaError_t configure_experts_stream(int hidden) {
-  const void* fn = hidden == 1024 ? reinterpret_cast<const void*>(&k_experts_stream<1>)
-                                  : reinterpret_cast<const void*>(&k_experts_stream<2>);
+cudaError_t configure_experts_stream(int hidden, int max_rows) {
+  const void* fn = stream_kernel(hidden, experts_stream_gathers(max_rows));
   cudaError_t e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)stream_smem_bytes(hidden));
   if (e == cudaSuccess) e = cudaFuncSetAttribute(fn, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
   return e;
 }
 
 cudaError_t launch_experts_stream(const void* x, const void* w_gate, const void* w_up, const void* w_down, Workspace ws,
-                                  float* y, Dims d, int grid, cudaStream_t s) {
+                                  float* y, Dims d, int max_rows, int grid, cudaStream_t s) {
   StArgs a;
   a.x = static_cast<const __nv_bfloat16*>(x);
   a.w_gate = static_cast<const __nv_bfloat16*>(w_gate);
@@ -341,7 +388,8 @@ cudaError_t launch_experts_stream(const void* x, const void* w_gate, const void*
   attrs[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attrs;
   cfg.numAttrs = 1;
-  return d.H == 1024 ? cudaLaunchKernelEx(&cfg, k_experts_stream<1>, a) : cudaLaunchKernelEx(&cfg, k_experts_stream<2>, a);
+  void* params[1] = {&a};
+  return cudaLaunchKernelExC(&cfg, stream_kernel(d.H, experts_stream_gathers(max_rows)), params);
 }
 
 }  // namespace team

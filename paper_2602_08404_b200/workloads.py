@@ -77,6 +77,10 @@ MINI_WRAP = Shape("mini_wrap_bf16", 768, 64, 4, 192, 0, "bf16", 16, 4, 3, 1, 2, 
 # holds, so its range spans several passes and windows are shared between neighbouring CTAs.
 STREAM_MULTI = Shape("stream_multi_bf16", 1024, 48, 8, 1024, 1, "bf16", 8, 4, 2, 1, 2, 0.7, seed=14)
 
+# More rows than the few-rows kernel keeps resident: its gather mode (work items of 8 token-slots, several
+# items for the experts that more than 8 rows chose), with a shared expert that every row uses.
+STREAM_GATHER = Shape("stream_gather_bf16", 1024, 48, 8, 512, 1, "bf16", 12, 4, 3, 1, 2, 0.7, seqs=2, seed=15)
+
 def round_to_bf16(a):
     """Round fp32 values to the nearest bf16-representable value (ties to even); returns fp32."""
     a = np.ascontiguousarray(a, dtype=np.float32)

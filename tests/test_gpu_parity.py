@@ -75,6 +75,13 @@ def test_few_rows_kernel_multi_pass_ranges_and_shared_expert(flags, weights_cach
 
 
 @pytest.mark.parametrize("flags", [0, 3])
+def test_few_rows_kernel_gather_mode_with_split_items(flags, weights_cache):
+    shape = W.STREAM_GATHER                      # 24 rows: the shared expert alone has three items of 8 slots
+    stats = P.run_schedule(shape, weights_cache(shape), W.make_schedule(shape), flags)
+    assert len(stats) == 4 and all(s["launches"] == 3 for s in stats)
+
+
+@pytest.mark.parametrize("flags", [0, 3])
 def test_c3_llada_shape_with_shared_expert(flags, weights_cache):
     stats = P.run_schedule(W.C3, weights_cache(W.C3), W.make_schedule(W.C3), flags)
     assert len(stats) == 8
