@@ -290,7 +290,7 @@ int team_select_experts(team_ctx* ctx, const team_step_state* st, team_routing* 
   cudaError_t e = team::launch_select(ctx->ws.logits, step_ptrs(st), ctx->ws, export_ptrs(out), d,
                                       policy_of(ctx->cfg), ctx->item_tile, s);
   if (e != cudaSuccess) return fail_cuda(ctx, e, "select");
-  ++ctx->last_launches;
+  ctx->last_launches += team::select_launches(d);
   return TEAM_OK;
 }
 
@@ -311,7 +311,7 @@ int team_moe_forward(team_ctx* ctx, const void* x, const team_step_state* st, te
   e = team::launch_select(ctx->ws.logits, step_ptrs(st), ctx->ws, export_ptrs(out), d, policy_of(ctx->cfg),
                           ctx->item_tile, s);
   if (e != cudaSuccess) return fail_cuda(ctx, e, "select");
-  ++ctx->last_launches;
+  ctx->last_launches += team::select_launches(d);
   cudaEvent_t ev0 = nullptr, ev1 = nullptr;
   if (ctx->timing) {
     if (ctx->ev_used + 2 > ctx->ev.size()) {

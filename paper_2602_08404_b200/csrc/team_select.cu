@@ -17,6 +17,7 @@ constexpr int kSelThreads = 1024;
 constexpr int kSelWarps = kSelThreads / 32;
 
 constexpr int kIdxInSmemMax = 8192;   // routed slots kept in shared memory between the rounds and the dispatch
+enum { kSelAll = 0, kSelRounds = 1, kSelDispatch = 2 };   // what one launch of the kernel does
 constexpr int kSmallSlots = 128;      // up to here every expert's thread counts and places its slots by itself
 
 struct SelSmem {
@@ -76,7 +77,7 @@ __device__ __forceinline__ bool is_decoded(uint8_t s) { return s == TEAM_TOK_NEW
 
 __global__ void __launch_bounds__(kSelThreads, 1)
 k_select(const float* __restrict__ logits, StepPtrs st, Workspace ws, RoutePtrs ex, Dims d, Policy p, int item_tile,
-         int wait_prior) {
+         int wait_prior, int mode) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   SelSmem s;
   sel_smem_layout(d, &s, smem_raw);
@@ -89,21 +90,25 @@ k_select(const float* __restrict__ logits, StepPtrs st, Workspace ws, RoutePtrs 
   const int S = T * k;
   // warps taking part in the dispatch walk: enough for 32 slots each, so small steps scan little
   const int nw = min(kSelWarps, (S + 31) / 32);
-  const bool one_row_per_warp = T <= kSelWarps;
+  const bool one_row_per_warp = T <= kSelWarps && mode == kSelAll;
+  // kSelRounds: CTA b of the grid routes the rows of the groups g with g % gridDim.x == b (the necessary set
+  // E_A is per group, so groups are independent up to the dispatch); every CTA classifies all rows.
+  const int nb = gridDim.x, cta = blockIdx.x;
 
   // ---- stage the step state (inputs of the call, not produced by the preceding kernel) ---------
   for (int i = tid; i < d.G * n_words32; i += kSelThreads) s.mask[i] = 0u;
   for (int i = tid; i < d.G; i += kSelThreads) s.has_first[i] = 0;
   for (int i = tid; i < nw * EN; i += kSelThreads) s.hist[i] = 0;
   // per-window publication counters of the expert kernel start every step from zero
-  for (int i = tid; i < ws.n_flags; i += kSelThreads) ws.win_flags[i] = 0;
+  if (mode != kSelDispatch)
+    for (int i = cta * kSelThreads + tid; i < ws.n_flags; i += nb * kSelThreads) ws.win_flags[i] = 0;
   float conf_r[TEAM_MAX_ROWS / kSelThreads];     // confidences of the rows this thread classifies, fetched with the rest
 #pragma unroll
   for (int i = 0; i < TEAM_MAX_ROWS / kSelThreads; ++i) {
     const int t = tid + i * kSelThreads;
     conf_r[i] = t < T ? st.conf[t] : 0.f;
   }
-  for (int t = tid; t < T; t += kSelThreads) {
+  for (int t = tid; t < T && mode != kSelDispatch; t += kSelThreads) {
     int g = st.group[t], b = st.branch[t];
     if (g < 0 || g >= d.G || b < 0 || b > 255) {
       set_status(ws.status, TEAM_ERR_STATE, 1);
@@ -117,7 +122,7 @@ k_select(const float* __restrict__ logits, StepPtrs st, Workspace ws, RoutePtrs 
   __syncthreads();
 
   // ---- Eq. 4: classification --------------------------------------------------------------
-  for (int t = tid; t < T; t += kSelThreads) {
+  for (int t = tid; t < T && mode != kSelDispatch; t += kSelThreads) {
     const uint8_t state = s.state[t];
     uint8_t c;
     if (state == TEAM_TOK_CACHED) {
@@ -145,7 +150,7 @@ k_select(const float* __restrict__ logits, StepPtrs st, Workspace ws, RoutePtrs 
   __syncthreads();
   // A group with no first-round row: its masked rows are all routed freely.  (Each thread only
   // rewrites rows it classified itself, so the next barrier is the one after round 1's reads.)
-  for (int t = tid; t < T; t += kSelThreads)
+  for (int t = tid; t < T && mode != kSelDispatch; t += kSelThreads)
     if (s.cls[t] == TEAM_CLS_COLD && !s.has_first[s.key[t] >> 8]) s.cls[t] = TEAM_CLS_FIRST;
 
   // Everything above depends on the step state only (inputs of the call) and overlaps the preceding
@@ -156,11 +161,18 @@ k_select(const float* __restrict__ logits, StepPtrs st, Workspace ws, RoutePtrs 
   float keep[kMaxPerLane];
   float keep_max = 0.f, keep_denom = 1.f;
   if (one_row_per_warp && warp < T) load_row(logits + (size_t)warp * E, E, lane, keep, keep_max, keep_denom);
+  if (mode == kSelDispatch) {
+    // classes and choices were left in the routing tables by the kSelRounds grid
+    for (int t = tid; t < T; t += kSelThreads) s.cls[t] = __ldcg(r.tok_class + t);
+    if (s.idx)
+      for (int i = tid; i < S; i += kSelThreads) s.idx[i] = __ldcg(r.topk_idx + i);
+  }
   __syncthreads();
 
   // ---- Algorithm 1, round 1 (free top-k) then round 2 (top-k inside E_A) -------------------
-  for (int round = 1; round <= 2; ++round) {
+  for (int round = 1; round <= 2 && mode != kSelDispatch; ++round) {
     for (int t = warp; t < T; t += kSelWarps) {
+      if (mode == kSelRounds && (s.key[t] >> 8) % nb != cta) continue;
       const uint8_t c = s.cls[t];
       if (round == 1 && c == TEAM_CLS_SKIP) {
         if (lane < k) {
@@ -223,19 +235,23 @@ k_select(const float* __restrict__ logits, StepPtrs st, Workspace ws, RoutePtrs 
   const int32_t* idx_src = s.idx ? s.idx : r.topk_idx;
 
   // ---- exports that need no further work: by the upper half of the CTA, beside the dispatch below ----
-  for (int t = tid - kSelThreads / 2; t >= 0 && t < T; t += kSelThreads / 2) {
+  for (int t = tid - kSelThreads / 2; t >= 0 && t < T && mode != kSelDispatch; t += kSelThreads / 2) {
+    if (mode == kSelRounds && (s.key[t] >> 8) % nb != cta) continue;
     r.tok_class[t] = s.cls[t];
     if (ex.tok_class) ex.tok_class[t] = s.cls[t];
   }
   {
     const int n_words64 = (E + 63) / 64;
-    for (int i = tid - kSelThreads / 2; i >= 0 && i < d.G * n_words64; i += kSelThreads / 2) {
+    for (int i = tid - kSelThreads / 2; i >= 0 && i < d.G * n_words64 && mode != kSelDispatch; i += kSelThreads / 2) {
       const int g = i / n_words64, wd = i % n_words64;
+      if (mode == kSelRounds && g % nb != cta) continue;
       const uint64_t m = (uint64_t)s.mask[g * n_words32 + 2 * wd] | ((uint64_t)s.mask[g * n_words32 + 2 * wd + 1] << 32);
       r.group_mask[i] = m;
       if (ex.group_mask) ex.group_mask[i] = m;
     }
   }
+
+  if (mode == kSelRounds) return;
 
   // ---- dispatch: stable counting sort of slots by expert ------------------------------------
   // Small steps (at most kSmallSlots routed slots): expert e's thread counts its slots by walking the
@@ -478,7 +494,18 @@ cudaError_t launch_select(const float* logits, StepPtrs st, Workspace ws, RouteP
   attr.val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = &attr;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, k_select, logits, st, ws, ex, d, p, item_tile, 1);
+  // Several groups and more rows than one CTA routes at once (one row per warp): the routing rounds run as
+  // one CTA per group (up to 32), the dispatch as a second single-CTA launch.
+  if (d.G > 1 && d.T > kSelWarps) {
+    cfg.gridDim = dim3(d.G < 32 ? d.G : 32);
+    cudaError_t e = cudaLaunchKernelEx(&cfg, k_select, logits, st, ws, ex, d, p, item_tile, 1, (int)kSelRounds);
+    if (e != cudaSuccess) return e;
+    cfg.gridDim = dim3(1);
+    return cudaLaunchKernelEx(&cfg, k_select, logits, st, ws, ex, d, p, item_tile, 1, (int)kSelDispatch);
+  }
+  return cudaLaunchKernelEx(&cfg, k_select, logits, st, ws, ex, d, p, item_tile, 1, (int)kSelAll);
 }
+
+int select_launches(Dims d) { return d.G > 1 && d.T > kSelWarps ? 2 : 1; }
 
 }  // namespace team

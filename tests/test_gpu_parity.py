@@ -48,7 +48,9 @@ def test_c1_tiny_fp32_all_steps(flags, weights_cache):
 @pytest.mark.parametrize("shape", [W.MINI_BF16, W.MINI_SHARED, W.MINI_WRAP], ids=lambda s: s.name)
 def test_mini_bf16_tensor_path(shape, flags, weights_cache):
     stats = P.run_schedule(shape, weights_cache(shape), W.make_schedule(shape), flags)
-    assert all(s["launches"] == 3 for s in stats)
+    # router, selection, experts; the selection is two launches (rounds per group, then dispatch) for several
+    # groups with more than 32 rows
+    assert all(s["launches"] == (4 if shape.seqs > 1 and shape.rows > 32 else 3) for s in stats)
 
 
 @pytest.mark.parametrize("shape", [W.MINI_BF16, W.MINI_SHARED], ids=lambda s: s.name)
