@@ -212,7 +212,8 @@ int team_select_experts(team_ctx *ctx, const team_step_state *st, team_routing *
 /* The whole layer step: route, select, dispatch, SwiGLU experts, weighted
  * combine.  y: fp32 [T, H]; rows with class TEAM_CLS_SKIP are left untouched
  * (they keep the previous step's output), all other rows are overwritten.
- * `out` may be NULL. */
+ * `out` may be NULL; tables nobody asked for may not be built at all (with at
+ * most 8 rows the expert kernel works from the rows' choices alone). */
 int team_moe_forward(team_ctx *ctx, const void *x, const team_step_state *st, team_routing *out,
                      float *y, void *stream);
 

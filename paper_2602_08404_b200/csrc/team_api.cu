@@ -288,7 +288,7 @@ int team_select_experts(team_ctx* ctx, const team_step_state* st, team_routing* 
   const team::Dims d = dims_of(ctx->cfg, st->n_rows);
   ctx->last_launches = 0;
   cudaError_t e = team::launch_select(ctx->ws.logits, step_ptrs(st), ctx->ws, export_ptrs(out), d,
-                                      policy_of(ctx->cfg), ctx->item_tile, s);
+                                      policy_of(ctx->cfg), ctx->item_tile, true, s);
   if (e != cudaSuccess) return fail_cuda(ctx, e, "select");
   ctx->last_launches += team::select_launches(d);
   return TEAM_OK;
@@ -308,8 +308,13 @@ int team_moe_forward(team_ctx* ctx, const void* x, const team_step_state* st, te
                                              st->tok_state, ctx->ws.logits, tc ? y : nullptr, d, ctx->cfg.flags, s);
   if (e != cudaSuccess) return fail_cuda(ctx, e, "router logits");
   ++ctx->last_launches;
+  // The resident few-rows expert kernel reads the rows' choices directly; the dispatch tables are built only
+  // when the caller asked for one of them.
+  const bool wants_tables = out != nullptr && (out->expert_count || out->expert_offset || out->perm || out->active ||
+                                               out->n_active || out->n_rows_active);
+  const bool resident = tc && ctx->stream_path && !team::experts_stream_gathers(ctx->cfg.max_rows);
   e = team::launch_select(ctx->ws.logits, step_ptrs(st), ctx->ws, export_ptrs(out), d, policy_of(ctx->cfg),
-                          ctx->item_tile, s);
+                          ctx->item_tile, wants_tables || !resident, s);
   if (e != cudaSuccess) return fail_cuda(ctx, e, "select");
   ctx->last_launches += team::select_launches(d);
   cudaEvent_t ev0 = nullptr, ev1 = nullptr;

@@ -109,7 +109,7 @@ cudaError_t launch_router_logits(const void* x, int dtype, const float* w_router
 cudaError_t launch_router_topk(const float* logits, const uint8_t* tok_state, RoutePtrs out, Dims d, Policy p,
                                cudaStream_t s);
 cudaError_t launch_select(const float* logits, StepPtrs st, Workspace ws, RoutePtrs ex, Dims d, Policy p,
-                          int item_tile, cudaStream_t s);
+                          int item_tile, bool need_tables, cudaStream_t s);
 int select_launches(Dims d);   // kernels launch_select issues for these sizes
 size_t select_smem_bytes(Dims d);
 cudaError_t launch_experts_simt(const void* x, int dtype, const void* w_gate, const void* w_up, const void* w_down,

@@ -43,6 +43,8 @@ struct StArgs {
   const __nv_bfloat16* w_up;
   const __nv_bfloat16* w_down;  // [E + ns, I/16, H, 16]
   const int32_t* perm;
+  const int32_t* topk_idx;      // [T, k] expert chosen per slot (-1: row skipped)
+  const uint8_t* tok_class;     // [T]
   const float* topk_w;
   const WorkItem* items;
   const int32_t* n_items;
@@ -128,7 +130,30 @@ __global__ void __launch_bounds__(kStThreads, 1) k_experts_stream(StArgs a) {
   asm volatile("griddepcontrol.wait;" ::: "memory");     // the selection kernel's tables are complete from here on
   __syncthreads();
 
-  const long long n_groups = (long long)(*a.n_items) * NG;
+  // Resident mode needs no dispatch tables: with at most 8 rows every warp reads the rows' choices (T*k slots)
+  // and forms the set of activated experts itself, word w of the bit set in lane w; activated expert number i
+  // is the i-th set bit.
+  int n_act = 0;
+  uint32_t act_word = 0u;
+  const int n_words = (d.E + d.ns + 31) >> 5;
+  if (!GATHER) {
+    const int S = T * d.k;
+    for (int base = 0; base < S; base += 32) {
+      const int i = base + lane;
+      const int e = i < S ? a.topk_idx[i] : -1;
+      for (int w = 0; w < n_words; ++w) {
+        const uint32_t m = __reduce_or_sync(0xffffffffu, (e >= 0 && (e >> 5) == w) ? 1u << (e & 31) : 0u);
+        if (lane == w) act_word |= m;
+      }
+    }
+    if (d.ns > 0) {     // shared experts are active as soon as one row is computed
+      const bool any = __ballot_sync(0xffffffffu, lane < T && a.tok_class[lane] != TEAM_CLS_SKIP) != 0u;
+      for (int sh = 0; sh < d.ns && any; ++sh)
+        if (lane == ((d.E + sh) >> 5)) act_word |= 1u << ((d.E + sh) & 31);
+    }
+    n_act = __reduce_add_sync(0xffffffffu, __popc(act_word));
+  }
+  const long long n_groups = (long long)(GATHER ? *a.n_items : n_act) * NG;
   const int g_lo = (int)(n_groups * blockIdx.x / gridDim.x), g_hi = (int)(n_groups * (blockIdx.x + 1) / gridDim.x);
 
   // ---- this warp's ring and its fixed lane roles ----
@@ -161,8 +186,17 @@ __global__ void __launch_bounds__(kStThreads, 1) k_experts_stream(StArgs a) {
     if (lane < ng) {
       const int grp = s_lo + lane;
       my_item = grp / NG;
-      my_e = a.items[my_item].e;
       my_gi = grp - my_item * NG;
+      if (GATHER) my_e = a.items[my_item].e;
+    }
+    if (!GATHER) {
+      int left = my_item;                   // the my_item-th set bit of the activated set (-1: no group in this lane)
+      for (int w = 0; w < n_words; ++w) {
+        const uint32_t m = __shfl_sync(0xffffffffu, act_word, w);
+        const int c = __popc(m);
+        if (left >= 0 && left < c) my_e = w * 32 + (int)__fns(m, 0, left + 1);
+        left = left >= c ? left - c : -1;
+      }
     }
     // ---- issue side: phase-1 chunks, then phase-2 chunks, then empty groups ----
     const int n1 = ng * NCH, n2 = ng * CPG;
@@ -231,16 +265,23 @@ __global__ void __launch_bounds__(kStThreads, 1) k_experts_stream(StArgs a) {
       }
     } else if (warp < ng) {
       // ---- routing weights of the pass's experts, per group and token (read in phase 2, after the barriers) ----
-      const int item = __shfl_sync(0xffffffffu, my_item, warp);
-      const WorkItem it = a.items[item];
-      if (lane < kStRows) s_w[warp][lane] = 0.f;
+      const int item = __shfl_sync(0xffffffffu, my_item, warp), e = __shfl_sync(0xffffffffu, my_e, warp);
       if (lane == 0) s_item[warp] = item;
-      __syncwarp();
-      if (lane < it.n) {
-        int row;
-        float wt;
-        slot_row_weight(a.perm[it.begin + lane], T, d.k, a.topk_w, row, wt);
-        s_w[warp][row] = wt;
+      if (lane < kStRows) {
+        float wt = 0.f;
+        if (lane < T) {
+          if (e >= d.E) {
+            wt = a.tok_class[lane] != TEAM_CLS_SKIP ? 1.f : 0.f;      // a shared expert: every computed row, weight 1
+          } else {
+            // all loads are independent of each other (no branch between them)
+            for (int j = 0; j < d.k; ++j) {
+              const int ej = a.topk_idx[lane * d.k + j];
+              const float wj = a.topk_w[lane * d.k + j];
+              wt = ej == e ? wj : wt;
+            }
+          }
+        }
+        s_w[warp][lane] = wt;
       }
     }
 
@@ -372,6 +413,8 @@ cudaError_t launch_experts_stream(const void* x, const void* w_gate, const void*
   a.w_up = static_cast<const __nv_bfloat16*>(w_up);
   a.w_down = static_cast<const __nv_bfloat16*>(w_down);
   a.perm = ws.r.perm;
+  a.topk_idx = ws.r.topk_idx;
+  a.tok_class = ws.r.tok_class;
   a.topk_w = ws.r.topk_w;
   a.items = ws.items;
   a.n_items = ws.n_items;

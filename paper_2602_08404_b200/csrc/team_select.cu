@@ -77,7 +77,7 @@ __device__ __forceinline__ bool is_decoded(uint8_t s) { return s == TEAM_TOK_NEW
 
 __global__ void __launch_bounds__(kSelThreads, 1)
 k_select(const float* __restrict__ logits, StepPtrs st, Workspace ws, RoutePtrs ex, Dims d, Policy p, int item_tile,
-         int wait_prior, int mode) {
+         int wait_prior, int mode, int skip_dispatch) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   SelSmem s;
   sel_smem_layout(d, &s, smem_raw);
@@ -251,7 +251,9 @@ k_select(const float* __restrict__ logits, StepPtrs st, Workspace ws, RoutePtrs 
     }
   }
 
-  if (mode == kSelRounds) return;
+  // The dispatch tables are skipped when nobody reads them: no export asked for, and an expert kernel that
+  // works from the rows' choices alone (at most 8 rows, all resident).
+  if (mode == kSelRounds || skip_dispatch) return;
 
   // ---- dispatch: stable counting sort of slots by expert ------------------------------------
   // Small steps (at most kSmallSlots routed slots): expert e's thread counts its slots by walking the
@@ -483,7 +485,7 @@ cudaError_t configure_select(Dims max_dims) {
 }
 
 cudaError_t launch_select(const float* logits, StepPtrs st, Workspace ws, RoutePtrs ex, Dims d, Policy p,
-                          int item_tile, cudaStream_t s) {
+                          int item_tile, bool need_tables, cudaStream_t s) {
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(1);
   cfg.blockDim = dim3(kSelThreads);
@@ -498,12 +500,12 @@ cudaError_t launch_select(const float* logits, StepPtrs st, Workspace ws, RouteP
   // one CTA per group (up to 32), the dispatch as a second single-CTA launch.
   if (d.G > 1 && d.T > kSelWarps) {
     cfg.gridDim = dim3(d.G < 32 ? d.G : 32);
-    cudaError_t e = cudaLaunchKernelEx(&cfg, k_select, logits, st, ws, ex, d, p, item_tile, 1, (int)kSelRounds);
+    cudaError_t e = cudaLaunchKernelEx(&cfg, k_select, logits, st, ws, ex, d, p, item_tile, 1, (int)kSelRounds, 0);
     if (e != cudaSuccess) return e;
     cfg.gridDim = dim3(1);
-    return cudaLaunchKernelEx(&cfg, k_select, logits, st, ws, ex, d, p, item_tile, 1, (int)kSelDispatch);
+    return cudaLaunchKernelEx(&cfg, k_select, logits, st, ws, ex, d, p, item_tile, 1, (int)kSelDispatch, 0);
   }
-  return cudaLaunchKernelEx(&cfg, k_select, logits, st, ws, ex, d, p, item_tile, 1, (int)kSelAll);
+  return cudaLaunchKernelEx(&cfg, k_select, logits, st, ws, ex, d, p, item_tile, 1, (int)kSelAll, need_tables ? 0 : 1);
 }
 
 int select_launches(Dims d) { return d.G > 1 && d.T > kSelWarps ? 2 : 1; }

@@ -188,3 +188,29 @@ def test_host_buffer_entry_point_matches_device_entry_point(weights_cache):
     finally:
         layer_a.close()
         layer_b.close()
+
+
+@pytest.mark.parametrize("shape", [W.C2, W.STREAM_MULTI], ids=lambda s: s.name)
+def test_forward_without_exports_skips_the_dispatch_tables_and_gives_the_same_y(shape, weights_cache):
+    """With at most 8 rows and no table asked for, the selection stops after the routing rounds and the expert
+    kernel works from the rows' choices; y must not depend on that."""
+    steps = W.make_schedule(shape)
+    for flags in (0, 3):
+        layer_a, layer_b = P.Layer(shape, weights_cache(shape), flags), P.Layer(shape, weights_cache(shape), flags)
+        try:
+            T, H = shape.rows, shape.hidden
+            y_a = torch.zeros((T, H), dtype=torch.float32, device="cuda")
+            y_b = torch.zeros((T, H), dtype=torch.float32, device="cuda")
+            for step in steps:
+                x = B.to_device(step["x"], B.TEAM_DTYPE_BF16)
+                st = B.state_to_device(step)
+                out = B.alloc_routing(layer_a.cfg, T)
+                B.team_moe_forward(layer_a.ctx, x, st, out, y_a)          # all tables exported
+                B.team_moe_forward(layer_b.ctx, x, st, None, y_b)         # none
+                torch.cuda.synchronize()
+                assert int(out["n_active"].item()) > 0
+                assert torch.allclose(y_b, y_a, rtol=0, atol=1e-5 * float(y_a.abs().max()))
+            assert B.team_read_status(layer_b.ctx)[0] == 0
+        finally:
+            layer_a.close()
+            layer_b.close()
