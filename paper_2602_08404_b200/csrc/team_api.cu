@@ -180,9 +180,11 @@ int team_create(const team_config* cfg, team_ctx** out) {
   const size_t o_act = take(cfg->dtype == TEAM_DTYPE_F32 ? S * cfg->inter * 4 : 256);
   const bool bf16 = cfg->dtype == TEAM_DTYPE_BF16;
   const size_t max_items = EN + S / ctx->item_tile + 2;
-  const size_t n_flags = bf16 ? max_items * (cfg->inter / 64) : 0;
+  // the exchange scratch and its counters belong to the tensor-memory expert kernel only
+  const bool exchange = bf16 && !ctx->stream_path;
+  const size_t n_flags = exchange ? max_items * (cfg->inter / 64) : 0;
   const size_t o_flags = take(n_flags * 4 + 4);
-  const size_t o_actg = take(bf16 ? max_items * ctx->item_tile * cfg->inter * 2 : 256);
+  const size_t o_actg = take(exchange ? max_items * ctx->item_tile * cfg->inter * 2 : 256);
   ctx->ws_bytes = off;
   e = cudaMalloc(&ctx->ws_base, ctx->ws_bytes);
   if (e != cudaSuccess) {
