@@ -119,15 +119,29 @@ __global__ void __launch_bounds__(kStThreads, 1) k_experts_stream(StArgs a) {
 
   // ---- token rows into shared memory (an input of the call: may overlap the selection kernel) ----
   constexpr int per_row = H / 8;
+  constexpr int kXLoads = kStRows * per_row / kStThreads;     // 16-byte pieces per thread
+  uint4 xv[kXLoads];
   if (!GATHER) {
-    for (int idx = tid; idx < kStRows * per_row; idx += kStThreads) {
-      const int n = idx / per_row, ci = idx - n * per_row;
-      uint4 v = make_uint4(0u, 0u, 0u, 0u);
-      if (n < T) v = st_ldg_stream(a.x + (size_t)n * H + ci * 8);
-      *reinterpret_cast<uint4*>(xs + (size_t)n * H * 2 + ((ci ^ n) << 4)) = v;
+#pragma unroll
+    for (int i = 0; i < kXLoads; ++i) {
+      const int idx = tid + i * kStThreads, n = idx / per_row, ci = idx - n * per_row;
+      xv[i] = n < T ? st_ldg_stream(a.x + (size_t)n * H + ci * 8) : make_uint4(0u, 0u, 0u, 0u);
     }
   }
   asm volatile("griddepcontrol.wait;" ::: "memory");     // the selection kernel's tables are complete from here on
+  // the rows' choices (resident mode) are requested before the token rows are parked in shared memory, so that
+  // the two round trips overlap when this kernel did not get to start ahead of the selection kernel's end
+  int e_slot[4] = {-1, -1, -1, -1};      // expert of slots lane, lane + 32, ... (T * k <= 128)
+  if (!GATHER) {
+#pragma unroll
+    for (int b = 0; b < 4; ++b)
+      if (b * 32 + lane < T * d.k) e_slot[b] = a.topk_idx[b * 32 + lane];
+#pragma unroll
+    for (int i = 0; i < kXLoads; ++i) {
+      const int idx = tid + i * kStThreads, n = idx / per_row, ci = idx - n * per_row;
+      *reinterpret_cast<uint4*>(xs + (size_t)n * H * 2 + ((ci ^ n) << 4)) = xv[i];
+    }
+  }
   __syncthreads();
 
   // Resident mode needs no dispatch tables: with at most 8 rows every warp reads the rows' choices (T*k slots)
@@ -137,10 +151,10 @@ __global__ void __launch_bounds__(kStThreads, 1) k_experts_stream(StArgs a) {
   uint32_t act_word = 0u;
   const int n_words = (d.E + d.ns + 31) >> 5;
   if (!GATHER) {
-    const int S = T * d.k;
-    for (int base = 0; base < S; base += 32) {
-      const int i = base + lane;
-      const int e = i < S ? a.topk_idx[i] : -1;
+#pragma unroll
+    for (int b = 0; b < 4; ++b) {
+      if (b * 32 >= T * d.k) break;
+      const int e = e_slot[b];
       for (int w = 0; w < n_words; ++w) {
         const uint32_t m = __reduce_or_sync(0xffffffffu, (e >= 0 && (e >> 5) == w) ? 1u << (e & 31) : 0u);
         if (lane == w) act_word |= m;
