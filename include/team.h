@@ -229,6 +229,10 @@ int team_moe_forward(team_ctx *ctx, const void *x, const team_step_state *st, te
  * DEVICE pointers as in team_moe_forward.  The first call on a context allocates
  * the staging block (device and pinned host, (6 H + 17) bytes per row of
  * max_rows for bf16); team_destroy frees it.  Not reentrant per context.
+ * On a stream that can be captured (not the legacy default stream, not already
+ * capturing) and with `out` NULL, the sequence copy in / kernels / copy out is
+ * recorded once per context and row count as a graph and replayed afterwards;
+ * team_set_weights, team_set_policy and team_debug_force_simt discard it.
  * Errors: as team_moe_forward. */
 int team_moe_forward_host(team_ctx *ctx, const void *x_host, const team_step_state *st_host,
                           team_routing *out, float *y_host, void *stream);

@@ -30,6 +30,10 @@ struct team_ctx {
   unsigned char* hs_dev;
   unsigned char* hs_pin;
   size_t hs_in_bytes, hs_y_off, hs_bytes;
+  // ... and the step (copy in, kernels, copy out) recorded once as a graph, replayed while nothing it bakes in changes
+  cudaGraphExec_t hs_graph;
+  int hs_graph_rows;
+  bool hs_graph_off;     // recording failed once: plain launches from then on
   char cuda_err[256];
   // expert-kernel timing
   bool timing;
@@ -99,6 +103,13 @@ team::RoutePtrs export_ptrs(const team_routing* r) {
   return e;
 }
 
+// Weight pointers, policy and kernel choice are baked into the recorded host-buffer step.
+void drop_host_graph(team_ctx* ctx) {
+  if (ctx->hs_graph) cudaGraphExecDestroy(ctx->hs_graph);
+  ctx->hs_graph = nullptr;
+  ctx->hs_graph_rows = 0;
+}
+
 bool use_tensor_path(const team_ctx* ctx) { return ctx->cfg.dtype == TEAM_DTYPE_BF16 && !ctx->force_simt; }
 
 int pick_item_tile(const team_config& c) { return team::experts_tc_item_tile(c.max_rows); }
@@ -143,6 +154,9 @@ int team_create(const team_config* cfg, team_ctx** out) {
   ctx->simt_act = nullptr;
   ctx->hs_dev = nullptr;
   ctx->hs_pin = nullptr;
+  ctx->hs_graph = nullptr;
+  ctx->hs_graph_rows = 0;
+  ctx->hs_graph_off = false;
   ctx->cuda_err[0] = 0;
   ctx->timing = false;
   ctx->ev_used = 0;
@@ -226,6 +240,7 @@ int team_destroy(team_ctx* ctx) {
   if (ctx->simt_act) cudaFree(ctx->simt_act);
   if (ctx->hs_dev) cudaFree(ctx->hs_dev);
   if (ctx->hs_pin) cudaFreeHost(ctx->hs_pin);
+  if (ctx->hs_graph) cudaGraphExecDestroy(ctx->hs_graph);
   delete ctx;
   return TEAM_OK;
 }
@@ -239,6 +254,7 @@ int team_set_weights(team_ctx* ctx, const team_weights* w) {
     return TEAM_ERR_ARG;
   ctx->w = *w;
   ctx->has_weights = true;
+  drop_host_graph(ctx);
   return TEAM_OK;
 }
 
@@ -251,6 +267,7 @@ int team_set_policy(team_ctx* ctx, const team_config* cfg) {
     return TEAM_ERR_SHAPE;
   if (cfg->L_hot < 0) return TEAM_ERR_ARG;
   ctx->cfg = *cfg;
+  drop_host_graph(ctx);
   return TEAM_OK;
 }
 
@@ -263,6 +280,7 @@ int team_debug_force_simt(team_ctx* ctx, int on) {
     ctx->ws.act = static_cast<float*>(ctx->simt_act);
   }
   ctx->force_simt = on;
+  drop_host_graph(ctx);
   return TEAM_OK;
 }
 
@@ -385,8 +403,6 @@ int team_moe_forward_host(team_ctx* ctx, const void* x_host, const team_step_sta
   memcpy(hp + o_br, st_host->branch, T * 4);
   // one copy in: with few rows the block is small and a single transfer beats six
   const size_t in_bytes = ctx->hs_in_bytes;
-  cudaError_t e = cudaMemcpyAsync(ctx->hs_dev, hp, in_bytes, cudaMemcpyHostToDevice, s);
-  if (e != cudaSuccess) return fail_cuda(ctx, e, "copy in");
   unsigned char* dp = ctx->hs_dev;
   team_step_state st = *st_host;
   st.tok_state = dp + o_ts;
@@ -395,11 +411,55 @@ int team_moe_forward_host(team_ctx* ctx, const void* x_host, const team_step_sta
   st.group = reinterpret_cast<const int32_t*>(dp + o_grp);
   st.branch = reinterpret_cast<const int32_t*>(dp + o_br);
   float* y_dev = reinterpret_cast<float*>(dp + ctx->hs_y_off);
-  rc = team_moe_forward(ctx, dp + o_x, &st, out, y_dev, stream);
-  if (rc != TEAM_OK) return rc;
-  e = cudaMemcpyAsync(hp + ctx->hs_y_off, y_dev, T * H * 4, cudaMemcpyDeviceToHost, s);
-  if (e == cudaSuccess) e = cudaStreamSynchronize(s);
-  if (e != cudaSuccess) return fail_cuda(ctx, e, "copy out");
+  // copy in, the layer, copy out: all addresses are the context's own, so the sequence is the same every step
+  auto issue = [&]() -> int {
+    cudaError_t e = cudaMemcpyAsync(ctx->hs_dev, hp, in_bytes, cudaMemcpyHostToDevice, s);
+    if (e != cudaSuccess) return fail_cuda(ctx, e, "copy in");
+    const int r = team_moe_forward(ctx, dp + o_x, &st, out, y_dev, stream);
+    if (r != TEAM_OK) return r;
+    e = cudaMemcpyAsync(hp + ctx->hs_y_off, y_dev, T * H * 4, cudaMemcpyDeviceToHost, s);
+    return e == cudaSuccess ? TEAM_OK : fail_cuda(ctx, e, "copy out");
+  };
+  // Replayed as one graph launch when possible: a stream that can be captured (not the legacy default stream,
+  // not already capturing), no exports, no expert timing.
+  bool replay = !ctx->hs_graph_off && s != nullptr && s != cudaStreamLegacy && out == nullptr && !ctx->timing;
+  if (replay) {
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(s, &cap) != cudaSuccess || cap != cudaStreamCaptureStatusNone) {
+      cudaGetLastError();
+      replay = false;
+    }
+  }
+  if (replay && (ctx->hs_graph == nullptr || ctx->hs_graph_rows != (int)T)) {
+    drop_host_graph(ctx);
+    cudaGraph_t g = nullptr;
+    bool good = cudaStreamBeginCapture(s, cudaStreamCaptureModeThreadLocal) == cudaSuccess;
+    if (good) {
+      const int r = issue();
+      const cudaError_t e = cudaStreamEndCapture(s, &g);
+      good = r == TEAM_OK && e == cudaSuccess && g != nullptr;
+    }
+    if (good) good = cudaGraphInstantiate(&ctx->hs_graph, g, 0) == cudaSuccess;
+    if (g) cudaGraphDestroy(g);
+    if (good) {
+      ctx->hs_graph_rows = (int)T;
+    } else {
+      cudaGetLastError();
+      ctx->hs_graph = nullptr;
+      ctx->hs_graph_off = true;
+      replay = false;
+    }
+  }
+  if (replay) {
+    const cudaError_t e = cudaGraphLaunch(ctx->hs_graph, s);
+    if (e != cudaSuccess) return fail_cuda(ctx, e, "graph launch");
+    ctx->last_launches = 2 + team::select_launches(dims_of(ctx->cfg, st_host->n_rows));
+  } else {
+    rc = issue();
+    if (rc != TEAM_OK) return rc;
+  }
+  const cudaError_t es = cudaStreamSynchronize(s);
+  if (es != cudaSuccess) return fail_cuda(ctx, es, "synchronise");
   memcpy(y_host, hp + ctx->hs_y_off, T * H * 4);
   return TEAM_OK;
 }

@@ -163,10 +163,23 @@ def test_c5_stack_sdar_shape_two_layers(weights_cache):
     _run_stack(W.C2, 2, 3, weights_cache)
 
 
-def test_host_buffer_entry_point_matches_device_entry_point(weights_cache):
-    """team_moe_forward_host on a whole schedule: same y as team_moe_forward, skipped rows keeping the previous step's."""
+@pytest.mark.parametrize("side_stream", [False, True], ids=["default_stream", "own_stream_graph_replay"])
+def test_host_buffer_entry_point_matches_device_entry_point(side_stream, weights_cache):
+    """team_moe_forward_host on a whole schedule, twice over (on a stream of its own the library replays the
+    recorded step from the second call on): same y as team_moe_forward, skipped rows keeping the previous step's."""
     shape, flags = W.C2, 3
-    steps = W.make_schedule(shape)
+    steps = W.make_schedule(shape) * 2
+    if side_stream:
+        stream = torch.cuda.Stream()
+        stream.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(stream):
+            _host_entry_schedule(shape, flags, steps, weights_cache)
+        torch.cuda.current_stream().wait_stream(stream)
+    else:
+        _host_entry_schedule(shape, flags, steps, weights_cache)
+
+
+def _host_entry_schedule(shape, flags, steps, weights_cache):
     layer_a, layer_b = P.Layer(shape, weights_cache(shape), flags), P.Layer(shape, weights_cache(shape), flags)
     try:
         T, H = shape.rows, shape.hidden
