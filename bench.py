@@ -45,8 +45,8 @@ def parse_args():
     ap.add_argument("--flags", type=int, default=TEAM_FLAGS, help="0 vanilla, 1 DCD, 3 DCD|LAC")
     ap.add_argument("--no-graph", action="store_true", help="issue every step as separate calls (no CUDA graph)")
     ap.add_argument("--cpu-seconds", type=float, default=15.0, help="budget of the oracle baseline leg")
-    ap.add_argument("--workload", default="c2", choices=["c2", "c3", "c4"],
-                    help="c2: the headline step (default); c3: 256 experts + shared, block 32; c4: c2 shape, --seqs x 4 branches x 4")
+    ap.add_argument("--workload", default="c2", choices=["c2", "c3", "c4", "paper"],
+                    help="c2: the headline step (default); c3: 256 experts + shared, block 32; c4: c2 shape, --seqs x 4 branches x 4; paper: c2 shape, block 32 x 4 branches in one group")
     ap.add_argument("--seqs", type=int, default=1, help="sequences of the c4 batch sweep")
     return ap.parse_args()
 
@@ -186,7 +186,7 @@ def main():
         dist.barrier()
     dev = torch.device("cuda", local_rank)
 
-    shape = {"c2": W.C2, "c3": W.C3, "c4": W.c4(args.seqs)}[args.workload]
+    shape = {"c2": W.C2, "c3": W.C3, "c4": W.c4(args.seqs), "paper": W.paper_point()}[args.workload]
     T, H, E, k, I = shape.rows, shape.hidden, shape.n_experts, shape.top_k, shape.inter
     ns = shape.n_shared
     workload = WORKLOAD if args.workload == "c2" else (

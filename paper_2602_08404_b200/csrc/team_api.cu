@@ -168,8 +168,8 @@ int team_create(const team_config* cfg, team_ctx** out) {
   }
   ctx->item_tile = pick_item_tile(*cfg);
   ctx->stream_path = cfg->dtype == TEAM_DTYPE_BF16 && team::experts_stream_supported(cfg->max_rows, cfg->hidden, cfg->inter);
-  // the few-rows kernel's gather mode takes work items of 8 token-slots
-  if (ctx->stream_path && team::experts_stream_gathers(cfg->max_rows)) ctx->item_tile = team::experts_stream_item_tile();
+  // the few-rows kernel's gather mode takes work items of 8 or 16 token-slots
+  if (ctx->stream_path && team::experts_stream_gathers(cfg->max_rows)) ctx->item_tile = team::experts_stream_item_tile(cfg->max_rows);
   e = team::configure_router(cfg->dtype, cfg->hidden);
   if (e == cudaSuccess) e = team::configure_select(dims_of(*cfg, cfg->max_rows));
   if (e == cudaSuccess && cfg->dtype == TEAM_DTYPE_BF16 && !ctx->stream_path) e = team::configure_experts_tc(ctx->item_tile);

@@ -100,7 +100,7 @@ cudaError_t configure_experts_tc(int item_tile);
 int experts_tc_item_tile(int max_rows);
 bool experts_stream_supported(int max_rows, int hidden, int inter);
 bool experts_stream_gathers(int max_rows);
-int experts_stream_item_tile();
+int experts_stream_item_tile(int max_rows);
 cudaError_t configure_experts_stream(int hidden, int max_rows);
 cudaError_t launch_experts_stream(const void* x, const void* w_gate, const void* w_up, const void* w_down, Workspace ws,
                                   float* y, Dims d, int max_rows, int grid, cudaStream_t s);

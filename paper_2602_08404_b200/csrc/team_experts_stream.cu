@@ -88,38 +88,45 @@ __device__ __forceinline__ void st_mma(float (&d)[4], const uint32_t (&a)[4], ui
                : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
 
-// shared memory: token rows | partial sums [group][slice][gate, up][16 rows][8 tokens] | per-warp rings
-__host__ __device__ inline size_t stream_smem_bytes(int H) {
-  return (size_t)kStRows * H * 2 + kStRedBytes + (size_t)kStWarps * kStSlots * kStChunkBytes;
+// shared memory: token rows | partial sums [group][slice][gate, up][16 rows][tokens] | per-warp rings.
+// ntl = token tiles of 8 (1 or 2): with 16 tokens a pass holds half the groups and a ring one slot less.
+__host__ __device__ inline int stream_slots(int ntl) { return ntl == 1 ? kStSlots : kStSlots - 1; }
+__host__ __device__ inline size_t stream_smem_bytes(int H, int ntl) {
+  return (size_t)kStRows * ntl * H * 2 + kStRedBytes + (size_t)kStWarps * stream_slots(ntl) * kStChunkBytes;
 }
 
 // CPG: 64-row chunks of a W_down slab per warp and group (H = CPG * 1024).
 // GATHER = false: the call has at most 8 rows; all of them are the mma's token columns for every expert, and a
 //                 row that did not choose the expert gets weight 0.
-// GATHER = true:  any number of rows; work items of at most 8 token-slots of one expert (built by the selection
-//                 kernel); a pass stays inside one item and the item's rows are gathered into shared memory.
-template <int CPG, bool GATHER>
+// GATHER = true:  any number of rows; work items of at most 8 * NTL token-slots of one expert (built by the
+//                 selection kernel); a pass stays inside one item and the item's rows are gathered into shared
+//                 memory.  NTL = 2 (two token tiles per weight fragment) halves how often an expert that many
+//                 rows chose is streamed; its pass holds 4 groups instead of 8.
+template <int CPG, bool GATHER, int NTL>
 __global__ void __launch_bounds__(kStThreads, 1) k_experts_stream(StArgs a) {
+  static_assert(NTL == 1 || (NTL == 2 && GATHER), "two token tiles only in gather mode");
+  constexpr int TOK = kStRows * NTL;                 // token columns
+  constexpr int PASS = kStPassGroups / NTL;          // groups per pass
   extern __shared__ __align__(128) unsigned char st_smem[];
-  __shared__ __align__(16) __nv_bfloat16 s_act[kStPassGroups][kStRows][16];    // a = silu(gate) * up of the pass
+  __shared__ __align__(16) __nv_bfloat16 s_act[PASS * TOK * 16];               // a = silu(gate) * up of the pass: [group][token][16]
   __shared__ float s_w[kStPassGroups][kStRows];                                // routing weight of token n for group q's expert
   __shared__ int s_item[kStPassGroups];
-  __shared__ int s_row[kStRows];        // gather: output row of token column n (-1: unused column)
-  __shared__ float s_wt[kStRows];       // gather: its routing weight
-  constexpr int SLOTS = kStSlots;
+  __shared__ int s_row[TOK];            // gather: output row of token column n (-1: unused column)
+  __shared__ float s_wt[TOK];           // gather: its routing weight
+  constexpr int SLOTS = NTL == 1 ? kStSlots : kStSlots - 1;
   constexpr int H = CPG * 1024, HW = H / kStWarps;      // output rows per warp in phase 2
   constexpr int KS = H / kStSlices, NCH = KS / 64;      // phase 1: elements per slice, 64-wide chunks per slice
   const Dims d = a.d;
   const int I = d.I, T = d.T;
-  unsigned char* xs = st_smem;                                                    // [8][H] bf16, 16-byte pieces swizzled
-  float* red = reinterpret_cast<float*>(st_smem + (size_t)kStRows * H * 2);      // [group][slice][2][16][8]
+  unsigned char* xs = st_smem;                                                    // [TOK][H] bf16, 16-byte pieces swizzled
+  float* red = reinterpret_cast<float*>(st_smem + (size_t)TOK * H * 2);          // [group][slice][2][16][TOK]
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int g = lane >> 2, c = lane & 3;        // fragment row (and token of the B fragment), k / token pair
   const int NG = I / 16;
 
   // ---- token rows into shared memory (an input of the call: may overlap the selection kernel) ----
   constexpr int per_row = H / 8;
-  constexpr int kXLoads = kStRows * per_row / kStThreads;     // 16-byte pieces per thread
+  constexpr int kXLoads = TOK * per_row / kStThreads;         // 16-byte pieces per thread
   uint4 xv[kXLoads];
   if (!GATHER) {
 #pragma unroll
@@ -171,7 +178,7 @@ __global__ void __launch_bounds__(kStThreads, 1) k_experts_stream(StArgs a) {
   const int g_lo = (int)(n_groups * blockIdx.x / gridDim.x), g_hi = (int)(n_groups * (blockIdx.x + 1) / gridDim.x);
 
   // ---- this warp's ring and its fixed lane roles ----
-  const uint32_t ring = st_smem_u32(st_smem + (size_t)kStRows * H * 2 + kStRedBytes + (size_t)warp * SLOTS * kStChunkBytes);
+  const uint32_t ring = st_smem_u32(st_smem + (size_t)TOK * H * 2 + kStRedBytes + (size_t)warp * SLOTS * kStChunkBytes);
   // phase-1 chunk: 16 rows x 128 bytes; lane copies one 16-byte piece of rows cp_row + 4j; piece p of row r sits at p ^ (r & 7)
   const int cp_row = lane >> 3, cp_piece = lane & 7;
   const uint32_t cp_off0 = cp_row * 128 + ((cp_piece ^ cp_row) << 4);          // rows cp_row, cp_row + 8 (+1024)
@@ -191,7 +198,7 @@ __global__ void __launch_bounds__(kStThreads, 1) k_experts_stream(StArgs a) {
 
   int cur_item = -1;
   for (int s_lo = g_lo, s_hi; s_lo < g_hi; s_lo = s_hi) {
-    s_hi = min(g_hi, s_lo + kStPassGroups);
+    s_hi = min(g_hi, s_lo + PASS);
     const int item0 = s_lo / NG;
     if (GATHER) s_hi = min(s_hi, (item0 + 1) * NG);      // a pass stays inside one work item
     const int ng = s_hi - s_lo;
@@ -233,18 +240,17 @@ __global__ void __launch_bounds__(kStThreads, 1) k_experts_stream(StArgs a) {
           if (++iq == ng) iq = 0;      // phase 2 walks the groups again
         }
       } else if (n_issued < n1 + n2) {
-        if (icc == 0) {
-          const int e = __shfl_sync(0xffffffffu, my_e, iq), gi = __shfl_sync(0xffffffffu, my_gi, iq);
-          i_src = a.w_down + (((size_t)e * NG + gi) * H + warp * HW) * 16 + lane * 8;
-        }
-        const __nv_bfloat16* p = i_src + icc * 1024;
+        // phase 2 walks (row chunk, group): all groups of the pass for the warp's first 64 output rows, then
+        // for the next 64, so that the accumulators cover 64 rows at a time
+        const int e = __shfl_sync(0xffffffffu, my_e, iq), gi = __shfl_sync(0xffffffffu, my_gi, iq);
+        const __nv_bfloat16* p = a.w_down + (((size_t)e * NG + gi) * H + warp * HW) * 16 + lane * 8 + icc * 1024;
         st_cp16(dst + cq_off, p, pol);
         st_cp16(dst + cq_off + 512, p + 256, pol);
         st_cp16(dst + cq_off + 1024, p + 512, pol);
         st_cp16(dst + cq_off + 1536, p + 768, pol);
-        if (++icc == CPG) {
-          icc = 0;
-          ++iq;
+        if (++iq == ng) {
+          iq = 0;
+          ++icc;
         }
       }
       st_commit();
@@ -258,7 +264,7 @@ __global__ void __launch_bounds__(kStThreads, 1) k_experts_stream(StArgs a) {
       //      chunks are already on their way) ----
       if (warp == 0 && lane < ng) s_item[lane] = item0;
       if (item0 != cur_item) {
-        if (warp == 0 && lane < kStRows) {
+        if (warp == 0 && lane < TOK) {
           const WorkItem it = a.items[item0];
           int row = -1;
           float wt = 0.f;
@@ -267,12 +273,12 @@ __global__ void __launch_bounds__(kStThreads, 1) k_experts_stream(StArgs a) {
           s_wt[lane] = wt;
         }
         __syncthreads();
-        for (int idx = tid; idx < kStRows * per_row; idx += kStThreads) {
+        for (int idx = tid; idx < TOK * per_row; idx += kStThreads) {
           const int n = idx / per_row, ci = idx - n * per_row;
           const int row = s_row[n];
           uint4 v = make_uint4(0u, 0u, 0u, 0u);
           if (row >= 0) v = st_ldg_stream(a.x + (size_t)row * H + ci * 8);
-          *reinterpret_cast<uint4*>(xs + (size_t)n * H * 2 + ((ci ^ n) << 4)) = v;
+          *reinterpret_cast<uint4*>(xs + (size_t)n * H * 2 + ((ci ^ (n & 7)) << 4)) = v;
         }
         __syncthreads();
         cur_item = item0;
@@ -302,7 +308,9 @@ __global__ void __launch_bounds__(kStThreads, 1) k_experts_stream(StArgs a) {
     // ---- phase 1 ----
     int t = 0;     // chunks consumed in this pass
     {
-      float acc[4] = {0.f, 0.f, 0.f, 0.f};
+      float acc[NTL][4];
+#pragma unroll
+      for (int nt = 0; nt < NTL; ++nt) acc[nt][0] = acc[nt][1] = acc[nt][2] = acc[nt][3] = 0.f;
       int q = 0, cc = 0;
       for (; t < n1; ++t) {
         issue_one();
@@ -310,24 +318,32 @@ __global__ void __launch_bounds__(kStThreads, 1) k_experts_stream(StArgs a) {
         __syncwarp();
         const uint32_t slot = ring + (uint32_t)(t % SLOTS) * kStChunkBytes;
         const int p0 = (ks * KS + cc * 64) >> 3;               // first 16-byte piece of the token rows
-        uint32_t bf0[4], bf1[4];
-        st_ldmatrix4(xs_lane + (uint32_t)((p0 + (b_m ^ b_tok)) << 4), bf0);
-        st_ldmatrix4(xs_lane + (uint32_t)((p0 + ((4 + b_m) ^ b_tok)) << 4), bf1);
-        uint32_t af[4];
-        st_ldmatrix4(slot + a1_base + (uint32_t)(((0 + a_hi) ^ a1_swz) << 4), af);
-        st_mma(acc, af, bf0[0], bf0[1]);
-        st_ldmatrix4(slot + a1_base + (uint32_t)(((2 + a_hi) ^ a1_swz) << 4), af);
-        st_mma(acc, af, bf0[2], bf0[3]);
-        st_ldmatrix4(slot + a1_base + (uint32_t)(((4 + a_hi) ^ a1_swz) << 4), af);
-        st_mma(acc, af, bf1[0], bf1[1]);
-        st_ldmatrix4(slot + a1_base + (uint32_t)(((6 + a_hi) ^ a1_swz) << 4), af);
-        st_mma(acc, af, bf1[2], bf1[3]);
+        uint32_t bf0[NTL][4], bf1[NTL][4];
+#pragma unroll
+        for (int nt = 0; nt < NTL; ++nt) {
+          const uint32_t xrow = xs_lane + (uint32_t)nt * 8 * H * 2;      // token nt * 8 + b_tok: same swizzle
+          st_ldmatrix4(xrow + (uint32_t)((p0 + (b_m ^ b_tok)) << 4), bf0[nt]);
+          st_ldmatrix4(xrow + (uint32_t)((p0 + ((4 + b_m) ^ b_tok)) << 4), bf1[nt]);
+        }
+#pragma unroll
+        for (int ks16 = 0; ks16 < 4; ++ks16) {
+          uint32_t af[4];
+          st_ldmatrix4(slot + a1_base + (uint32_t)(((2 * ks16 + a_hi) ^ a1_swz) << 4), af);
+#pragma unroll
+          for (int nt = 0; nt < NTL; ++nt) {
+            const uint32_t* bf = ks16 < 2 ? bf0[nt] : bf1[nt];
+            st_mma(acc[nt], af, bf[(ks16 & 1) * 2], bf[(ks16 & 1) * 2 + 1]);
+          }
+        }
         __syncwarp();                                           // the slot may be overwritten from here on
         if (++cc == NCH) {
-          float* r = red + ((size_t)((q * kStSlices + ks) * 2 + tile) * 16) * kStRows;
-          *reinterpret_cast<float2*>(r + g * kStRows + 2 * c) = make_float2(acc[0], acc[1]);
-          *reinterpret_cast<float2*>(r + (g + 8) * kStRows + 2 * c) = make_float2(acc[2], acc[3]);
-          acc[0] = acc[1] = acc[2] = acc[3] = 0.f;
+          float* r = red + ((size_t)((q * kStSlices + ks) * 2 + tile) * 16) * TOK;
+#pragma unroll
+          for (int nt = 0; nt < NTL; ++nt) {
+            *reinterpret_cast<float2*>(r + g * TOK + nt * 8 + 2 * c) = make_float2(acc[nt][0], acc[nt][1]);
+            *reinterpret_cast<float2*>(r + (g + 8) * TOK + nt * 8 + 2 * c) = make_float2(acc[nt][2], acc[nt][3]);
+            acc[nt][0] = acc[nt][1] = acc[nt][2] = acc[nt][3] = 0.f;
+          }
           cc = 0;
           ++q;
         }
@@ -335,58 +351,68 @@ __global__ void __launch_bounds__(kStThreads, 1) k_experts_stream(StArgs a) {
     }
     __syncthreads();
     // ---- sum the slices, SwiGLU ----
-    for (int idx = tid; idx < ng * 16 * kStRows; idx += kStThreads) {
-      const int qq = idx >> 7, r = (idx >> 3) & 15, n = idx & 7;
+    for (int idx = tid; idx < ng * 16 * TOK; idx += kStThreads) {
+      const int qq = idx / (16 * TOK), r = (idx / TOK) & 15, n = idx % TOK;
       float gs = 0.f, us = 0.f;
 #pragma unroll
       for (int s = 0; s < kStSlices; ++s) {
-        const float* base = red + ((size_t)((qq * kStSlices + s) * 2) * 16) * kStRows + r * kStRows + n;
+        const float* base = red + ((size_t)((qq * kStSlices + s) * 2) * 16) * TOK + r * TOK + n;
         gs += base[0];
-        us += base[16 * kStRows];
+        us += base[16 * TOK];
       }
-      s_act[qq][n][r] = __float2bfloat16_rn(gs / (1.f + expf(-gs)) * us);     // rows n >= T are zero (x is)
+      s_act[(qq * TOK + n) * 16 + r] = __float2bfloat16_rn(gs / (1.f + expf(-gs)) * us);     // unused token columns are zero (x is)
     }
     __syncthreads();
-    // ---- phase 2 ----
-    {
-      float acc[CPG * 4][4];
+    // ---- phase 2: for each 64-row chunk of this warp's output rows, all groups of the pass ----
+#pragma unroll 1
+    for (int ch = 0; ch < CPG; ++ch) {
+      float acc[4][NTL][4];
 #pragma unroll
-      for (int u = 0; u < CPG * 4; ++u) acc[u][0] = acc[u][1] = acc[u][2] = acc[u][3] = 0.f;
-      for (int q = 0; q < ng; ++q) {
-        const uint32_t b0 = *reinterpret_cast<const uint32_t*>(&s_act[q][g][2 * c]);
-        const uint32_t b1 = *reinterpret_cast<const uint32_t*>(&s_act[q][g][8 + 2 * c]);
+      for (int u = 0; u < 4; ++u)
 #pragma unroll
-        for (int ch = 0; ch < CPG; ++ch, ++t) {
-          issue_one();
-          st_wait_group<SLOTS - 1>();
-          __syncwarp();
-          const uint32_t slot = ring + (uint32_t)(t % SLOTS) * kStChunkBytes;
+        for (int nt = 0; nt < NTL; ++nt) acc[u][nt][0] = acc[u][nt][1] = acc[u][nt][2] = acc[u][nt][3] = 0.f;
+      for (int q = 0; q < ng; ++q, ++t) {
+        issue_one();
+        st_wait_group<SLOTS - 1>();
+        __syncwarp();
+        const uint32_t slot = ring + (uint32_t)(t % SLOTS) * kStChunkBytes;
+        uint32_t b0[NTL], b1[NTL];
 #pragma unroll
-          for (int u = 0; u < 4; ++u) {
-            uint32_t af[4];
-            st_ldmatrix4(slot + u * 512 + a2_off, af);
-            st_mma(acc[ch * 4 + u], af, b0, b1);
-          }
-          __syncwarp();
+        for (int nt = 0; nt < NTL; ++nt) {
+          const __nv_bfloat16* ar = s_act + (q * TOK + nt * 8 + g) * 16;
+          b0[nt] = *reinterpret_cast<const uint32_t*>(ar + 2 * c);
+          b1[nt] = *reinterpret_cast<const uint32_t*>(ar + 8 + 2 * c);
         }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          uint32_t af[4];
+          st_ldmatrix4(slot + u * 512 + a2_off, af);
+#pragma unroll
+          for (int nt = 0; nt < NTL; ++nt) st_mma(acc[u][nt], af, b0[nt], b1[nt]);
+        }
+        __syncwarp();
         // the expert's groups in this pass are summed: scale by the routing weights and add to y
         if (q == ng - 1 || s_item[q + 1] != s_item[q]) {
-          const float wA = GATHER ? s_wt[2 * c] : s_w[q][2 * c], wB = GATHER ? s_wt[2 * c + 1] : s_w[q][2 * c + 1];
-          const int rA = GATHER ? s_row[2 * c] : 2 * c, rB = GATHER ? s_row[2 * c + 1] : 2 * c + 1;
-          float* y0 = a.y + warp * HW + g;
-          float* yA = y0 + (size_t)max(rA, 0) * H;
-          float* yB = y0 + (size_t)max(rB, 0) * H;
+          float* y0 = a.y + warp * HW + ch * 64 + g;
 #pragma unroll
-          for (int u = 0; u < CPG * 4; ++u) {
-            if (wA != 0.f) {
-              atomicAdd(yA + u * 16, wA * acc[u][0]);
-              atomicAdd(yA + u * 16 + 8, wA * acc[u][2]);
+          for (int nt = 0; nt < NTL; ++nt) {
+            const int cA = nt * 8 + 2 * c, cB = cA + 1;          // this thread's two token columns
+            const float wA = GATHER ? s_wt[cA] : s_w[q][cA], wB = GATHER ? s_wt[cB] : s_w[q][cB];
+            const int rA = GATHER ? s_row[cA] : cA, rB = GATHER ? s_row[cB] : cB;
+            float* yA = y0 + (size_t)max(rA, 0) * H;
+            float* yB = y0 + (size_t)max(rB, 0) * H;
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+              if (wA != 0.f) {
+                atomicAdd(yA + u * 16, wA * acc[u][nt][0]);
+                atomicAdd(yA + u * 16 + 8, wA * acc[u][nt][2]);
+              }
+              if (wB != 0.f) {
+                atomicAdd(yB + u * 16, wB * acc[u][nt][1]);
+                atomicAdd(yB + u * 16 + 8, wB * acc[u][nt][3]);
+              }
+              acc[u][nt][0] = acc[u][nt][1] = acc[u][nt][2] = acc[u][nt][3] = 0.f;
             }
-            if (wB != 0.f) {
-              atomicAdd(yB + u * 16, wB * acc[u][1]);
-              atomicAdd(yB + u * 16 + 8, wB * acc[u][3]);
-            }
-            acc[u][0] = acc[u][1] = acc[u][2] = acc[u][3] = 0.f;
           }
         }
       }
@@ -396,25 +422,33 @@ __global__ void __launch_bounds__(kStThreads, 1) k_experts_stream(StArgs a) {
   }
 }
 
-// Few rows: all rows resident.  Up to kStGatherMaxRows rows: items of 8 token-slots, rows gathered per item
-// (an expert with more than 8 slots is streamed once per item, which beyond that size costs more than the
-// tensor-memory kernel's larger tiles).
+// Few rows: all rows resident.  Up to kStGatherMaxRows rows: work items whose rows are gathered per item, of
+// 8 token-slots up to kStOneTileMaxRows rows per call (few experts see more than 8 rows there) and of 16 above
+// (an expert with more slots than an item holds is streamed once per item, which beyond kStGatherMaxRows costs
+// more than the tensor-memory kernel's larger tiles).
 constexpr int kStGatherMaxRows = 512;
+constexpr int kStOneTileMaxRows = 64;
 bool experts_stream_supported(int max_rows, int hidden, int inter) {
   return max_rows <= kStGatherMaxRows && (hidden == 1024 || hidden == 2048) && inter % 16 == 0;
 }
 bool experts_stream_gathers(int max_rows) { return max_rows > kStRows; }
-int experts_stream_item_tile() { return kStRows; }
+static int stream_token_tiles(int max_rows) { return max_rows > kStOneTileMaxRows ? 2 : 1; }
+int experts_stream_item_tile(int max_rows) { return kStRows * stream_token_tiles(max_rows); }
 
-static const void* stream_kernel(int hidden, bool gather) {
-  if (hidden == 1024)
-    return gather ? reinterpret_cast<const void*>(&k_experts_stream<1, true>) : reinterpret_cast<const void*>(&k_experts_stream<1, false>);
-  return gather ? reinterpret_cast<const void*>(&k_experts_stream<2, true>) : reinterpret_cast<const void*>(&k_experts_stream<2, false>);
+static const void* stream_kernel(int hidden, int max_rows) {
+  const bool gather = experts_stream_gathers(max_rows), two = stream_token_tiles(max_rows) == 2;
+  if (hidden == 1024) {
+    if (!gather) return reinterpret_cast<const void*>(&k_experts_stream<1, false, 1>);
+    return two ? reinterpret_cast<const void*>(&k_experts_stream<1, true, 2>) : reinterpret_cast<const void*>(&k_experts_stream<1, true, 1>);
+  }
+  if (!gather) return reinterpret_cast<const void*>(&k_experts_stream<2, false, 1>);
+  return two ? reinterpret_cast<const void*>(&k_experts_stream<2, true, 2>) : reinterpret_cast<const void*>(&k_experts_stream<2, true, 1>);
 }
 
 cudaError_t configure_experts_stream(int hidden, int max_rows) {
-  const void* fn = stream_kernel(hidden, experts_stream_gathers(max_rows));
-  cudaError_t e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)stream_smem_bytes(hidden));
+  const void* fn = stream_kernel(hidden, max_rows);
+  cudaError_t e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       (int)stream_smem_bytes(hidden, stream_token_tiles(max_rows)));
   if (e == cudaSuccess) e = cudaFuncSetAttribute(fn, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
   return e;
 }
@@ -438,7 +472,7 @@ cudaError_t launch_experts_stream(const void* x, const void* w_gate, const void*
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(grid);
   cfg.blockDim = dim3(kStThreads);
-  cfg.dynamicSmemBytes = stream_smem_bytes(d.H);
+  cfg.dynamicSmemBytes = stream_smem_bytes(d.H, stream_token_tiles(max_rows));
   cfg.stream = s;
   cudaLaunchAttribute attrs[1];
   attrs[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
@@ -446,7 +480,7 @@ cudaError_t launch_experts_stream(const void* x, const void* w_gate, const void*
   cfg.attrs = attrs;
   cfg.numAttrs = 1;
   void* params[1] = {&a};
-  return cudaLaunchKernelExC(&cfg, stream_kernel(d.H, experts_stream_gathers(max_rows)), params);
+  return cudaLaunchKernelExC(&cfg, stream_kernel(d.H, max_rows), params);
 }
 
 }  // namespace team

@@ -56,6 +56,12 @@ def c4(seqs):
     return replace(C2, name=f"c4_sdar_b{seqs}", seqs=seqs, branches=4, seed=4 + seqs)
 
 
+def paper_point():
+    """The operating point of the paper's experiments (Sec. 5.1) on the SDAR shape: one sequence, block of 32
+    tokens, 4 speculative branches (128 rows in one group), L_hot = 3, 4 tokens accepted per step."""
+    return replace(C2, name="paper_block32_x4", block=32, branches=4, n_steps=8, unmask_per_step=4, L_hot=3, seed=17)
+
+
 C5_LAYERS = 48
 C5_BLOCKS = 64
 
@@ -80,6 +86,9 @@ STREAM_MULTI = Shape("stream_multi_bf16", 1024, 48, 8, 1024, 1, "bf16", 8, 4, 2,
 # More rows than the few-rows kernel keeps resident: its gather mode (work items of 8 token-slots, several
 # items for the experts that more than 8 rows chose), with a shared expert that every row uses.
 STREAM_GATHER = Shape("stream_gather_bf16", 1024, 48, 8, 512, 1, "bf16", 12, 4, 3, 1, 2, 0.7, seqs=2, seed=15)
+
+# Enough rows per call that the gather mode works on items of 16 token-slots (two token tiles per weight fragment).
+STREAM_GATHER16 = Shape("stream_gather16_bf16", 1024, 48, 8, 512, 1, "bf16", 40, 4, 6, 1, 3, 0.7, seqs=2, seed=16)
 
 def round_to_bf16(a):
     """Round fp32 values to the nearest bf16-representable value (ties to even); returns fp32."""

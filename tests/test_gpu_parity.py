@@ -84,9 +84,22 @@ def test_few_rows_kernel_gather_mode_with_split_items(flags, weights_cache):
 
 
 @pytest.mark.parametrize("flags", [0, 3])
+def test_few_rows_kernel_gather_mode_items_of_16_slots(flags, weights_cache):
+    shape = W.STREAM_GATHER16                    # 80 rows in 2 groups: items of 16 slots, the shared expert has five
+    stats = P.run_schedule(shape, weights_cache(shape), W.make_schedule(shape), flags)
+    assert len(stats) == 4 and all(s["launches"] == 4 for s in stats)
+
+
+@pytest.mark.parametrize("flags", [0, 3])
 def test_c3_llada_shape_with_shared_expert(flags, weights_cache):
     stats = P.run_schedule(W.C3, weights_cache(W.C3), W.make_schedule(W.C3), flags)
     assert len(stats) == 8
+
+
+def test_paper_operating_point_block32_four_branches_one_group(weights_cache):
+    shape = W.paper_point()                      # 128 rows, one group: single-CTA selection, gathered expert items
+    steps = W.make_schedule(shape)[1:4]
+    P.run_schedule(shape, weights_cache(shape), steps, 3)
 
 
 @pytest.mark.parametrize("seqs", [1, 4, 16, 64])
