@@ -346,7 +346,7 @@ def main():
     peak, peak_kind = measured_peaks()
     achieved = algo_bytes / (kernel_ms * 1e-3) / 1e9
     value = R_.whole_job_rate(T, ms_per_step)
-    stream_kernel = T <= 512 and H in (1024, 2048)      # the library's choice: few-rows kernel (resident or gather mode)
+    stream_kernel = H in (1024, 2048)      # the library's choice: weight-streaming kernel (resident or gather mode)
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,

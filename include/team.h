@@ -88,8 +88,8 @@ typedef struct {
   int32_t inter;       /* I; multiple of 64 for bf16, of 16 for fp32                     */
   int32_t n_shared;    /* always-on experts appended after the routed ones              */
   int32_t max_rows;    /* largest n_rows of any call on this context; it also picks the
-                          expert kernel (bf16, H 1024 or 2048): <= 8 rows resident,
-                          <= 512 gathered per work item, above that tensor-memory tiles  */
+                          expert kernel's mode (bf16, H 1024 or 2048): <= 8 rows all
+                          resident, <= 64 items of 8 token-slots, above items of 16     */
   int32_t max_groups;  /* group ids are in [0, max_groups), <= TEAM_MAX_GROUPS; branch ids in [0, 256) */
   int32_t dtype;       /* TEAM_DTYPE_F32: x and expert weights fp32 (plain FMA kernels);
                           TEAM_DTYPE_BF16: x and expert weights bf16, fp32 accumulation

@@ -426,7 +426,7 @@ __global__ void __launch_bounds__(kStThreads, 1) k_experts_stream(StArgs a) {
 // 8 token-slots up to kStOneTileMaxRows rows per call (few experts see more than 8 rows there) and of 16 above
 // (an expert with more slots than an item holds is streamed once per item, which beyond kStGatherMaxRows costs
 // more than the tensor-memory kernel's larger tiles).
-constexpr int kStGatherMaxRows = 512;
+constexpr int kStGatherMaxRows = TEAM_MAX_ROWS;
 constexpr int kStOneTileMaxRows = 64;
 bool experts_stream_supported(int max_rows, int hidden, int inter) {
   return max_rows <= kStGatherMaxRows && (hidden == 1024 || hidden == 2048) && inter % 16 == 0;
