@@ -1,29 +1,33 @@
-// Expert kernel for the few-rows regime (T <= 8 rows, bf16 weights): a weight-streaming kernel.
+// Weight-streaming expert kernel (bf16 weights, hidden size 1024 or 2048).
 //
-// With a handful of rows the SwiGLU experts (Eq. 1) are a matrix-vector problem: ~1 MB of weights per
-// SM and a few hundred kFLOP.  Staging tiles for the tensor-memory path costs more in hand-offs between
-// warps than the math is worth, so here every warp is its own pipeline: it copies 2 KB chunks of
-// weights from HBM into a private ring in shared memory with asynchronous copies, several chunks
-// ahead, and multiplies each chunk with the token rows using warp-level mma (m16n8k16: 16 weight rows
-// x 8 tokens).  No warp waits for another one inside a phase, and no CTA ever waits for another CTA.
+// With a handful of rows per expert the SwiGLU experts (Eq. 1) are a matrix-vector problem: ~1 MB of weights
+// per SM and a few hundred kFLOP.  Staging tiles for the tensor-memory path costs more in hand-offs between
+// warps than the math is worth, so here every warp is its own pipeline: it copies 2 KB chunks of weights from
+// HBM into a private ring in shared memory with asynchronous copies, several chunks ahead, and multiplies each
+// chunk with the token rows using warp-level mma (m16n8k16: 16 weight rows x 8 tokens).  No warp waits for
+// another one inside a phase, and no CTA ever waits for another CTA.
 //
-// Work partition: the intermediate dimension of every activated expert is cut into groups of 16
-// columns, the global list of groups into one contiguous range per CTA.  A group is self-contained:
-// its 16 gate rows and 16 up rows of W give 16 activations per token (phase 1), and those multiply
-// the group's slab of W_down, 16 columns of all H rows, stored contiguously ([I/16][H][16]), into a
-// partial y that is added to the output with fp32 reductions (phase 2).  Groups are handled in passes
-// of up to 8:
+// Work partition: the intermediate dimension of every activated expert (or work item of an expert) is cut
+// into groups of 16 columns, the global list of groups into one contiguous range per CTA.  A group is
+// self-contained: its 16 gate rows and 16 up rows of W give 16 activations per token (phase 1), and those
+// multiply the group's slab of W_down, 16 columns of all H rows, stored contiguously ([I/16][H][16]), into a
+// partial y that is added to the output with fp32 reductions (phase 2).  Groups are handled in passes of up
+// to 8 (4 with 16 token columns):
 //
 //   phase 1   warp = (gate | up tile of 16 rows) x (one of 8 slices of the hidden dimension), for every
 //             group of the pass in turn; chunk = 16 rows x 128 bytes; partial sums of a slice go to
 //             shared memory.
 //   barrier   sum the 8 slices, a = silu(gate) * up, round to bf16, keep in shared memory.
-//   phase 2   warp = H/16 consecutive output rows, for every group of the pass in turn; chunk = 64
-//             slab rows x 32 bytes; the accumulators stay in registers across the groups of one
+//   phase 2   warp = H/16 consecutive output rows, 64 at a time, for every group of the pass in turn;
+//             chunk = 64 slab rows x 32 bytes; the accumulators stay in registers across the groups of one
 //             expert and are scaled by the routing weights and added to y when the expert changes.
 //
-// A warp's copies run ahead across the barrier: while the slices are being summed, its first slab
-// chunks of phase 2 are already on their way.
+// A warp's copies run ahead across the barrier: while the slices are being summed, its first slab chunks of
+// phase 2 are already on their way.
+//
+// Token columns.  Up to 8 rows per call: the call's rows themselves, for every expert (weight 0 where a row
+// did not choose it), and the activated set is formed here from the rows' choices.  More rows: work items
+// of 8 or 16 token-slots of one expert, built by the selection kernel, gathered into shared memory per item.
 #include "team_common.cuh"
 
 namespace team {
