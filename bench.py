@@ -237,6 +237,8 @@ def main():
         code, detail = B.team_read_status(ctxs[combos[i][0]])
         if code != 0:
             raise SystemExit(f"device status {code} detail {detail}")
+    one_step(0)                                   # as the timed steps run: no exports
+    torch.cuda.synchronize()
     launches_per_step = B.team_last_launch_count(ctxs[0])
     bytes_per_expert = 3 * H * I * 2
 
