@@ -6,6 +6,8 @@
 //
 // Layout contract: rows with equal (group, branch) are contiguous (one decoding block, at most
 // TEAM_MAX_BLOCK rows), so the "distance to a decoded token" test of Eq. 4 only walks a row's own run.
+#include <cooperative_groups.h>
+
 #include <mutex>
 
 #include "team_common.cuh"
@@ -13,16 +15,19 @@
 
 namespace team {
 
+namespace cg = cooperative_groups;
+
 constexpr int kSelThreads = 1024;
 constexpr int kSelWarps = kSelThreads / 32;
 
 constexpr int kIdxInSmemMax = 8192;   // routed slots kept in shared memory between the rounds and the dispatch
-enum { kSelAll = 0, kSelRounds = 1, kSelDispatch = 2 };   // what one launch of the kernel does
+enum { kSelAll = 0, kSelRounds = 1, kSelDispatch = 2, kSelCluster = 3 };   // what one launch of the kernel does
 constexpr int kSmallSlots = 128;      // up to here every expert's thread counts and places its slots by itself
 
 struct SelSmem {
   // carved from dynamic shared memory in this order
   uint32_t* mask;      // [G][8]  E_A bits (256 experts max)
+  uint32_t* mask2;     // [G][8]  cluster mode: the union over the cluster's CTAs while it is being formed
   int32_t* hist;       // [kSelWarps][E+ns]
   int32_t* off;        // [E+ns+1]
   int32_t* key;        // [T] group*256 + branch
@@ -45,6 +50,7 @@ __host__ __device__ inline size_t sel_smem_layout(Dims d, SelSmem* s, unsigned c
   const int EN = d.E + d.ns;
   const int n_idx = d.T * d.k <= kIdxInSmemMax ? d.T * d.k : 0;
   size_t a_mask = take((size_t)d.G * 8 * 4);
+  size_t a_mask2 = take((size_t)d.G * 8 * 4);
   size_t a_hist = take((size_t)kSelWarps * EN * 4);
   size_t a_off = take((size_t)(EN + 1) * 4);
   size_t a_key = take((size_t)d.T * 4);
@@ -57,6 +63,7 @@ __host__ __device__ inline size_t sel_smem_layout(Dims d, SelSmem* s, unsigned c
   size_t a_hf = take((size_t)d.G);
   if (s != nullptr) {
     s->mask = reinterpret_cast<uint32_t*>(base + a_mask);
+    s->mask2 = reinterpret_cast<uint32_t*>(base + a_mask2);
     s->hist = reinterpret_cast<int32_t*>(base + a_hist);
     s->off = reinterpret_cast<int32_t*>(base + a_off);
     s->key = reinterpret_cast<int32_t*>(base + a_key);
@@ -93,7 +100,15 @@ k_select(const float* __restrict__ logits, StepPtrs st, Workspace ws, RoutePtrs 
   const bool one_row_per_warp = T <= kSelWarps && mode == kSelAll;
   // kSelRounds: CTA b of the grid routes the rows of the groups g with g % gridDim.x == b (the necessary set
   // E_A is per group, so groups are independent up to the dispatch); every CTA classifies all rows.
+  // kSelCluster: the grid is one thread-block cluster; CTA b routes the rows of the 32-row blocks b, b + C, ...,
+  // the CTAs' partial E_A sets are united through distributed shared memory between the rounds, and CTA 0
+  // goes on to the dispatch.
   const int nb = gridDim.x, cta = blockIdx.x;
+  auto own_row = [&](int t) {
+    if (mode == kSelRounds) return (s.key[t] >> 8) % nb == cta;
+    if (mode == kSelCluster) return (t >> 5) % nb == cta;
+    return true;
+  };
 
   // ---- stage the step state (inputs of the call, not produced by the preceding kernel) ---------
   for (int i = tid; i < d.G * n_words32; i += kSelThreads) s.mask[i] = 0u;
@@ -172,7 +187,7 @@ k_select(const float* __restrict__ logits, StepPtrs st, Workspace ws, RoutePtrs 
   // ---- Algorithm 1, round 1 (free top-k) then round 2 (top-k inside E_A) -------------------
   for (int round = 1; round <= 2 && mode != kSelDispatch; ++round) {
     for (int t = warp; t < T; t += kSelWarps) {
-      if (mode == kSelRounds && (s.key[t] >> 8) % nb != cta) continue;
+      if (!own_row(t)) continue;
       const uint8_t c = s.cls[t];
       if (round == 1 && c == TEAM_CLS_SKIP) {
         if (lane < k) {
@@ -231,12 +246,25 @@ k_select(const float* __restrict__ logits, StepPtrs st, Workspace ws, RoutePtrs 
       }
     }
     __syncthreads();
+    if (mode == kSelCluster && round == 1) {
+      // every group's E_A = union of what the cluster's CTAs collected from their own first-round rows
+      cg::cluster_group cluster = cg::this_cluster();
+      cluster.sync();
+      for (int i = tid; i < d.G * n_words32; i += kSelThreads) {
+        uint32_t m = 0u;
+        for (int rr = 0; rr < nb; ++rr) m |= cluster.map_shared_rank(s.mask, rr)[i];
+        s.mask2[i] = m;
+      }
+      cluster.sync();                   // nobody reads a peer's partial set after this
+      for (int i = tid; i < d.G * n_words32; i += kSelThreads) s.mask[i] = s.mask2[i];
+      __syncthreads();
+    }
   }
   const int32_t* idx_src = s.idx ? s.idx : r.topk_idx;
 
   // ---- exports that need no further work: by the upper half of the CTA, beside the dispatch below ----
   for (int t = tid - kSelThreads / 2; t >= 0 && t < T && mode != kSelDispatch; t += kSelThreads / 2) {
-    if (mode == kSelRounds && (s.key[t] >> 8) % nb != cta) continue;
+    if (!own_row(t)) continue;
     r.tok_class[t] = s.cls[t];
     if (ex.tok_class) ex.tok_class[t] = s.cls[t];
   }
@@ -244,7 +272,7 @@ k_select(const float* __restrict__ logits, StepPtrs st, Workspace ws, RoutePtrs 
     const int n_words64 = (E + 63) / 64;
     for (int i = tid - kSelThreads / 2; i >= 0 && i < d.G * n_words64 && mode != kSelDispatch; i += kSelThreads / 2) {
       const int g = i / n_words64, wd = i % n_words64;
-      if (mode == kSelRounds && g % nb != cta) continue;
+      if ((mode == kSelRounds && g % nb != cta) || (mode == kSelCluster && cta != 0)) continue;
       const uint64_t m = (uint64_t)s.mask[g * n_words32 + 2 * wd] | ((uint64_t)s.mask[g * n_words32 + 2 * wd + 1] << 32);
       r.group_mask[i] = m;
       if (ex.group_mask) ex.group_mask[i] = m;
@@ -254,6 +282,14 @@ k_select(const float* __restrict__ logits, StepPtrs st, Workspace ws, RoutePtrs 
   // The dispatch tables are skipped when nobody reads them: no export asked for, and an expert kernel that
   // works from the rows' choices alone (at most 8 rows, all resident).
   if (mode == kSelRounds || skip_dispatch) return;
+  if (mode == kSelCluster) {
+    // all CTAs' choices are in the routing tables and visible; CTA 0 alone builds the dispatch tables from them
+    cg::this_cluster().sync();
+    if (cta != 0) return;
+    if (s.idx)
+      for (int i = tid; i < S; i += kSelThreads) s.idx[i] = __ldcg(r.topk_idx + i);
+    __syncthreads();
+  }
 
   // ---- dispatch: stable counting sort of slots by expert ------------------------------------
   // Small steps (at most kSmallSlots routed slots): expert e's thread counts its slots by walking the
@@ -498,8 +534,24 @@ cudaError_t launch_select(const float* logits, StepPtrs st, Workspace ws, RouteP
   cfg.numAttrs = 1;
   // Several groups and more rows than one CTA routes at once (one row per warp): the routing rounds run as
   // one CTA per group (up to 32), the dispatch as a second single-CTA launch.
+  const int group_ctas = d.G < 32 ? d.G : 32;
+  if (d.T > kSelWarps && (d.G == 1 || d.T / group_ctas > kSelWarps)) {
+    // one group, or groups of more rows than a CTA routes at once: one cluster, rows split over its CTAs
+    int c = (d.T + kSelWarps - 1) / kSelWarps;
+    c = c >= 8 ? 8 : (c >= 4 ? 4 : 2);
+    cfg.gridDim = dim3(c);
+    cudaLaunchAttribute attrs[2];
+    attrs[0] = attr;
+    attrs[1].id = cudaLaunchAttributeClusterDimension;
+    attrs[1].val.clusterDim.x = c;
+    attrs[1].val.clusterDim.y = 1;
+    attrs[1].val.clusterDim.z = 1;
+    cfg.attrs = attrs;
+    cfg.numAttrs = 2;
+    return cudaLaunchKernelEx(&cfg, k_select, logits, st, ws, ex, d, p, item_tile, 1, (int)kSelCluster, 0);
+  }
   if (d.G > 1 && d.T > kSelWarps) {
-    cfg.gridDim = dim3(d.G < 32 ? d.G : 32);
+    cfg.gridDim = dim3(group_ctas);
     cudaError_t e = cudaLaunchKernelEx(&cfg, k_select, logits, st, ws, ex, d, p, item_tile, 1, (int)kSelRounds, 0);
     if (e != cudaSuccess) return e;
     cfg.gridDim = dim3(1);
@@ -508,6 +560,10 @@ cudaError_t launch_select(const float* logits, StepPtrs st, Workspace ws, RouteP
   return cudaLaunchKernelEx(&cfg, k_select, logits, st, ws, ex, d, p, item_tile, 1, (int)kSelAll, need_tables ? 0 : 1);
 }
 
-int select_launches(Dims d) { return d.G > 1 && d.T > kSelWarps ? 2 : 1; }
+int select_launches(Dims d) {
+  const int group_ctas = d.G < 32 ? d.G : 32;
+  if (d.T > kSelWarps && (d.G == 1 || d.T / group_ctas > kSelWarps)) return 1;
+  return d.G > 1 && d.T > kSelWarps ? 2 : 1;
+}
 
 }  // namespace team

@@ -87,7 +87,8 @@ def test_few_rows_kernel_gather_mode_with_split_items(flags, weights_cache):
 def test_few_rows_kernel_gather_mode_items_of_16_slots(flags, weights_cache):
     shape = W.STREAM_GATHER16                    # 80 rows in 2 groups: items of 16 slots, the shared expert has five
     stats = P.run_schedule(shape, weights_cache(shape), W.make_schedule(shape), flags)
-    assert len(stats) == 4 and all(s["launches"] == 4 for s in stats)
+    # 40 rows per group are more than a CTA routes at once: the selection is one launch of a 2-CTA cluster
+    assert len(stats) == 4 and all(s["launches"] == 3 for s in stats)
 
 
 @pytest.mark.parametrize("flags", [0, 3])
