@@ -97,18 +97,21 @@ k_select(const float* __restrict__ logits, StepPtrs st, Workspace ws, RoutePtrs 
   const int S = T * k;
   // warps taking part in the dispatch walk: enough for 32 slots each, so small steps scan little
   const int nw = min(kSelWarps, (S + 31) / 32);
-  const bool one_row_per_warp = T <= kSelWarps && mode == kSelAll;
   // kSelRounds: CTA b of the grid routes the rows of the groups g with g % gridDim.x == b (the necessary set
   // E_A is per group, so groups are independent up to the dispatch); every CTA classifies all rows.
-  // kSelCluster: the grid is one thread-block cluster; CTA b routes the rows of the 32-row blocks b, b + C, ...,
-  // the CTAs' partial E_A sets are united through distributed shared memory between the rounds, and CTA 0
-  // goes on to the dispatch.
+  // kSelCluster: the grid is one thread-block cluster; CTA b routes a contiguous block of ceil(T / C) rows
+  // (routing 32 rows at once is bound by one SM's issue rate, so the rows are spread over SMs), the CTAs'
+  // partial E_A sets are united through distributed shared memory between the rounds, and CTA 0 goes on to the
+  // dispatch.
   const int nb = gridDim.x, cta = blockIdx.x;
+  const int rows_per_cta = mode == kSelCluster ? (T + nb - 1) / nb : T;
+  const int t0 = mode == kSelCluster ? min(T, cta * rows_per_cta) : 0, t1 = min(T, t0 + rows_per_cta);
   auto own_row = [&](int t) {
     if (mode == kSelRounds) return (s.key[t] >> 8) % nb == cta;
-    if (mode == kSelCluster) return (t >> 5) % nb == cta;
-    return true;
+    return t >= t0 && t < t1;
   };
+  // at most one row per warp: the row's logits are fetched once and stay in registers through both rounds
+  const bool one_row_per_warp = (mode == kSelAll || mode == kSelCluster) && t1 - t0 <= kSelWarps;
 
   // ---- stage the step state (inputs of the call, not produced by the preceding kernel) ---------
   for (int i = tid; i < d.G * n_words32; i += kSelThreads) s.mask[i] = 0u;
@@ -175,7 +178,7 @@ k_select(const float* __restrict__ logits, StepPtrs st, Workspace ws, RoutePtrs 
   // both routing rounds.
   float keep[kMaxPerLane];
   float keep_max = 0.f, keep_denom = 1.f;
-  if (one_row_per_warp && warp < T) load_row(logits + (size_t)warp * E, E, lane, keep, keep_max, keep_denom);
+  if (one_row_per_warp && t0 + warp < t1) load_row(logits + (size_t)(t0 + warp) * E, E, lane, keep, keep_max, keep_denom);
   if (mode == kSelDispatch) {
     // classes and choices were left in the routing tables by the kSelRounds grid
     for (int t = tid; t < T; t += kSelThreads) s.cls[t] = __ldcg(r.tok_class + t);
@@ -186,7 +189,7 @@ k_select(const float* __restrict__ logits, StepPtrs st, Workspace ws, RoutePtrs 
 
   // ---- Algorithm 1, round 1 (free top-k) then round 2 (top-k inside E_A) -------------------
   for (int round = 1; round <= 2 && mode != kSelDispatch; ++round) {
-    for (int t = warp; t < T; t += kSelWarps) {
+    for (int t = t0 + warp; t < t1; t += kSelWarps) {
       if (!own_row(t)) continue;
       const uint8_t c = s.cls[t];
       if (round == 1 && c == TEAM_CLS_SKIP) {
@@ -537,8 +540,7 @@ cudaError_t launch_select(const float* logits, StepPtrs st, Workspace ws, RouteP
   const int group_ctas = d.G < 32 ? d.G : 32;
   if (d.T > kSelWarps && (d.G == 1 || d.T / group_ctas > kSelWarps)) {
     // one group, or groups of more rows than a CTA routes at once: one cluster, rows split over its CTAs
-    int c = (d.T + kSelWarps - 1) / kSelWarps;
-    c = c >= 8 ? 8 : (c >= 4 ? 4 : 2);
+    const int c = d.T > 64 ? 8 : 4;        // 16 rows or fewer per CTA up to 128 rows
     cfg.gridDim = dim3(c);
     cudaLaunchAttribute attrs[2];
     attrs[0] = attr;
