@@ -27,6 +27,16 @@ k_router_logits(const XT* __restrict__ x, const float* __restrict__ w_router, co
   const int nt = min(kRowTile, d.T - t0);
   const int tid = threadIdx.x;
   const int H = d.H;
+  // this warp's expert: the first batch of its weight row is requested before anything else
+  const int warp = tid >> 5, lane = tid & 31;
+  const int e = blockIdx.x * kExpertsPerCta + warp;
+  const float4* wrow = reinterpret_cast<const float4*>(w_router + (size_t)min(e, d.E - 1) * H);
+  const int n4 = H >> 2;
+  constexpr int kBatch = 8;             // float4 per lane and batch: 4 KB of the row per warp in flight
+  float4 wv[kBatch];
+#pragma unroll
+  for (int i = 0; i < kBatch; ++i)
+    wv[i] = lane + 32 * i < n4 ? __ldg(wrow + lane + 32 * i) : make_float4(0.f, 0.f, 0.f, 0.f);
 
   if constexpr (sizeof(XT) == 2) {
     const uint2* src = reinterpret_cast<const uint2*>(x + (size_t)t0 * H);
@@ -54,25 +64,35 @@ k_router_logits(const XT* __restrict__ x, const float* __restrict__ w_router, co
   }
   __syncthreads();
 
-  const int warp = tid >> 5, lane = tid & 31;
-  const int e = blockIdx.x * kExpertsPerCta + warp;
   if (e >= d.E) return;
-  const float4* wrow = reinterpret_cast<const float4*>(w_router + (size_t)e * H);
   float acc[kRowTile];
 #pragma unroll
   for (int r = 0; r < kRowTile; ++r) acc[r] = 0.f;
-  const int n4 = H >> 2;
-#pragma unroll 4
-  for (int c = lane; c < n4; c += 32) {
-    const float4 w = __ldg(wrow + c);
+  // batches of kBatch float4 per lane; the next batch is requested before the current one is used
+  // (the summation order over c is unchanged: ascending c within a lane)
+  for (int base = 0; base < n4; base += 32 * kBatch) {
+    float4 wn[kBatch];
+    const int nbase = base + 32 * kBatch;
 #pragma unroll
-    for (int r = 0; r < kRowTile; ++r) {
-      const float4 xv = *reinterpret_cast<const float4*>(s_x + r * H + c * 4);
-      acc[r] = fmaf(w.x, xv.x, acc[r]);
-      acc[r] = fmaf(w.y, xv.y, acc[r]);
-      acc[r] = fmaf(w.z, xv.z, acc[r]);
-      acc[r] = fmaf(w.w, xv.w, acc[r]);
+    for (int i = 0; i < kBatch; ++i)
+      wn[i] = nbase + lane + 32 * i < n4 ? __ldg(wrow + nbase + lane + 32 * i) : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+    for (int i = 0; i < kBatch; ++i) {
+      const int c = base + lane + 32 * i;
+      if (c < n4) {
+        const float4 w = wv[i];
+#pragma unroll
+        for (int r = 0; r < kRowTile; ++r) {
+          const float4 xv = *reinterpret_cast<const float4*>(s_x + r * H + c * 4);
+          acc[r] = fmaf(w.x, xv.x, acc[r]);
+          acc[r] = fmaf(w.y, xv.y, acc[r]);
+          acc[r] = fmaf(w.z, xv.z, acc[r]);
+          acc[r] = fmaf(w.w, xv.w, acc[r]);
+        }
+      }
     }
+#pragma unroll
+    for (int i = 0; i < kBatch; ++i) wv[i] = wn[i];
   }
 #pragma unroll
   for (int r = 0; r < kRowTile; ++r) {
