@@ -90,6 +90,10 @@ STREAM_GATHER = Shape("stream_gather_bf16", 1024, 48, 8, 512, 1, "bf16", 12, 4, 
 # Enough rows per call that the gather mode works on items of 16 token-slots (two token tiles per weight fragment).
 STREAM_GATHER16 = Shape("stream_gather16_bf16", 1024, 48, 8, 512, 1, "bf16", 40, 4, 6, 1, 3, 0.7, seqs=2, seed=16)
 
+# The limits of the resident mode: 8 rows x top-16 = 128 slots, 256 routed experts + 2 shared ones (a bit set
+# of 258 bits), narrow experts (8 column groups each).
+STREAM_WIDE = Shape("stream_k16_e256_bf16", 1024, 256, 16, 128, 2, "bf16", 8, 3, 2, 1, 2, 0.7, seed=18)
+
 def round_to_bf16(a):
     """Round fp32 values to the nearest bf16-representable value (ties to even); returns fp32."""
     a = np.ascontiguousarray(a, dtype=np.float32)

@@ -77,6 +77,13 @@ def test_few_rows_kernel_multi_pass_ranges_and_shared_expert(flags, weights_cach
 
 
 @pytest.mark.parametrize("flags", [0, 3])
+def test_few_rows_kernel_resident_mode_at_its_limits(flags, weights_cache):
+    shape = W.STREAM_WIDE                        # 128 slots, 258 experts: every word of the activated bit set is used
+    stats = P.run_schedule(shape, weights_cache(shape), W.make_schedule(shape), flags)
+    assert len(stats) == 3
+
+
+@pytest.mark.parametrize("flags", [0, 3])
 def test_few_rows_kernel_gather_mode_with_split_items(flags, weights_cache):
     shape = W.STREAM_GATHER                      # 24 rows: the shared expert alone has three items of 8 slots
     stats = P.run_schedule(shape, weights_cache(shape), W.make_schedule(shape), flags)
@@ -217,7 +224,7 @@ def _host_entry_schedule(shape, flags, steps, weights_cache):
         layer_b.close()
 
 
-@pytest.mark.parametrize("shape", [W.C2, W.STREAM_MULTI], ids=lambda s: s.name)
+@pytest.mark.parametrize("shape", [W.C2, W.STREAM_MULTI, W.STREAM_WIDE], ids=lambda s: s.name)
 def test_forward_without_exports_skips_the_dispatch_tables_and_gives_the_same_y(shape, weights_cache):
     """With at most 8 rows and no table asked for, the selection stops after the routing rounds and the expert
     kernel works from the rows' choices; y must not depend on that."""
