@@ -92,6 +92,20 @@ __device__ __forceinline__ void st_mma(float (&d)[4], const uint32_t (&a)[4], ui
                : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
 
+// Position of the n-th (0-based) set bit of m; popcount(m) > n.  Five halvings instead of a bit-by-bit walk.
+__device__ __forceinline__ int st_nth_set_bit(uint32_t m, int n) {
+  int pos = 0;
+#pragma unroll
+  for (int width = 16; width >= 1; width >>= 1) {
+    const int c = __popc(m & (((1u << width) - 1u) << pos));
+    if (n >= c) {
+      n -= c;
+      pos += width;
+    }
+  }
+  return pos;
+}
+
 // shared memory: token rows | partial sums [group][slice][gate, up][16 rows][tokens] | per-warp rings.
 // ntl = token tiles of 8 (1 or 2): with 16 tokens a pass holds half the groups and a ring one slot less.
 __host__ __device__ inline int stream_slots(int ntl) { return ntl == 1 ? kStSlots : kStSlots - 1; }
@@ -219,7 +233,7 @@ __global__ void __launch_bounds__(kStThreads, 1) k_experts_stream(StArgs a) {
       for (int w = 0; w < n_words; ++w) {
         const uint32_t m = __shfl_sync(0xffffffffu, act_word, w);
         const int c = __popc(m);
-        if (left >= 0 && left < c) my_e = w * 32 + (int)__fns(m, 0, left + 1);
+        if (left >= 0 && left < c) my_e = w * 32 + st_nth_set_bit(m, left);
         left = left >= c ? left - c : -1;
       }
     }
