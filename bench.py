@@ -51,6 +51,17 @@ def parse_args():
     return ap.parse_args()
 
 
+def sm_max_hz():
+    """Maximum SM clock in Hz (for sizing the device-side delay); 1.965 GHz if NVML is not there."""
+    try:
+        import pynvml
+        pynvml.nvmlInit()
+        h = pynvml.nvmlDeviceGetHandleByIndex(int(os.environ.get("LOCAL_RANK", "0")))
+        return pynvml.nvmlDeviceGetMaxClockInfo(h, pynvml.NVML_CLOCK_SM) * 1e6
+    except Exception:
+        return 1.965e9
+
+
 def measured_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -296,9 +307,15 @@ def main():
         # ---- expert-kernel duration (CUDA events around every launch, on the launching stream) -------
         for c in ctxs:
             B.team_expert_timing(c, 1)
-        n_roof = min(args.steps, 50 * period)
+        # These steps are plain launches with event records in between: about five stream operations per step.
+        # A host slower than the GPU would leave the GPU waiting between the first event and the kernel, and that
+        # wait would be counted as kernel time.  So the stream is held back for a moment (a bounded device-side
+        # spin) while the host queues the whole batch, and the batch is kept below the launch queue's depth.
+        n_roof = min(args.steps, 18 * period)
         n_roof -= n_roof % period
         n_roof = max(n_roof, period)
+        torch.cuda.synchronize()
+        torch.cuda._sleep(int(sm_max_hz() * 0.012))            # ~12 ms; the host needs a few ms for the batch
         for i in range(n_roof):
             one_step(i)
         tot_ms, tot_n = 0.0, 0
