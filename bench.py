@@ -387,8 +387,8 @@ def main():
                      "frac_of_8TBs_nominal": achieved / 8000.0, "kernel_ms": kernel_ms,
                      "algorithmic_bytes_per_launch": algo_bytes, "launches_timed": tot_n,
                      # DRAM read + write bytes per launch: ncu capture at 16 activated experts (151.08 MB read +
-                     # 3.3 MB written, profiles/experts_stream_c2_bench.md), scaled to this run's mean
-                     "traffic": mean_act * (151.08e6 + 3.3e6) / 16.0 if args.workload == "c2" else None,
+                     # 3.25 MB written, profiles/experts_stream_c2_bench.md), scaled to this run's mean
+                     "traffic": mean_act * (151.08e6 + 3.25e6) / 16.0 if args.workload == "c2" else None,
                      # the same launches as a contraction: 6 H I flops per token-slot (routed and shared)
                      "tensor_tflops": mean_rows * (k + ns) * 6.0 * H * I / (kernel_ms * 1e-3) / 1e12},
     }
