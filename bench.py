@@ -1,19 +1,23 @@
 #!/usr/bin/env python
 """Benchmark of the TEAM MoE-layer step on B200.
 
-Workload: the SDAR-30B-A3B-shaped MoE layer (hidden 2048, 128 experts top-8, SwiGLU intermediate 768,
-bf16 weights, fp32 router), batch 1, block of 4 tokens, the scripted 4-step denoising schedule (one
-token accepted per step), TEAM's activation rule on (delayed caching + limited activation).  One
-"step" is one pass of the whole hot path -- router, selection/dispatch, grouped SwiGLU experts,
-weighted combine -- i.e. one call of team_moe_forward for one denoising step of one layer.  Successive
-steps cycle through the 4 denoising steps and through R independent layers (R sets of weights,
-~1.2 GB each) so that expert weights always come from HBM, never from L2.
+Headline workload (the default): the SDAR-30B-A3B-shaped MoE layer (hidden 2048, 128 experts top-8, SwiGLU
+intermediate 768, bf16 weights, fp32 router), batch 1, block of 4 tokens, the scripted 4-step denoising
+schedule (one token accepted per step), TEAM's activation rule on (delayed caching + limited activation).
+One "step" is one pass of the whole hot path -- router, selection/dispatch, grouped SwiGLU experts, weighted
+combine -- i.e. one call of team_moe_forward for one denoising step of one layer.  Successive steps cycle
+through the 4 denoising steps and through R independent layers (R sets of weights, ~1.2 GB each) so that expert
+weights always come from HBM, never from L2.
 
-Prints ONE JSON line (rank 0).  `value` = rows presented per second over all GPUs, inputs resident in
-HBM; `e2e` = the same through the C ABI with host buffers (pinned host -> device copies of the step's
-inputs and a device -> host read of y inside the timed region); `roofline` = the expert kernel's
-achieved HBM bandwidth on activated-expert weight bytes; `cpu_baseline` = the oracle on host cores.
-`--impl reference` times the oracle instead (it is the reference arm for this build).
+Prints ONE JSON line (rank 0).  `value` = rows presented per second over all GPUs, inputs resident in HBM;
+`e2e` = the same through the C ABI with host buffers (pinned host -> device copies of the step's inputs and a
+device -> host read of y inside the timed region); `roofline` = the expert kernel's achieved HBM bandwidth on
+activated-expert weight bytes, with the whole step's fraction beside it; `cpu_baseline` = the oracle on host
+cores.  `--impl reference` times the oracle instead (it is the reference arm here: there is no reference code).
+
+Other workloads: `--workload c3 | c4 --seqs N | paper` time the larger layer configurations the same way;
+`--workload c5` runs the 48-layer MoE-only stack through the 4-step block loop for `--blocks` blocks, once with
+TEAM's selection and once with vanilla top-k.  `--gpus N` without a launcher starts N replicas itself.
 """
 import argparse
 import json
@@ -33,22 +37,26 @@ METRIC = "MoE-layer tokens/s per denoising step (rows presented / s)"
 UNIT = "tokens/s"
 WORKLOAD = "c2_sdar_bf16: H2048 E128 top8 I768 bf16, batch 1 x block 4, 4 denoising steps, TEAM (DCD|LAC)"
 TEAM_FLAGS = 3
+L2_NOTE = "inputs larger than L2: expert weights rotate over independent layers (GPU arm); the CPU oracle arm uses one layer"
 
 
-def parse_args():
+def parse_args(argv=None):
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=8000)
     ap.add_argument("--warmup", type=int, default=400)
     ap.add_argument("--impl", default="team", choices=["team", "reference"])
-    ap.add_argument("--layers", type=int, default=8, help="independent weight sets cycled through (L2 defeat)")
+    ap.add_argument("--layers", type=int, default=None,
+                    help="independent weight sets: cycled through by the layer workloads (default 8), depth of the c5 stack (default 48)")
     ap.add_argument("--flags", type=int, default=TEAM_FLAGS, help="0 vanilla, 1 DCD, 3 DCD|LAC")
     ap.add_argument("--no-graph", action="store_true", help="issue every step as separate calls (no CUDA graph)")
     ap.add_argument("--cpu-seconds", type=float, default=15.0, help="budget of the oracle baseline leg")
-    ap.add_argument("--workload", default="c2", choices=["c2", "c3", "c4", "paper"],
-                    help="c2: the headline step (default); c3: 256 experts + shared, block 32; c4: c2 shape, --seqs x 4 branches x 4; paper: c2 shape, block 32 x 4 branches in one group")
+    ap.add_argument("--workload", default="c2", choices=["c2", "c3", "c4", "paper", "c5"],
+                    help="c2: the headline step (default); c3: 256 experts + shared, block 32; c4: c2 shape, --seqs x 4 "
+                         "branches x 4; paper: c2 shape, block 32 x 4 branches in one group; c5: stack of c2 layers, block loop")
     ap.add_argument("--seqs", type=int, default=1, help="sequences of the c4 batch sweep")
-    return ap.parse_args()
+    ap.add_argument("--blocks", type=int, default=64, help="decoding blocks of the c5 stack run")
+    return ap.parse_args(argv)
 
 
 def sm_max_hz():
@@ -63,12 +71,13 @@ def sm_max_hz():
 
 
 def measured_peaks():
+    """(HBM GB/s, bf16 TFLOP/s burst, sustained, kind) from the measured-peaks file, else the pool's earlier figures."""
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
         with open(path) as f:
             p = json.load(f)
-        return float(p["hbm_gbs"]), "measured"
-    return 6650.0, "fallback"
+        return float(p["hbm_gbs"]), float(p.get("bf16_tflops", 1590.0)), float(p.get("bf16_tflops_sustained", 1400.0)), "measured"
+    return 6650.0, 1590.0, 1400.0, "fallback"
 
 
 class ClockSampler:
@@ -126,27 +135,43 @@ class ClockSampler:
                 "samples": len(self.samples)}
 
 
-def oracle_leg(args, shape, weights_host, steps, budget_s):
-    """Times the oracle, as it stands, on the host cores over a bounded sample of the same workload."""
+def workload_of(args):
+    """(shape, workload string) of a layer workload."""
+    from paper_2602_08404_b200 import workloads as W
+    shape = {"c2": W.C2, "c3": W.C3, "c4": W.c4(args.seqs), "paper": W.paper_point(), "c5": W.C2}[args.workload]
+    if args.workload == "c2" and args.flags == TEAM_FLAGS:
+        return shape, WORKLOAD
+    ns = shape.n_shared
+    return shape, (f"{shape.name}: H{shape.hidden} E{shape.n_experts}{'+%d shared' % ns if ns else ''} top{shape.top_k} "
+                   f"I{shape.inter} bf16, {shape.seqs} seq x {shape.branches} branches x block {shape.block} = {shape.rows} "
+                   f"rows, {shape.n_steps} denoising steps, flags {args.flags}")
+
+
+def config_of(args, shape, workload):
+    """The workload's description: the same dictionary in the GPU arm and in the reference (oracle) arm."""
+    return {"workload": workload, "flags": args.flags, "rows_presented": shape.rows, "l2": L2_NOTE,
+            "parallelism": "replicas (one process per GPU, no exchange on the data path)"}
+
+
+def oracle_leg(args, shape, weights_host, steps, budget_s, threads=None):
+    """Times the oracle, as it stands, on the host cores over a bounded sample of the same workload.
+    threads=None: whatever numpy's BLAS uses by default (all cores); threads=1: one thread."""
     from oracle import team_oracle as O
     from tests import _parity as P
-    try:
-        from threadpoolctl import threadpool_info
-        cores = max([p.get("num_threads", 1) for p in threadpool_info()] or [1])
-    except Exception:
-        cores = len(os.sched_getaffinity(0))
+    from threadpoolctl import threadpool_info, threadpool_limits
     ocfg = P.oracle_config(shape, args.flags)
     t_total, n = 0.0, 0
     y_prev = None
-    while t_total < budget_s and n < 400:
-        step = steps[n % len(steps)]
-        t0 = time.perf_counter()
-        y_prev, _ = O.moe_forward(ocfg, weights_host, step["x"], step["tok_state"], step["conf"], step["pos"],
-                                  step["group"], step["branch"], y_prev=y_prev if n % len(steps) else None)
-        t_total += time.perf_counter() - t0
-        n += 1
-    rows = shape.rows
-    return {"value": rows * n / t_total, "unit": UNIT, "cores": cores, "kind": "oracle",
+    with threadpool_limits(limits=threads):
+        cores = max([p.get("num_threads", 1) for p in threadpool_info()] or [1])
+        while t_total < budget_s and n < 400:
+            step = steps[n % len(steps)]
+            t0 = time.perf_counter()
+            y_prev, _ = O.moe_forward(ocfg, weights_host, step["x"], step["tok_state"], step["conf"], step["pos"],
+                                      step["group"], step["branch"], y_prev=y_prev if n % len(steps) else None)
+            t_total += time.perf_counter() - t0
+            n += 1
+    return {"value": shape.rows * n / t_total, "unit": UNIT, "cores": cores, "kind": "oracle",
             "sample": f"{n} layer-steps of the same schedule on one layer's weights ({t_total:.1f} s of CPU time)"}, \
         t_total / n
 
@@ -157,7 +182,7 @@ def run_reference(args):
     if rank != 0:
         return
     from paper_2602_08404_b200 import workloads as W
-    shape = W.C2
+    shape, workload = workload_of(args)
     weights = W.make_weights(shape)
     steps = W.make_schedule(shape)
     budget = max(5.0, min(120.0, 0.05 * (args.steps + args.warmup)))
@@ -165,24 +190,17 @@ def run_reference(args):
     line = {"impl": "reference", "metric": METRIC, "value": cb["value"], "unit": UNIT, "n_gpus": 0,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": s_per_step * 1e3,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
-            "data": "synthetic", "config": {"workload": WORKLOAD, "flags": args.flags},
+            "data": "synthetic", "config": config_of(args, shape, workload),
             "cpu_baseline": cb,
             "e2e": {"value": cb["value"], "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
     print(json.dumps(line))
 
 
-def main():
-    args = parse_args()
-    if args.impl == "reference":
-        return run_reference(args)
-
+def init_device(args):
+    """Process group (if launched as several ranks), device, library build.  Returns (world, rank, device)."""
     import torch
     import torch.distributed as dist
-    from paper_2602_08404_b200 import binding as B
-    from paper_2602_08404_b200 import replicas as R_
     from paper_2602_08404_b200 import build as build_mod
-    from paper_2602_08404_b200 import workloads as W
-
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
@@ -195,26 +213,29 @@ def main():
         build_mod.build()
     if world > 1:
         dist.barrier()
-    dev = torch.device("cuda", local_rank)
+    return world, rank, torch.device("cuda", local_rank)
 
-    shape = {"c2": W.C2, "c3": W.C3, "c4": W.c4(args.seqs), "paper": W.paper_point()}[args.workload]
+
+def run_layer(args):
+    """The layer workloads (c2 headline, c3, c4, paper)."""
+    import torch
+    import torch.distributed as dist
+    from paper_2602_08404_b200 import binding as B
+    from paper_2602_08404_b200 import replicas as R_
+    from paper_2602_08404_b200 import workloads as W
+
+    world, rank, dev = init_device(args)
+    shape, workload = workload_of(args)
     T, H, E, k, I = shape.rows, shape.hidden, shape.n_experts, shape.top_k, shape.inter
     ns = shape.n_shared
-    workload = WORKLOAD if args.workload == "c2" else (
-        f"{shape.name}: H{H} E{E}{'+%d shared' % ns if ns else ''} top{k} I{I} bf16, {shape.seqs} seq x {shape.branches} "
-        f"branches x block {shape.block} = {T} rows, {shape.n_steps} denoising steps, flags {args.flags}")
     steps_host = W.make_schedule(shape)                      # the scripted denoising steps, seeded
     n_sched = len(steps_host)
-    R = args.layers
+    R = args.layers or 8
 
     # R independent layers, generated on the device (seeded); layer 0 also goes to the host for the oracle leg
-    gen = torch.Generator(device=dev)
     layers, packed = [], []
     for r in range(R):
-        gen.manual_seed(1000 + r)
-        wr = (torch.randn((E, H), generator=gen, device=dev, dtype=torch.float32) * 0.02).contiguous()
-        wg, wu, wd = [(torch.randn(s, generator=gen, device=dev, dtype=torch.float32) * 0.02).to(torch.bfloat16)
-                      for s in ((E + ns, I, H), (E + ns, I, H), (E + ns, H, I))]
+        wr, wg, wu, wd = W.device_layer_weights(shape, 1000 + r, dev)
         layers.append((wr, wg, wu, wd if r == 0 else None))
         packed.append(B.team_pack_w_down(wd))      # the layout the library reads; row-major kept for the oracle leg
     cfg = B.make_config(H, E, k, I, ns, max_rows=T, max_groups=shape.seqs, dtype=B.TEAM_DTYPE_BF16, flags=args.flags,
@@ -253,8 +274,17 @@ def main():
     launches_per_step = B.team_last_launch_count(ctxs[0])
     bytes_per_expert = 3 * H * I * 2
 
-    # CUDA graph of one full cycle (period steps); replayed for the timed region
-    graph = None
+    # CUDA graphs: one full cycle (period steps), and the remainder of the timed region (steps % period), so that
+    # the timed region consists of graph replays only, whatever --steps is
+    def capture(n):
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            for i in range(n):
+                one_step(i)
+        return g
+
+    graph = tail_graph = None
+    n_tail = args.steps % period
     if not args.no_graph:
         try:
             side = torch.cuda.Stream(device=dev)
@@ -264,25 +294,27 @@ def main():
                     one_step(i)
             torch.cuda.current_stream().wait_stream(side)
             torch.cuda.synchronize()
-            g = torch.cuda.CUDAGraph()
-            with torch.cuda.graph(g):
-                for i in range(period):
-                    one_step(i)
-            graph = g
+            graph = capture(period)
+            tail_graph = capture(n_tail) if n_tail else None
         except Exception as e:                                   # report, and time plain launches instead
             print(f"[bench] CUDA graph capture failed ({e}); timing plain launches", file=sys.stderr)
-            graph = None
+            graph = tail_graph = None
 
     def run_steps(n):
-        """Issues exactly n steps: whole cycles as graph replays, the remainder as plain calls."""
+        """Issues exactly n steps: whole cycles as graph replays, the remainder as one more replay (n % period ==
+        steps % period) or as plain calls."""
         if graph is None:
             for i in range(n):
                 one_step(i)
             return n
         for _ in range(n // period):
             graph.replay()
-        for i in range(n % period):
-            one_step(i)
+        if n % period:
+            if tail_graph is not None and n % period == n_tail:
+                tail_graph.replay()
+            else:
+                for i in range(n % period):
+                    one_step(i)
         return n
 
     def barrier():
@@ -290,10 +322,16 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
-    sampler = ClockSampler(local_rank)
+    sampler = ClockSampler(dev.index)
     with sampler:
         # ---- device-resident timing -----------------------------------------------------------------
-        run_steps(max(args.warmup, 3))
+        # Untimed, whatever --warmup says: every graph replayed at least twice, every context called, and at least
+        # ~20 ms of the workload so that the clocks have settled.  Then the caller's warm-up steps.
+        warm = 0
+        for _ in range(2):
+            warm += run_steps(period + n_tail)
+        warm += run_steps(max(args.warmup, 3))
+        warm += run_steps(period * max(0, (600 - warm + period - 1) // period))
         barrier()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record()
@@ -311,7 +349,7 @@ def main():
         # A host slower than the GPU would leave the GPU waiting between the first event and the kernel, and that
         # wait would be counted as kernel time.  So the stream is held back for a moment (a bounded device-side
         # spin) while the host queues the whole batch, and the batch is kept below the launch queue's depth.
-        n_roof = min(args.steps, 18 * period)
+        n_roof = max(period, min(18 * period, 144))
         n_roof -= n_roof % period
         n_roof = max(n_roof, period)
         torch.cuda.synchronize()
@@ -347,7 +385,10 @@ def main():
         # legacy default stream cannot do
         e2e_stream = torch.cuda.Stream(device=dev)
         with torch.cuda.stream(e2e_stream):
-            for i in range(max(3, min(args.warmup, 100))):
+            # untimed: every context allocates its staging block and records its step on its first call, so every
+            # context is called (twice) before the clock starts, whatever --warmup says
+            e2e_warm = max(2 * period, min(args.warmup, 200))
+            for i in range(e2e_warm):
                 e2e_step(i)
             barrier()
             t0 = time.perf_counter()
@@ -362,48 +403,231 @@ def main():
     mean_act = float(np.mean(n_act))
     mean_rows = float(np.mean(n_rows))
     algo_bytes = mean_act * bytes_per_expert                      # activated-expert weight bytes per launch
-    peak, peak_kind = measured_peaks()
+    peak, tf_burst, tf_sustained, peak_kind = measured_peaks()
     achieved = algo_bytes / (kernel_ms * 1e-3) / 1e9
     value = R_.whole_job_rate(T, ms_per_step)
-    stream_kernel = H in (1024, 2048)      # the library's choice: weight-streaming kernel (resident or gather mode)
+    step_bytes = algo_bytes + 4 * E * H                           # + the router's weights
+    step_frac = step_bytes / (ms_per_step * 1e-3) / 1e9 / peak
+    tensor_tflops = mean_rows * (k + ns) * 6.0 * H * I / (kernel_ms * 1e-3) / 1e12
+    kernel_name = B.team_expert_kernel_name(ctxs[0])
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": workload, "flags": args.flags, "rows_presented": T, "rows_computed_mean": mean_rows,
-                   "activated_experts_mean": mean_act, "layers_cycled": R,
-                   "l2": f"inputs larger than L2: weights rotate over {R} layers ({R * E * bytes_per_expert / 1e9:.1f} GB)",
-                   "cuda_graph": graph is not None, "steps_issued": issued, "parallelism": f"replicas x{world}"},
+        "config": config_of(args, shape, workload),
+        "run": {"layers_cycled": R, "weights_gb": R * (E + ns) * bytes_per_expert / 1e9, "cuda_graph": graph is not None,
+                "steps_issued": issued, "warmup_issued": warm, "e2e_warmup_issued": e2e_warm,
+                "rows_computed_mean": mean_rows, "activated_experts_mean": mean_act},
         "clocks": clocks,
         "e2e": {"value": R_.whole_job_rate(T, e2e_ms_per_step), "unit": UNIT, "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms_per_step, "steps": n_e2e},
         "gpu_launches": launches_per_step * issued,
         "activated_experts_per_s": R_.whole_job_rate(mean_act, ms_per_step),
         "rows_computed_per_s": R_.whole_job_rate(mean_rows, ms_per_step),
-        "step_hbm_frac": (algo_bytes + 4 * E * H) / (ms_per_step * 1e-3) / 1e9 / peak,
-        "roofline": {"bound": "hbm", "kernel": "k_experts_stream" if stream_kernel else "k_experts_tc", "achieved": achieved, "peak": peak,
+        "step_hbm_frac": step_frac,
+        "roofline": {"bound": "hbm", "kernel": kernel_name, "achieved": achieved, "peak": peak,
                      "peak_kind": f"of {peak_kind}", "unit": "GB/s", "frac": achieved / peak,
                      "frac_of_8TBs_nominal": achieved / 8000.0, "kernel_ms": kernel_ms,
                      "algorithmic_bytes_per_launch": algo_bytes, "launches_timed": tot_n,
-                     # DRAM read + write bytes per launch: ncu capture at 16 activated experts (151.08 MB read +
-                     # 3.25 MB written, profiles/experts_stream_c2_bench.md), scaled to this run's mean
-                     "traffic": mean_act * (151.08e6 + 3.25e6) / 16.0 if args.workload == "c2" else None,
+                     # the whole step (router + selection + experts, graph replay) on its algorithmic bytes
+                     "step_frac": step_frac, "step_frac_of_8TBs_nominal": step_bytes / (ms_per_step * 1e-3) / 8e12,
+                     "step_bytes": step_bytes,
+                     # DRAM read + write bytes per launch from the committed ncu capture, scaled to this run's mean
+                     "traffic": traffic_per_launch(args, kernel_name, mean_act),
                      # the same launches as a contraction: 6 H I flops per token-slot (routed and shared)
-                     "tensor_tflops": mean_rows * (k + ns) * 6.0 * H * I / (kernel_ms * 1e-3) / 1e12},
+                     "tensor_tflops": tensor_tflops, "tensor_frac_of_sustained": tensor_tflops / tf_sustained,
+                     "tensor_frac_of_burst": tensor_tflops / tf_burst},
     }
 
     if rank == 0:
         if world == 1 and args.cpu_seconds > 0:
             weights_host = {n: t.float().cpu().numpy() for n, t in
                             zip(("w_router", "w_gate", "w_up", "w_down"), layers[0])}
-            cb, _ = oracle_leg(args, shape, weights_host, steps_host, args.cpu_seconds)
+            cb, _ = oracle_leg(args, shape, weights_host, steps_host, args.cpu_seconds * 0.75)
+            one, _ = oracle_leg(args, shape, weights_host, steps_host, args.cpu_seconds * 0.25, threads=1)
+            cb["single_thread"] = {"value": one["value"], "cores": one["cores"], "sample": one["sample"]}
             line["cpu_baseline"] = cb
         print(json.dumps(line))
     for c in ctxs:
         B.team_destroy(c)
     if world > 1:
         dist.destroy_process_group()
+
+
+# DRAM bytes (read + write) per launch of the expert kernel at 16 activated experts, from the ncu capture whose
+# summary is committed under profiles/ (None once the kernel has changed since the counters were taken).
+TRAFFIC_AT_16_EXPERTS = {"k_experts_stream": None}
+
+
+def traffic_per_launch(args, kernel_name, mean_act):
+    t = TRAFFIC_AT_16_EXPERTS.get(kernel_name)
+    return mean_act * t / 16.0 if (t is not None and args.workload == "c2") else None
+
+
+def run_c5(args):
+    """Config 5: a stack of SDAR-shaped MoE layers with residual adds, run through the 4-step denoising loop of
+    `--blocks` decoding blocks, once with TEAM's selection (delayed caching + limited activation) and once with
+    vanilla top-k.  A step here is one denoising step of the whole stack (all layers)."""
+    import torch
+    import torch.distributed as dist
+    from paper_2602_08404_b200 import binding as B
+    from paper_2602_08404_b200 import replicas as R_
+    from paper_2602_08404_b200 import workloads as W
+    import dataclasses
+
+    world, rank, dev = init_device(args)
+    shape = W.C2
+    T, H, E, k, I = shape.rows, shape.hidden, shape.n_experts, shape.top_k, shape.inter
+    L = args.layers or W.C5_LAYERS
+    n_blocks = args.blocks
+    bytes_per_expert = 3 * H * I * 2
+    layers = []
+    for l in range(L):
+        wr, wg, wu, wd = W.device_layer_weights(shape, 5000 + l, dev)
+        layers.append((wr, wg, wu, B.team_pack_w_down(wd)))
+        del wd
+    # every block has its own seeded schedule (hidden states, confidences); the acceptance pattern is the scripted one
+    blocks = [W.make_schedule(shape, seed=shape.seed * 1000 + 29 + 7919 * b) for b in range(n_blocks)]
+    n_sched = len(blocks[0])
+    x_all = torch.stack([torch.stack([B.to_device(s["x"], B.TEAM_DTYPE_BF16, dev) for s in blk]) for blk in blocks])
+    conf_all = torch.stack([torch.stack([torch.as_tensor(s["conf"]).to(dev) for s in blk]) for blk in blocks])
+    st_static = [B.state_to_device(s, dev) for s in blocks[0]]      # states, positions, groups: the same in every block
+    x_work = torch.zeros((T, H), dtype=torch.bfloat16, device=dev)
+    y_dev = torch.zeros((T, H), dtype=torch.float32, device=dev)
+
+    results = {}
+    sampler = ClockSampler(dev.index)
+    with sampler:
+        for name, flags in (("team", TEAM_FLAGS), ("vanilla", 0)):
+            cfg = B.make_config(H, E, k, I, 0, max_rows=T, max_groups=1, dtype=B.TEAM_DTYPE_BF16, flags=flags,
+                                tau_hot=shape.tau_hot, L_hot=shape.L_hot)
+            ctxs = []
+            for l in range(L):
+                c = B.team_create(cfg)
+                B.team_set_weights(c, *layers[l])
+                ctxs.append(c)
+
+            def stack_step(s, n_act_out=None, bi=0):
+                """One denoising step of the stack: x <- x + layer(x) on the computed rows, layer after layer."""
+                for l, c in enumerate(ctxs):
+                    out = None
+                    if n_act_out is not None:
+                        out = {"n_active": n_act_out[bi, s, l:l + 1], "n_rows_active": n_act_out[bi, s, L + l:L + l + 1]}
+                    B.team_moe_forward(c, x_work, st_static[s], out, y_dev)
+                    B.team_residual_add(c, x_work, y_dev, T)
+
+            def load_block(b, s):
+                x_work.copy_(x_all[b, s])
+                st_static[s]["conf"].copy_(conf_all[b, s])
+
+            # accounting pass (untimed): activated experts and computed rows of every (block, step, layer)
+            counts = torch.zeros((n_blocks, n_sched, 2 * L), dtype=torch.int32, device=dev)
+            for b in range(n_blocks):
+                for s in range(n_sched):
+                    load_block(b, s)
+                    stack_step(s, counts, b)
+            torch.cuda.synchronize()
+            for c in ctxs:
+                code, detail = B.team_read_status(c)
+                if code != 0:
+                    raise SystemExit(f"device status {code} detail {detail}")
+            counts = counts.cpu().numpy().astype(np.int64)
+            n_act, n_rows = counts[:, :, :L], counts[:, :, L:]
+            x_final_check = float(x_work.float().abs().max())
+
+            # one graph per denoising step of the stack (L layers: router, selection, experts, residual add each)
+            graphs = []
+            side = torch.cuda.Stream(device=dev)
+            side.wait_stream(torch.cuda.current_stream())
+            with torch.cuda.stream(side):
+                for s in range(n_sched):
+                    load_block(0, s)
+                    stack_step(s)
+            torch.cuda.current_stream().wait_stream(side)
+            torch.cuda.synchronize()
+            for s in range(n_sched):
+                g = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g):
+                    stack_step(s)
+                graphs.append(g)
+
+            def run_blocks(nb):
+                for b in range(nb):
+                    for s in range(n_sched):
+                        load_block(b, s)
+                        graphs[s].replay()
+
+            run_blocks(min(n_blocks, 4))                       # warm-up
+            if world > 1:
+                dist.barrier()
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            run_blocks(n_blocks)
+            e1.record()
+            if world > 1:
+                dist.barrier()
+            torch.cuda.synchronize()
+            ms = R_.max_over_ranks(e0.elapsed_time(e1), dev)
+            results[name] = dict(ms=ms, n_act=n_act, n_rows=n_rows, x_absmax=x_final_check)
+            for c in ctxs:
+                B.team_destroy(c)
+    clocks = sampler.summary()
+
+    peak, _, _, peak_kind = measured_peaks()
+    stack_steps = n_blocks * n_sched
+
+    def summarise(r):
+        layer_steps = stack_steps * L
+        act_total = float(r["n_act"].sum())
+        bytes_total = act_total * bytes_per_expert + layer_steps * 4 * E * H
+        return {"ms_total": r["ms"], "ms_per_stack_step": r["ms"] / stack_steps, "us_per_layer_step": r["ms"] * 1e3 / layer_steps,
+                "rows_presented_per_s": R_.whole_job_rate(T * stack_steps, r["ms"]),
+                "rows_computed_per_s": R_.whole_job_rate(float(r["n_rows"][:, :, 0].sum()), r["ms"]),
+                "activated_experts_per_s": R_.whole_job_rate(act_total, r["ms"]),
+                "activated_experts_per_layer_step": act_total / layer_steps,
+                "step_frac": bytes_total / (r["ms"] * 1e-3) / 1e9 / peak,
+                "step_frac_of_8TBs_nominal": bytes_total / (r["ms"] * 1e-3) / 8e12}
+
+    team, vanilla = summarise(results["team"]), summarise(results["vanilla"])
+    workload = (f"c5_stack: {L} x (H{H} E{E} top{k} I{I} bf16) MoE-only layers with residual adds, batch 1 x block {shape.block}, "
+                f"{n_sched} denoising steps x {n_blocks} blocks, TEAM (DCD|LAC) vs vanilla top-k")
+    line = {
+        "metric": METRIC, "value": team["rows_presented_per_s"], "unit": UNIT, "n_gpus": world,
+        "steps": stack_steps, "warmup": min(n_blocks, 4) * n_sched, "ms_per_step": team["ms_per_stack_step"],
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": workload, "flags": TEAM_FLAGS, "rows_presented": T,
+                   "l2": f"inputs larger than L2: {L} layers of weights ({L * E * bytes_per_expert / 1e9:.1f} GB) are walked once per denoising step",
+                   "parallelism": "replicas (one process per GPU, no exchange on the data path)"},
+        "note": "a step is one denoising step of the whole stack; value counts rows presented to the stack per second "
+                "(each row passes through every layer)",
+        "clocks": clocks, "team": team, "vanilla": vanilla,
+        "vanilla_over_team_time": vanilla["ms_total"] / team["ms_total"],
+        "paper_context": "the paper reports up to 2.2x end-to-end decoding speed-up of TEAM over the vanilla model on one "
+                         "A100 80GB (whole SDAR 30B-A3B model incl. attention and speculative branches); not comparable",
+        "roofline": {"bound": "hbm", "kernel": "whole stack step (router, selection, experts, residual add per layer)",
+                     "achieved": team["step_frac"] * peak, "peak": peak, "peak_kind": f"of {peak_kind}", "unit": "GB/s",
+                     "frac": team["step_frac"], "traffic": None},
+        "gpu_launches": stack_steps * L * 4,
+    }
+    if rank == 0:
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main(argv=None):
+    args = parse_args(argv)
+    from paper_2602_08404_b200 import replicas as R_
+    if R_.needs_launcher(args.gpus):
+        # --gpus N without a launcher: start the N replicas ourselves (one process per GPU), pass their output through
+        raise SystemExit(R_.run_under_launcher(os.path.abspath(__file__), sys.argv[1:] if argv is None else argv, args.gpus))
+    if args.impl == "reference":
+        return run_reference(args)
+    if args.workload == "c5":
+        return run_c5(args)
+    return run_layer(args)
 
 
 if __name__ == "__main__":

@@ -255,6 +255,10 @@ int team_last_launch_count(const team_ctx *ctx);
  * stream when timing is enabled.  Synchronises the stream. */
 int team_expert_timing(team_ctx *ctx, int32_t enable, void *stream, float *avg_ms_out, int32_t *launches_out);
 
+/* Name of the expert kernel this context's team_moe_forward launches (static string), e.g. for labelling a
+ * measurement.  NULL context: "". */
+const char *team_expert_kernel_name(const team_ctx *ctx);
+
 /* Diagnostic: run the expert FFNs of a bf16 context through the plain-FMA
  * kernels instead of the tensor-core kernel (allocates scratch on first use).
  * Meant for triage of a parity failure, not for production. */

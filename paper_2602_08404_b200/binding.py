@@ -24,7 +24,7 @@ TEAM_DTYPE_F32, TEAM_DTYPE_BF16 = 0, 1
 
 EXPORTS = ["team_create", "team_destroy", "team_set_weights", "team_set_policy", "team_route",
            "team_route_static", "team_pack_w_down", "team_select_experts", "team_moe_forward", "team_moe_forward_host", "team_residual_add", "team_read_status",
-           "team_last_launch_count", "team_expert_timing", "team_debug_force_simt", "team_strerror",
+           "team_last_launch_count", "team_expert_kernel_name", "team_expert_timing", "team_debug_force_simt", "team_strerror",
            "team_last_cuda_error", "team_version"]
 
 
@@ -81,6 +81,8 @@ def lib():
         L.team_debug_force_simt.argtypes = [vp, i32]
         L.team_strerror.argtypes = [i32]
         L.team_strerror.restype = ctypes.c_char_p
+        L.team_expert_kernel_name.argtypes = [vp]
+        L.team_expert_kernel_name.restype = ctypes.c_char_p
         L.team_last_cuda_error.argtypes = [vp]
         L.team_last_cuda_error.restype = ctypes.c_char_p
         for name in EXPORTS:
@@ -214,6 +216,10 @@ def team_read_status(ctx):
 
 def team_last_launch_count(ctx):
     return lib().team_last_launch_count(ctx)
+
+
+def team_expert_kernel_name(ctx):
+    return lib().team_expert_kernel_name(ctx).decode()
 
 
 def team_expert_timing(ctx, enable):

@@ -487,6 +487,12 @@ int team_read_status(team_ctx* ctx, void* stream, int32_t* detail_out) {
 
 int team_last_launch_count(const team_ctx* ctx) { return ctx ? ctx->last_launches : 0; }
 
+const char* team_expert_kernel_name(const team_ctx* ctx) {
+  if (ctx == nullptr) return "";
+  if (!use_tensor_path(ctx)) return "k_gate_up + k_down";
+  return ctx->stream_path ? "k_experts_stream" : "k_experts_tc";
+}
+
 int team_expert_timing(team_ctx* ctx, int32_t enable, void* stream, float* avg_ms_out, int32_t* launches_out) {
   if (ctx == nullptr) return TEAM_ERR_ARG;
   cudaStream_t s = static_cast<cudaStream_t>(stream);

@@ -95,6 +95,7 @@ __device__ __forceinline__ void slot_row_weight(int slot, int T, int k, const fl
 
 // Kernel launchers (host side), one per translation unit.
 cudaError_t configure_router(int dtype, int hidden);
+int router_smem_bytes(int hidden);   // dynamic shared memory the logits kernels are opted in to for this hidden size
 cudaError_t configure_select(Dims max_dims);
 cudaError_t configure_experts_tc(int item_tile);
 int experts_tc_item_tile(int max_rows);

@@ -252,13 +252,15 @@ static cudaError_t prepare_kernel(K kernel, int smem) {
 // The opt-in is a per-device property of the kernel, shared by every context (and by the context-free
 // entry point): it is only ever raised, so that preparing for a small hidden size cannot take away
 // what a larger one needs.
+int router_smem_bytes(int hidden) { return kRowTile * hidden * (int)sizeof(float) + 1024; }
+
 cudaError_t configure_router(int dtype, int hidden) {
   static std::mutex mu;
   static int prepared[64][2] = {};   // [device][dtype]: shared-memory bytes opted in so far
   int dev = 0;
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return e;
-  const int smem = kRowTile * hidden * (int)sizeof(float) + 1024;
+  const int smem = router_smem_bytes(hidden);
   const int di = dtype == TEAM_DTYPE_F32 ? 0 : 1;
   std::lock_guard<std::mutex> lock(mu);
   if (dev >= 0 && dev < 64 && prepared[dev][di] >= smem) return cudaSuccess;

@@ -69,6 +69,14 @@ extern "C" int team_route_static(const team_config* cfg, const void* x, const vo
     cudaGetLastError();
     return TEAM_ERR_CUDA;
   }
+  // the logits kernels stage 8 rows of fp32 activations in shared memory: a hidden size that does not fit is a
+  // shape the kernels do not support, not a runtime failure
+  int smem_optin = 0;
+  if (cudaDeviceGetAttribute(&smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess) {
+    cudaGetLastError();
+    return TEAM_ERR_CUDA;
+  }
+  if ((long long)team::router_smem_bytes(cfg->hidden) > smem_optin) return TEAM_ERR_SHAPE;
   float* logits = nullptr;
   const int rc = team::setup_device(dev, cfg->dtype, cfg->hidden, &logits);
   if (rc != TEAM_OK) return rc;

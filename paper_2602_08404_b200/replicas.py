@@ -29,3 +29,26 @@ def whole_job_rate(units_per_rank_per_step, ms_per_step):
 def barrier():
     if world_size() > 1:
         dist.barrier()
+
+
+def launcher_command(script, argv, n, port=None, python=None):
+    """The command that runs `script argv...` as n ranks of one node (one process per GPU), rendezvous on
+    127.0.0.1: what `--gpus n` means when no launcher has set WORLD_SIZE yet."""
+    import os
+    import sys
+    port = port or 29500 + os.getpid() % 20000
+    return [python or sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={int(n)}",
+            "--master-addr", "127.0.0.1", "--master-port", str(port), script] + list(argv)
+
+
+def needs_launcher(n_requested, env=None):
+    """True when more than one replica was asked for and this process was not started by a launcher."""
+    import os
+    env = os.environ if env is None else env
+    return int(n_requested) > 1 and "WORLD_SIZE" not in env
+
+
+def run_under_launcher(script, argv, n, timeout=None, port=None):
+    """Runs the script as n ranks and passes its output through; returns the launcher's exit code."""
+    import subprocess
+    return subprocess.run(launcher_command(script, argv, n, port=port), timeout=timeout).returncode

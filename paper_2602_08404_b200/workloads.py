@@ -128,6 +128,22 @@ def make_weights(shape, seed=None, std=0.02):
     )
 
 
+def device_layer_weights(shape, layer_seed, device, std=0.02):
+    """One layer's weights generated ON THE DEVICE with torch's seeded generator (same distribution as
+    make_weights): router fp32 [E,H]; gate/up [E+ns,I,H] and down [E+ns,H,I] (row-major) in the storage type.
+    For workloads whose weights are too many to draw on the host (a 48-layer stack is 58 GB in bf16); a host-side
+    consumer copies the tensors back, so both sides see the same values."""
+    import torch
+    E, H, I, ns = shape.n_experts, shape.hidden, shape.inter, shape.n_shared
+    store = torch.bfloat16 if shape.dtype == "bf16" else torch.float32
+    gen = torch.Generator(device=device)
+    gen.manual_seed(int(layer_seed))
+    wr = (torch.randn((E, H), generator=gen, device=device, dtype=torch.float32) * std).contiguous()
+    wg, wu, wd = [(torch.randn(dims, generator=gen, device=device, dtype=torch.float32) * std).to(store).contiguous()
+                  for dims in ((E + ns, I, H), (E + ns, I, H), (E + ns, H, I))]
+    return wr, wg, wu, wd
+
+
 def _accept_step(shape, p):
     """Step at whose end position p is accepted (it is NEW at the following step)."""
     return (p // shape.unmask_per_step + 1) * shape.unmask_every - 1

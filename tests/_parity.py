@@ -75,11 +75,26 @@ def pinned_rows(cfg, ref, group):
         all(group_ok.values())
 
 
-def compare_routing(cfg, ref, got, group, what=""):
+PROBS_ATOL = 1e-6      # softmax probabilities: fp32 exp and division against fp64, on the same fp32 logits
+
+
+def compare_probs(ref, got, what=""):
+    """The exported softmax table against the oracle's router: computed rows within PROBS_ATOL, skipped rows zero."""
+    comp = ref["tok_class"] != O.CLS_SKIP
+    if comp.any():
+        np.testing.assert_allclose(got["probs"][comp], ref["probs"][comp], rtol=0, atol=PROBS_ATOL,
+                                   err_msg=f"{what} probs")
+        np.testing.assert_allclose(got["probs"][comp].sum(axis=1), 1.0, rtol=0, atol=1e-5, err_msg=f"{what} probs sum")
+    if (~comp).any():
+        assert not got["probs"][~comp].any(), f"{what}: probs of skipped rows must be zero"
+
+
+def compare_routing(cfg, ref, got, group, what="", return_pin=False):
     """Integer tables bit-exact where pinned; floating-point tables within fp32 rounding."""
     pin, groups_ok = pinned_rows(cfg, ref, group)
     np.testing.assert_array_equal(got["tok_class"], ref["tok_class"], err_msg=what)
     assert got["n_rows_active"] == ref["n_rows_active"], what
+    compare_probs(ref, got, what)
     for t in np.flatnonzero(pin):
         np.testing.assert_array_equal(got["topk_idx"][t], ref["topk_idx"][t], err_msg=f"{what} row {t}")
         np.testing.assert_allclose(got["topk_w"][t], ref["topk_w"][t], atol=2e-6, rtol=1e-5, err_msg=what)
@@ -92,6 +107,8 @@ def compare_routing(cfg, ref, got, group, what=""):
             np.testing.assert_array_equal(got[name], ref[name], err_msg=f"{what} {name}")
         assert got["n_active"] == ref["n_active"], what
     check_self_consistency(cfg, got, group)
+    if return_pin:
+        return bool(pin.all() and groups_ok), pin
     return bool(pin.all() and groups_ok)
 
 
@@ -131,6 +148,55 @@ def check_self_consistency(cfg, got, group):
     np.testing.assert_array_equal(got["active"], np.flatnonzero(cnt > 0))
 
 
+def y_from_choices(cfg, weights, x, T, row, idx_row, w_row):
+    """Layer output of one row from a given set of choices: sum_j w_j * expert(idx_j)(x) + shared experts.
+    Used for rows whose own choice is not pinned (a near-tie): the oracle's expert arithmetic on the choice the
+    library reports, so that the row's y is still checked against the oracle and never against itself."""
+    y = np.zeros(cfg.hidden, dtype=np.float64)
+    xr = np.asarray(x)[row:row + 1]
+    for e, wt in zip(idx_row, w_row):
+        y += float(wt) * O.expert_ffn(xr, weights["w_gate"][int(e)], weights["w_up"][int(e)], weights["w_down"][int(e)])[0]
+    for sh in range(cfg.n_shared):
+        e = cfg.n_experts + sh
+        y += O.expert_ffn(xr, weights["w_gate"][e], weights["w_up"][e], weights["w_down"][e])[0]
+    return y
+
+
+MIN_PINNED_FRACTION = 0.99     # of the rows of a step; below it the seed is a bad one and the test must say so
+
+
+def compare_y_rows(shape, cfg, weights, x, ref_y, ref, got, got_y, pin, y_before, what="", max_unpinned=None):
+    """Every computed row against the oracle at the stated tolerance: pinned rows against the oracle's layer
+    output, the others against the oracle's expert arithmetic on the choices the library reports.  Skipped rows
+    must be bit-identical to what was there before.  Returns (max relative error, oracle y with the unpinned rows
+    replaced).  max_unpinned: how many rows of the step may have a near-tie (default: 1 % of the rows, i.e. none in
+    a small step; callers whose inputs are not under a seed's control, such as the activations inside a stack, say
+    how many they tolerate)."""
+    tol = TOL_BF16 if shape.dtype == "bf16" else TOL_F32
+    cls = ref["tok_class"]
+    T = len(cls)
+    comp = cls != O.CLS_SKIP
+    n_unpinned = int((~pin).sum())
+    if max_unpinned is None:
+        max_unpinned = int((1.0 - MIN_PINNED_FRACTION) * T)
+    assert n_unpinned <= max_unpinned, \
+        f"{what}: {n_unpinned} of {T} rows have a near-tie: too many for a meaningful comparison, pick another seed"
+    want = np.array(ref_y, dtype=np.float64)
+    for t in np.flatnonzero(comp & ~pin):
+        want[t] = y_from_choices(cfg, weights, x, T, t, got["topk_idx"][t], got["topk_w"][t])
+    rel = 0.0
+    if comp.any():
+        scale = np.abs(want[comp]).max()
+        err_rows = np.abs(got_y[comp] - want[comp]).max(axis=1)
+        worst = int(np.flatnonzero(comp)[err_rows.argmax()])
+        assert err_rows.max() <= tol * scale, \
+            f"{what}: row {worst} max|err| {err_rows.max():.3e} > {tol} * {scale:.3e}"
+        rel = float(err_rows.max() / scale) if scale > 0 else 0.0
+    if (~comp).any():
+        np.testing.assert_array_equal(got_y[~comp], y_before[~comp], err_msg=f"{what}: cached rows changed")
+    return rel, want
+
+
 def compare_y(shape, ref_y, got_y, cls, y_before, what=""):
     tol = TOL_BF16 if shape.dtype == "bf16" else TOL_F32
     comp = cls != O.CLS_SKIP
@@ -143,8 +209,12 @@ def compare_y(shape, ref_y, got_y, cls, y_before, what=""):
     return (np.abs(got_y[comp] - ref_y[comp]).max() / np.abs(ref_y[comp]).max()) if comp.any() else 0.0
 
 
-def run_schedule(shape, weights, steps, flags, force_simt=False, check_routing=True, **kw):
-    """Runs every step of a schedule through team_moe_forward and the oracle; returns per-step stats."""
+def run_schedule(shape, weights, steps, flags, force_simt=False, policy_switch=None, **kw):
+    """Runs every step of a schedule through team_moe_forward and the oracle; returns per-step stats.
+
+    Every computed row of every step is compared with the oracle (compare_y_rows): there is no step whose layer
+    output goes unchecked.  `policy_switch` = (step index, dict of policy fields): from that step on both sides use
+    the changed policy (the library through team_set_policy on the same context)."""
     ocfg = oracle_config(shape, flags, **kw)
     layer = Layer(shape, weights, flags, **kw)
     if force_simt:
@@ -155,6 +225,15 @@ def run_schedule(shape, weights, steps, flags, force_simt=False, check_routing=T
     stats = []
     try:
         for si, step in enumerate(steps):
+            if policy_switch is not None and si == policy_switch[0]:
+                import dataclasses
+                changed = dict(policy_switch[1])
+                new_flags = changed.pop("flags", flags)
+                ocfg = dataclasses.replace(ocfg, flags=new_flags, **changed)
+                for name, v in changed.items():
+                    setattr(layer.cfg, name, v)
+                layer.cfg.flags = new_flags
+                B.team_set_policy(layer.ctx, layer.cfg)
             x_dev = B.to_device(step["x"], dtype_code(shape))
             st = B.state_to_device(step)
             out = B.alloc_routing(layer.cfg, T)
@@ -165,16 +244,13 @@ def run_schedule(shape, weights, steps, flags, force_simt=False, check_routing=T
             got = B.routing_to_host(out)
             y_ref, ref = O.moe_forward(ocfg, weights, step["x"], step["tok_state"], step["conf"], step["pos"],
                                        step["group"], step["branch"], y_prev=y_ref)
-            what = f"{shape.name} flags={flags} step={si}"
-            exact = compare_routing(ocfg, ref, got, step["group"], what) if check_routing else True
+            what = f"{shape.name} flags={ocfg.flags} step={si}"
+            exact, pin = compare_routing(ocfg, ref, got, step["group"], what, return_pin=True)
             got_y = y_dev.cpu().numpy()
-            if exact:
-                rel = compare_y(shape, y_ref, got_y, ref["tok_class"], y_before, what)
-            else:
-                rel = float("nan")      # a near-tie changed an expert choice; y is checked by self-consistency only
-                y_ref = got_y.astype(np.float64)
+            rel, y_ref = compare_y_rows(shape, ocfg, weights, step["x"], y_ref, ref, got, got_y, pin, y_before, what)
             stats.append(dict(step=si, n_active=got["n_active"], rows=got["n_rows_active"], rel_err=rel,
-                              exact=exact, launches=B.team_last_launch_count(layer.ctx)))
+                              exact=exact, pinned=int(pin.sum()), classes=ref["tok_class"].copy(),
+                              launches=B.team_last_launch_count(layer.ctx)))
     finally:
         layer.close()
     return stats

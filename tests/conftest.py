@@ -12,12 +12,6 @@ def pytest_configure(config):
     config.addinivalue_line("markers", "gpu: needs a CUDA device (run on the B200 box)")
 
 
-def pytest_collection_modifyitems(config, items):
-    # Tests marked gpu fail loudly rather than skip when no device is present:
-    # they are only selected with -m gpu, on a machine that has one.
-    pass
-
-
 @pytest.fixture(scope="session")
 def golden_dir():
     return os.path.join(ROOT, "tests", "golden")

@@ -155,15 +155,15 @@ def _run_stack(shape, n_layers, flags, weights_cache):
                 y_ref, ref = O.moe_forward(ocfg, layers_w[li], x_in, step["tok_state"], step["conf"], step["pos"],
                                            step["group"], step["branch"], y_prev=y_before)
                 what = f"{shape.name} stack step={si} layer={li}"
-                exact = P.compare_routing(ocfg, ref, got, step["group"], what)
+                exact, pin = P.compare_routing(ocfg, ref, got, step["group"], what, return_pin=True)
                 all_exact = all_exact and exact
-                if exact:
-                    P.compare_y(shape, y_ref, y_dev.cpu().numpy(), ref["tok_class"], y_before, what)
-                    # the residual add: fp32 add, stored in the activation type
-                    comp = ref["tok_class"] != O.CLS_SKIP
-                    want = x_in.astype(np.float64).copy()
-                    want[comp] = round_fn(x_in[comp].astype(np.float32) + y_dev.cpu().numpy()[comp])
-                    np.testing.assert_array_equal(x_dev.float().cpu().numpy().astype(np.float64), want, err_msg=what)
+                P.compare_y_rows(shape, ocfg, layers_w[li], x_in, y_ref, ref, got, y_dev.cpu().numpy(), pin, y_before, what,
+                                 max_unpinned=max(1, T // 32))      # inputs of deeper layers come from the stack itself
+                # the residual add: fp32 add, stored in the activation type
+                comp = ref["tok_class"] != O.CLS_SKIP
+                want = x_in.astype(np.float64).copy()
+                want[comp] = round_fn(x_in[comp].astype(np.float32) + y_dev.cpu().numpy()[comp])
+                np.testing.assert_array_equal(x_dev.float().cpu().numpy().astype(np.float64), want, err_msg=what)
             if all_exact:
                 x_ref, _ = O.stack_forward(ocfg, layers_w, step["x"], step["tok_state"], step["conf"], step["pos"],
                                            step["group"], step["branch"], round_fn=round_fn)

@@ -170,6 +170,35 @@ def test_stack_glue_is_a_residual_add_on_computed_rows():
     assert len(n_act) == 3
 
 
+def test_stack_with_single_expert_layers_is_a_residual_mlp_stack_with_rounding():
+    """Pin of the stack glue against library ops, including the store-back rounding: with one expert and k = 1 every
+    layer is a dense SwiGLU MLP, so the stack is x <- round(x + mlp_l(x)) layer after layer, written here with torch
+    CPU ops and a bf16 round trip through torch's own conversion."""
+    rng = np.random.default_rng(10)
+    T, H, I, L = 5, 16, 8, 4
+    layers = [_weights(rng, 1, H, I) for _ in range(L)]
+    x = torch.from_numpy(rng.standard_normal((T, H)).astype(np.float32)).to(torch.bfloat16).float().numpy()
+    cfg = O.Config(hidden=H, n_experts=1, top_k=1, inter=I, flags=0)
+
+    def to_bf16(a):
+        return torch.from_numpy(np.asarray(a, dtype=np.float32)).to(torch.bfloat16).double().numpy()
+
+    for round_fn in (None, to_bf16):
+        out, n_act = O.stack_forward(cfg, layers, x, *_state(T), round_fn=round_fn)
+        ref = x.astype(np.float64)
+        for w in layers:
+            ref = ref + _torch_mlp(ref, w["w_gate"][0], w["w_up"][0], w["w_down"][0])
+            if round_fn is not None:
+                ref = to_bf16(ref)
+        np.testing.assert_allclose(out, ref, rtol=1e-12, atol=1e-13)
+        assert n_act == [1] * L
+    # zero down projections: the stack is the identity
+    for w in layers:
+        w["w_down"][:] = 0
+    out, _ = O.stack_forward(cfg, layers, x, *_state(T), round_fn=to_bf16)
+    np.testing.assert_array_equal(out, x.astype(np.float64))
+
+
 # --- planted mistakes: each must be caught by at least one pin ---------------------
 def _fails(pins, mod):
     for pin in pins:
@@ -209,10 +238,11 @@ def _no_sigmoid_scale(x, wg, wu, wd):
 
 
 def _transposed_down(x, wg, wu, wd):
-    wd = np.asarray(wd, np.float64)
-    if wd.shape[0] == wd.shape[1]:
-        return O.expert_ffn(x, wg, wu, wd.T)
-    return O.expert_ffn(x, wg, wu, wd) * 0.5
+    """The down projection read with its two axes exchanged: the [H, I] matrix is taken as if it were stored [I, H]
+    (same bytes, other strides), which is what a transposed operand is for a non-square matrix."""
+    wd = np.ascontiguousarray(np.asarray(wd, np.float64))
+    H, I = wd.shape
+    return O.expert_ffn(x, wg, wu, wd.reshape(I, H).T)
 
 
 def _unnormalised_weights(p, idx, norm):

@@ -65,3 +65,47 @@ def test_reference_arm_prints_nothing_on_other_ranks():
                        env=env, capture_output=True, text=True, timeout=300)
     assert r.returncode == 0
     assert r.stdout.strip() == ""
+
+
+def test_gpus_flag_without_a_launcher_starts_the_replicas_itself():
+    """`--gpus 2` with no WORLD_SIZE in the environment: the same arguments are re-run as 2 ranks under
+    torch.distributed.run (rendezvous on 127.0.0.1) and rank 0 prints the one line."""
+    sys.path.insert(0, ROOT)
+    from paper_2602_08404_b200 import replicas as R
+    env = {k: v for k, v in os.environ.items() if k not in ("WORLD_SIZE", "RANK", "LOCAL_RANK")}
+    assert R.needs_launcher(2, env) and not R.needs_launcher(1, env)
+    assert not R.needs_launcher(2, dict(env, WORLD_SIZE="2"))          # already under a launcher
+    stub = os.path.join(ROOT, "tests", "_replica_stub.py")
+    cmd = R.launcher_command(stub, ["--gpus", "2", "--steps", "7"], 2, port=29500 + (os.getpid() + 977) % 2000)
+    assert "--nproc-per-node=2" in cmd and "127.0.0.1" in cmd
+    r = subprocess.run(cmd, env=env, capture_output=True, text=True, timeout=300)
+    assert r.returncode == 0, r.stderr[-2000:]
+    lines = [json.loads(l) for l in r.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1                                             # rank 0 alone prints
+    assert lines[0]["n_gpus"] == 2 and lines[0]["asked"] == 2 and lines[0]["steps"] == 7
+    assert abs(lines[0]["ms_per_step"] - 0.050) < 1e-12
+    assert abs(lines[0]["value"] - 2 * 4 / 0.050e-3) < 1e-6
+
+
+def test_bench_hands_gpus_n_to_the_launcher(monkeypatch):
+    """bench.py --gpus 2, started plainly: before touching any device it re-runs itself under the launcher with the
+    same arguments and exits with the launcher's code."""
+    sys.path.insert(0, ROOT)
+    import bench
+    from paper_2602_08404_b200 import replicas as R
+    for k in ("WORLD_SIZE", "RANK", "LOCAL_RANK"):
+        monkeypatch.delenv(k, raising=False)
+    seen = {}
+
+    def fake(script, argv, n, **kw):
+        seen.update(script=script, argv=list(argv), n=n)
+        return 17
+
+    monkeypatch.setattr(R, "run_under_launcher", fake)
+    try:
+        bench.main(["--gpus", "2", "--steps", "20", "--warmup", "5"])
+        raise AssertionError("bench.main should have exited")
+    except SystemExit as e:
+        assert e.code == 17
+    assert seen["n"] == 2 and seen["argv"] == ["--gpus", "2", "--steps", "20", "--warmup", "5"]
+    assert os.path.basename(seen["script"]) == "bench.py"
