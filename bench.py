@@ -387,7 +387,7 @@ def run_layer(args):
         with torch.cuda.stream(e2e_stream):
             # untimed: every context allocates its staging block and records its step on its first call, so every
             # context is called (twice) before the clock starts, whatever --warmup says
-            e2e_warm = max(2 * period, min(args.warmup, 200))
+            e2e_warm = max(8 * period, min(args.warmup, 200))
             for i in range(e2e_warm):
                 e2e_step(i)
             barrier()
