@@ -264,6 +264,18 @@ const char *team_expert_kernel_name(const team_ctx *ctx);
  * Meant for triage of a parity failure, not for production. */
 int team_debug_force_simt(team_ctx *ctx, int on);
 
+/* Diagnostic knobs of a context (not for production use).
+ *   TEAM_KNOB_NO_FUSE (value 0/1): with at most 8 rows and no dispatch table asked for, team_moe_forward runs the
+ *     whole step as one kernel; 1 keeps the three-kernel sequence (router, selection, experts) instead.
+ *   TEAM_KNOB_WAIT_LIMIT_US (1 .. 10,000,000): how long a device-side wait (the one-kernel step's grid barrier) may
+ *     last before the kernel gives up, records TEAM_ERR_TIMEOUT in the status word and returns; default about 1 s.
+ *   TEAM_KNOB_EXTRA_ARRIVALS (0/1): 1 makes that barrier wait for one arrival that never comes, so that the
+ *     give-up path can be exercised (with a short limit) without any kernel hanging; y is then left unspecified
+ *     for the computed rows of that call.
+ * Errors: TEAM_ERR_ARG. */
+enum { TEAM_KNOB_NO_FUSE = 1, TEAM_KNOB_EXTRA_ARRIVALS = 2, TEAM_KNOB_WAIT_LIMIT_US = 3 };
+int team_debug_knob(team_ctx *ctx, int knob, long long value);
+
 const char *team_strerror(int code);
 const char *team_last_cuda_error(const team_ctx *ctx);
 int team_version(void);

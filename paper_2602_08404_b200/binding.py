@@ -24,7 +24,7 @@ TEAM_DTYPE_F32, TEAM_DTYPE_BF16 = 0, 1
 
 EXPORTS = ["team_create", "team_destroy", "team_set_weights", "team_set_policy", "team_route",
            "team_route_static", "team_pack_w_down", "team_select_experts", "team_moe_forward", "team_moe_forward_host", "team_residual_add", "team_read_status",
-           "team_last_launch_count", "team_expert_kernel_name", "team_expert_timing", "team_debug_force_simt", "team_strerror",
+           "team_last_launch_count", "team_expert_kernel_name", "team_expert_timing", "team_debug_force_simt", "team_debug_knob", "team_strerror",
            "team_last_cuda_error", "team_version"]
 
 
@@ -79,6 +79,7 @@ def lib():
         L.team_last_launch_count.argtypes = [vp]
         L.team_expert_timing.argtypes = [vp, i32, vp, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(i32)]
         L.team_debug_force_simt.argtypes = [vp, i32]
+        L.team_debug_knob.argtypes = [vp, i32, ctypes.c_longlong]
         L.team_strerror.argtypes = [i32]
         L.team_strerror.restype = ctypes.c_char_p
         L.team_expert_kernel_name.argtypes = [vp]
@@ -228,6 +229,13 @@ def team_expert_timing(ctx, enable):
     return ms.value, n.value
 
 
+TEAM_KNOB_NO_FUSE, TEAM_KNOB_EXTRA_ARRIVALS, TEAM_KNOB_WAIT_LIMIT_US = 1, 2, 3
+
+
+def team_debug_knob(ctx, knob, value):
+    _check(lib().team_debug_knob(ctx, int(knob), int(value)), ctx)
+
+
 def team_debug_force_simt(ctx, on):
     _check(lib().team_debug_force_simt(ctx, int(on)), ctx)
 
@@ -246,10 +254,12 @@ def alloc_routing(cfg, n_rows, device="cuda"):
 
 def routing_to_host(out):
     r = {n: v.cpu().numpy() for n, v in out.items()}
-    r["group_mask"] = r["group_mask"].view(np.uint64)
-    r["n_active"] = int(r["n_active"][0])
-    r["n_rows_active"] = int(r["n_rows_active"][0])
-    r["active"] = r["active"][:r["n_active"]]
+    if "group_mask" in r:
+        r["group_mask"] = r["group_mask"].view(np.uint64)
+    if "n_active" in r:
+        r["n_active"] = int(r["n_active"][0])
+        r["n_rows_active"] = int(r["n_rows_active"][0])
+        r["active"] = r["active"][:r["n_active"]]
     return r
 
 

@@ -25,6 +25,10 @@ struct team_ctx {
   int last_launches;
   int force_simt;
   bool stream_path;   // few rows: the weight-streaming expert kernel instead of the tensor-memory one
+  bool fused_ok;      // at most 8 rows: the whole step can run as one kernel (router and selection in its prologue)
+  int no_fuse;        // diagnostic knob: keep the three-kernel sequence
+  int extra_arrivals; // diagnostic knob: arrivals the fused step's barrier waits for beyond the grid's own
+  long long spin_cycles;   // limit of device-side waits, in SM clock cycles
   void* simt_act;   // diagnostic fp32-FMA path on bf16 weights: activation scratch
   // team_moe_forward_host: one device block and its pinned host mirror, [inputs | y]
   unsigned char* hs_dev;
@@ -110,6 +114,20 @@ void drop_host_graph(team_ctx* ctx) {
   ctx->hs_graph_rows = 0;
 }
 
+// The next pair of timing events of the context (created on demand).
+cudaError_t timing_events(team_ctx* ctx, cudaEvent_t* e0, cudaEvent_t* e1) {
+  while (ctx->ev_used + 2 > ctx->ev.size()) {
+    cudaEvent_t ne;
+    const cudaError_t e = cudaEventCreate(&ne);
+    if (e != cudaSuccess) return e;
+    ctx->ev.push_back(ne);
+  }
+  *e0 = ctx->ev[ctx->ev_used];
+  *e1 = ctx->ev[ctx->ev_used + 1];
+  ctx->ev_used += 2;
+  return cudaSuccess;
+}
+
 bool use_tensor_path(const team_ctx* ctx) { return ctx->cfg.dtype == TEAM_DTYPE_BF16 && !ctx->force_simt; }
 
 int pick_item_tile(const team_config& c) { return team::experts_tc_item_tile(c.max_rows); }
@@ -160,6 +178,10 @@ int team_create(const team_config* cfg, team_ctx** out) {
   ctx->cuda_err[0] = 0;
   ctx->timing = false;
   ctx->ev_used = 0;
+  ctx->fused_ok = false;
+  ctx->no_fuse = 0;
+  ctx->extra_arrivals = 0;
+  ctx->spin_cycles = 2000000000ll;      // about a second
   cudaError_t e = cudaGetDevice(&ctx->device);
   if (e == cudaSuccess) e = cudaDeviceGetAttribute(&ctx->n_sms, cudaDevAttrMultiProcessorCount, ctx->device);
   if (e != cudaSuccess) {
@@ -178,6 +200,7 @@ int team_create(const team_config* cfg, team_ctx** out) {
     delete ctx;
     return TEAM_ERR_CUDA;
   }
+  ctx->fused_ok = ctx->stream_path && team::step_fused_supported(cfg->hidden, cfg->max_rows, cfg->n_experts, ctx->n_sms);
 
   const size_t T = cfg->max_rows, E = cfg->n_experts, k = cfg->top_k, ns = cfg->n_shared, EN = E + ns;
   const size_t S = T * (k + ns);
@@ -224,6 +247,7 @@ int team_create(const team_config* cfg, team_ctx** out) {
   ws.r.n_rows_active = scal + 1;
   ws.n_items = scal + 2;
   ws.status = scal + 4;
+  ws.arrivals = reinterpret_cast<unsigned long long*>(scal + 8);
   ws.items = reinterpret_cast<team::WorkItem*>(b + o_items);
   ws.act = reinterpret_cast<float*>(b + o_act);
   ws.win_flags = reinterpret_cast<int32_t*>(b + o_flags);
@@ -324,31 +348,35 @@ int team_moe_forward(team_ctx* ctx, const void* x, const team_step_state* st, te
   const team::Dims d = dims_of(ctx->cfg, st->n_rows);
   const bool tc = use_tensor_path(ctx);
   ctx->last_launches = 0;
-  cudaError_t e = team::launch_router_logits(x, ctx->cfg.dtype, static_cast<const float*>(ctx->w.w_router),
-                                             st->tok_state, ctx->ws.logits, tc ? y : nullptr, d, ctx->cfg.flags, s);
-  if (e != cudaSuccess) return fail_cuda(ctx, e, "router logits");
-  ++ctx->last_launches;
   // The resident few-rows expert kernel reads the rows' choices directly; the dispatch tables are built only
   // when the caller asked for one of them.
   const bool wants_tables = out != nullptr && (out->expert_count || out->expert_offset || out->perm || out->active ||
                                                out->n_active || out->n_rows_active);
   const bool resident = tc && ctx->stream_path && !team::experts_stream_gathers(ctx->cfg.max_rows);
+  cudaError_t e = cudaSuccess;
+  cudaEvent_t ev0 = nullptr, ev1 = nullptr;
+  if (resident && !wants_tables && ctx->fused_ok && !ctx->no_fuse) {
+    // at most 8 rows and no dispatch table asked for: the whole step is one kernel
+    if (ctx->timing && (e = timing_events(ctx, &ev0, &ev1)) != cudaSuccess) return fail_cuda(ctx, e, "event create");
+    if (ev0) cudaEventRecord(ev0, s);
+    e = team::launch_step_fused(x, static_cast<const float*>(ctx->w.w_router), ctx->w.w_gate, ctx->w.w_up, ctx->w.w_down,
+                                step_ptrs(st), ctx->ws, export_ptrs(out), y, d, policy_of(ctx->cfg), ctx->n_sms,
+                                ctx->spin_cycles, ctx->extra_arrivals, s);
+    if (e != cudaSuccess) return fail_cuda(ctx, e, "fused step");
+    if (ev1) cudaEventRecord(ev1, s);
+    ctx->last_launches = 1;
+    return TEAM_OK;
+  }
+  e = team::launch_router_logits(x, ctx->cfg.dtype, static_cast<const float*>(ctx->w.w_router), st->tok_state,
+                                 ctx->ws.logits, tc ? y : nullptr, d, ctx->cfg.flags, s);
+  if (e != cudaSuccess) return fail_cuda(ctx, e, "router logits");
+  ++ctx->last_launches;
   e = team::launch_select(ctx->ws.logits, step_ptrs(st), ctx->ws, export_ptrs(out), d, policy_of(ctx->cfg),
                           ctx->item_tile, wants_tables || !resident, s);
   if (e != cudaSuccess) return fail_cuda(ctx, e, "select");
   ctx->last_launches += team::select_launches(d);
-  cudaEvent_t ev0 = nullptr, ev1 = nullptr;
   if (ctx->timing) {
-    if (ctx->ev_used + 2 > ctx->ev.size()) {
-      for (int i = 0; i < 2; ++i) {
-        cudaEvent_t ne;
-        if ((e = cudaEventCreate(&ne)) != cudaSuccess) return fail_cuda(ctx, e, "event create");
-        ctx->ev.push_back(ne);
-      }
-    }
-    ev0 = ctx->ev[ctx->ev_used];
-    ev1 = ctx->ev[ctx->ev_used + 1];
-    ctx->ev_used += 2;
+    if ((e = timing_events(ctx, &ev0, &ev1)) != cudaSuccess) return fail_cuda(ctx, e, "event create");
     cudaEventRecord(ev0, s);
   }
   if (tc) {
@@ -490,7 +518,27 @@ int team_last_launch_count(const team_ctx* ctx) { return ctx ? ctx->last_launche
 const char* team_expert_kernel_name(const team_ctx* ctx) {
   if (ctx == nullptr) return "";
   if (!use_tensor_path(ctx)) return "k_gate_up + k_down";
-  return ctx->stream_path ? "k_experts_stream" : "k_experts_tc";
+  if (!ctx->stream_path) return "k_experts_tc";
+  const bool fused = ctx->fused_ok && !ctx->no_fuse && !team::experts_stream_gathers(ctx->cfg.max_rows);
+  return fused ? "k_experts_stream (fused step: router, selection and experts in one launch)" : "k_experts_stream";
+}
+
+int team_debug_knob(team_ctx* ctx, int knob, long long value) {
+  if (ctx == nullptr) return TEAM_ERR_ARG;
+  switch (knob) {
+    case TEAM_KNOB_NO_FUSE: ctx->no_fuse = value != 0; break;
+    case TEAM_KNOB_EXTRA_ARRIVALS:
+      if (value < 0 || value > 1) return TEAM_ERR_ARG;
+      ctx->extra_arrivals = (int)value;
+      break;
+    case TEAM_KNOB_WAIT_LIMIT_US:
+      if (value < 1 || value > 10000000) return TEAM_ERR_ARG;
+      ctx->spin_cycles = value * 2000;       // SM cycles at about 2 GHz
+      break;
+    default: return TEAM_ERR_ARG;
+  }
+  drop_host_graph(ctx);
+  return TEAM_OK;
 }
 
 int team_expert_timing(team_ctx* ctx, int32_t enable, void* stream, float* avg_ms_out, int32_t* launches_out) {

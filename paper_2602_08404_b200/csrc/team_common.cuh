@@ -73,6 +73,7 @@ struct Workspace {
   __nv_bfloat16* act_g; // bf16 path: [items][item_tile][I] activations published between CTAs
   int32_t* win_flags;   // bf16 path: [n_flags] groups published per 64-column window, zeroed per step
   int32_t n_flags;
+  unsigned long long* arrivals;   // fused step: CTA arrivals at the grid barrier, counted over all launches
 };
 
 __device__ __forceinline__ void set_status(int32_t* status, int code, int detail) {
@@ -105,6 +106,10 @@ int experts_stream_item_tile(int max_rows);
 cudaError_t configure_experts_stream(int hidden, int max_rows);
 cudaError_t launch_experts_stream(const void* x, const void* w_gate, const void* w_up, const void* w_down, Workspace ws,
                                   float* y, Dims d, int max_rows, int grid, cudaStream_t s);
+bool step_fused_supported(int hidden, int max_rows, int n_experts, int grid);
+cudaError_t launch_step_fused(const void* x, const float* w_router, const void* w_gate, const void* w_up, const void* w_down,
+                              StepPtrs st, Workspace ws, RoutePtrs ex, float* y, Dims d, Policy p, int grid,
+                              long long spin_cycles, int extra_arrivals, cudaStream_t s);
 cudaError_t launch_router_logits(const void* x, int dtype, const float* w_router, const uint8_t* tok_state,
                                  float* logits, float* y_zero, Dims d, int flags, cudaStream_t s);
 cudaError_t launch_router_topk(const float* logits, const uint8_t* tok_state, RoutePtrs out, Dims d, Policy p,

@@ -28,7 +28,15 @@
 // Token columns.  Up to 8 rows per call: the call's rows themselves, for every expert (weight 0 where a row
 // did not choose it), and the activated set is formed here from the rows' choices.  More rows: work items
 // of 8 or 16 token-slots of one expert, built by the selection kernel, gathered into shared memory per item.
+//
+// Fused step (up to 8 rows, no dispatch table asked for).  The whole layer step is this one kernel: every CTA
+// first computes the router logits of "its" experts (expert e on CTA e mod grid: the 4*E*H bytes of router
+// weights are read once, spread over the SMs), the CTAs meet at a grid-wide barrier (cooperative launch, one
+// arrival counter, bounded spin), and then every CTA repeats the tiny selection for the call's rows by itself
+// from the T*E logits (Eq. 4, the two routing rounds of Algorithm 1, one warp per row) instead of waiting for
+// a selection kernel: no second and third launch, no dependency hop between them.  CTA 0 writes the exports.
 #include "team_common.cuh"
+#include "team_topk.cuh"
 
 namespace team {
 
@@ -54,6 +62,17 @@ struct StArgs {
   const int32_t* n_items;
   float* y;                     // [T, H]
   Dims d;
+  // fused step only: router and selection run inside the kernel
+  const float* w_router;        // [E, H] fp32
+  float* logits;                // [T, E] scratch (context workspace)
+  StepPtrs st;
+  Policy p;
+  RoutePtrs r;                  // context tables (choices, classes, E_A) written by CTA 0
+  RoutePtrs ex;                 // caller's exports, members may be null
+  unsigned long long* arrivals; // grid barrier: counts CTA arrivals over all launches, never reset
+  int32_t* status;
+  long long spin_cycles;        // limit of the barrier's wait
+  int extra_arrivals;           // diagnostic: arrivals the barrier waits for beyond the grid's own (0 in normal use)
 };
 
 __device__ __forceinline__ uint32_t st_smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -109,8 +128,22 @@ __device__ __forceinline__ int st_nth_set_bit(uint32_t m, int n) {
 // shared memory: token rows | partial sums [group][slice][gate, up][16 rows][tokens] | per-warp rings.
 // ntl = token tiles of 8 (1 or 2): with 16 tokens a pass holds half the groups and a ring one slot less.
 __host__ __device__ inline int stream_slots(int ntl) { return ntl == 1 ? kStSlots : kStSlots - 1; }
-__host__ __device__ inline size_t stream_smem_bytes(int H, int ntl) {
-  return (size_t)kStRows * ntl * H * 2 + kStRedBytes + (size_t)kStWarps * stream_slots(ntl) * kStChunkBytes;
+// The fused step keeps the rows' choices and a little scratch in shared memory; a pass of 7 groups instead
+// of 8 makes the room.
+constexpr int kStFusedPass = kStPassGroups - 1;
+constexpr int kStFusedScratch = kStRedBytes / kStPassGroups;      // what the eighth group's partial sums took
+__host__ __device__ inline size_t stream_red_bytes(bool fused) {
+  return fused ? (size_t)kStRedBytes / kStPassGroups * kStFusedPass : (size_t)kStRedBytes;
+}
+__host__ __device__ inline size_t stream_smem_bytes(int H, int ntl, bool fused = false) {
+  return (size_t)kStRows * ntl * H * 2 + stream_red_bytes(fused) + (size_t)kStWarps * stream_slots(ntl) * kStChunkBytes +
+         (fused ? kStFusedScratch : 0);
+}
+
+__device__ __forceinline__ unsigned long long st_ld_acquire(const unsigned long long* p) {
+  unsigned long long v;
+  asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+  return v;
 }
 
 // CPG: 64-row chunks of a W_down slab per warp and group (H = CPG * 1024).
@@ -120,11 +153,13 @@ __host__ __device__ inline size_t stream_smem_bytes(int H, int ntl) {
 //                 selection kernel); a pass stays inside one item and the item's rows are gathered into shared
 //                 memory.  NTL = 2 (two token tiles per weight fragment) halves how often an expert that many
 //                 rows chose is streamed; its pass holds 4 groups instead of 8.
-template <int CPG, bool GATHER, int NTL>
+// FUSED = true (resident mode only): router logits, grid barrier and selection run in this kernel's prologue.
+template <int CPG, bool GATHER, int NTL, bool FUSED = false>
 __global__ void __launch_bounds__(kStThreads, 1) k_experts_stream(StArgs a) {
   static_assert(NTL == 1 || (NTL == 2 && GATHER), "two token tiles only in gather mode");
+  static_assert(!FUSED || !GATHER, "the fused step keeps all rows resident");
   constexpr int TOK = kStRows * NTL;                 // token columns
-  constexpr int PASS = kStPassGroups / NTL;          // groups per pass
+  constexpr int PASS = FUSED ? kStFusedPass : kStPassGroups / NTL;          // groups per pass
   extern __shared__ __align__(128) unsigned char st_smem[];
   __shared__ __align__(16) __nv_bfloat16 s_act[PASS * TOK * 16];               // a = silu(gate) * up of the pass: [group][token][16]
   __shared__ float s_w[kStPassGroups][kStRows];                                // routing weight of token n for group q's expert
@@ -138,6 +173,19 @@ __global__ void __launch_bounds__(kStThreads, 1) k_experts_stream(StArgs a) {
   const int I = d.I, T = d.T;
   unsigned char* xs = st_smem;                                                    // [TOK][H] bf16, 16-byte pieces swizzled
   float* red = reinterpret_cast<float*>(st_smem + (size_t)TOK * H * 2);          // [group][slice][2][16][TOK]
+  constexpr size_t RED_BYTES = FUSED ? (size_t)kStRedBytes / kStPassGroups * kStFusedPass : (size_t)kStRedBytes;
+  // fused step: the rows' choices, weights and classes live here for the whole launch
+  unsigned char* fz = st_smem + (size_t)TOK * H * 2 + RED_BYTES + (size_t)kStWarps * SLOTS * kStChunkBytes;
+  int32_t* f_idx = reinterpret_cast<int32_t*>(fz);                 // [T * k] (<= 128)
+  float* f_wt = reinterpret_cast<float*>(fz + 512);                // [T * k]
+  float* f_part = reinterpret_cast<float*>(fz + 1024);             // [warps][8] router partial sums
+  uint32_t* f_mask = reinterpret_cast<uint32_t*>(fz + 1536);       // [8 group slots][8 words] E_A
+  uint8_t* f_cls = fz + 1792;                                      // [8]
+  int32_t* f_gslot = reinterpret_cast<int32_t*>(fz + 1808);        // [8] first row of the row's group
+  int32_t* f_flag = reinterpret_cast<int32_t*>(fz + 1840);         // [1] barrier gave up
+  const int32_t* c_idx = FUSED ? f_idx : a.topk_idx;
+  const float* c_wt = FUSED ? f_wt : a.topk_w;
+  const uint8_t* c_cls = FUSED ? f_cls : a.tok_class;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int g = lane >> 2, c = lane & 3;        // fragment row (and token of the B fragment), k / token pair
   const int NG = I / 16;
@@ -146,6 +194,26 @@ __global__ void __launch_bounds__(kStThreads, 1) k_experts_stream(StArgs a) {
   constexpr int per_row = H / 8;
   constexpr int kXLoads = TOK * per_row / kStThreads;         // 16-byte pieces per thread
   uint4 xv[kXLoads];
+  // fused step: this CTA's first router weight row is requested ahead of everything (weights are never an
+  // output of the preceding kernel); warp w owns H/16 consecutive elements, RV of them per lane
+  constexpr int RV = H / (kStWarps * 32);                     // 4 (H = 2048) or 2 (H = 1024)
+  float rw[4] = {0.f, 0.f, 0.f, 0.f};
+  const int h_lane = warp * (H / kStWarps) + lane * RV;       // first hidden element of this lane
+  auto load_router_row = [&](int e) {
+    const float* src = a.w_router + (size_t)e * H + h_lane;
+    if constexpr (RV == 4) {
+      const float4 v = __ldg(reinterpret_cast<const float4*>(src));
+      rw[0] = v.x; rw[1] = v.y; rw[2] = v.z; rw[3] = v.w;
+    } else {
+      const float2 v = __ldg(reinterpret_cast<const float2*>(src));
+      rw[0] = v.x; rw[1] = v.y;
+    }
+  };
+  if constexpr (FUSED) {
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the next kernel may be scheduled behind this one
+    if ((int)blockIdx.x < d.E) load_router_row(blockIdx.x);
+    asm volatile("griddepcontrol.wait;" ::: "memory");               // x and y may come from / go to the preceding kernel
+  }
   if (!GATHER) {
 #pragma unroll
     for (int i = 0; i < kXLoads; ++i) {
@@ -153,21 +221,262 @@ __global__ void __launch_bounds__(kStThreads, 1) k_experts_stream(StArgs a) {
       xv[i] = n < T ? st_ldg_stream(a.x + (size_t)n * H + ci * 8) : make_uint4(0u, 0u, 0u, 0u);
     }
   }
-  asm volatile("griddepcontrol.wait;" ::: "memory");     // the selection kernel's tables are complete from here on
-  // the rows' choices (resident mode) are requested before the token rows are parked in shared memory, so that
-  // the two round trips overlap when this kernel did not get to start ahead of the selection kernel's end
   int e_slot[4] = {-1, -1, -1, -1};      // expert of slots lane, lane + 32, ... (T * k <= 128)
-  if (!GATHER) {
+  if constexpr (!FUSED) {
+    asm volatile("griddepcontrol.wait;" ::: "memory");     // the selection kernel's tables are complete from here on
+    // the rows' choices (resident mode) are requested before the token rows are parked in shared memory, so that
+    // the two round trips overlap when this kernel did not get to start ahead of the selection kernel's end
+    if (!GATHER) {
 #pragma unroll
-    for (int b = 0; b < 4; ++b)
-      if (b * 32 + lane < T * d.k) e_slot[b] = a.topk_idx[b * 32 + lane];
+      for (int b = 0; b < 4; ++b)
+        if (b * 32 + lane < T * d.k) e_slot[b] = a.topk_idx[b * 32 + lane];
+    }
+  }
+  // fused step: the step state of row `lane` (every warp holds a copy)
+  int f_state = TEAM_TOK_CACHED, f_pos = 0, f_group = 0, f_branch = 0;
+  float f_conf = 0.f;
+  if constexpr (FUSED) {
+    if (lane < T) {
+      f_state = a.st.tok_state[lane];
+      f_conf = a.st.conf[lane];
+      f_pos = a.st.pos[lane];
+      f_group = a.st.group[lane];
+      f_branch = a.st.branch[lane];
+    }
+  }
+  if (!GATHER) {
 #pragma unroll
     for (int i = 0; i < kXLoads; ++i) {
       const int idx = tid + i * kStThreads, n = idx / per_row, ci = idx - n * per_row;
       *reinterpret_cast<uint4*>(xs + (size_t)n * H * 2 + ((ci ^ n) << 4)) = xv[i];
     }
   }
+  if constexpr (FUSED) {
+    // the output rows that will be accumulated into start from zero: the CTAs share the job
+    {
+      const int total4 = T * H / 4;
+      for (int i = blockIdx.x * kStThreads + tid; i < total4; i += gridDim.x * kStThreads) {
+        const int t = (i * 4) / H;
+        const bool skip = (a.p.flags & TEAM_F_DCD) && a.st.tok_state[t] == TEAM_TOK_CACHED;
+        if (!skip) reinterpret_cast<float4*>(a.y)[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+      }
+    }
+    if (tid < 64) f_mask[tid] = 0u;
+    if (tid == 64) *f_flag = 0;
+    // E_A of groups nobody belongs to is empty: CTA 0 clears the tables before the present groups are filled in
+    if (blockIdx.x == 0) {
+      const int n_words64 = (d.E + 63) / 64;
+      for (int i = tid; i < d.G * n_words64; i += kStThreads) {
+        a.r.group_mask[i] = 0ull;
+        if (a.ex.group_mask) a.ex.group_mask[i] = 0ull;
+      }
+    }
+    // ---- Eq. 4 classification (needs no logits): warp 0, lane u = row u ----
+    if (warp == 0) {
+      if (lane < T && (f_group < 0 || f_group >= d.G || f_branch < 0 || f_branch > 255)) {
+        if (blockIdx.x == 0) set_status(a.status, TEAM_ERR_STATE, 1);
+        f_group = min(max(f_group, 0), d.G - 1);
+        f_branch = min(max(f_branch, 0), 255);
+      }
+      const bool decoded = f_state == TEAM_TOK_NEW || f_state == TEAM_TOK_CACHED;
+      const int lim = a.p.inclusive ? a.p.L_hot : a.p.L_hot - 1;      // |pos - j| <= lim
+      bool near = a.p.prefix_decoded && f_pos + 1 <= lim;
+      int gslot = lane;
+      for (int v = T - 1; v >= 0; --v) {
+        const int gv = __shfl_sync(0xffffffffu, f_group, v), bv = __shfl_sync(0xffffffffu, f_branch, v);
+        const int pv = __shfl_sync(0xffffffffu, f_pos, v);
+        const bool dv = __shfl_sync(0xffffffffu, (int)decoded, v) != 0;
+        if (gv == f_group) {
+          gslot = v;                                                     // ends at the group's first row
+          if (bv == f_branch && dv && abs(f_pos - pv) <= lim) near = true;
+        }
+      }
+      int cls;
+      if (f_state == TEAM_TOK_CACHED) cls = (a.p.flags & TEAM_F_DCD) ? TEAM_CLS_SKIP : TEAM_CLS_FIRST;
+      else if (f_state == TEAM_TOK_NEW || !(a.p.flags & TEAM_F_LAC)) cls = TEAM_CLS_FIRST;
+      else cls = (f_conf > a.p.tau_hot || near) ? TEAM_CLS_FIRST : TEAM_CLS_COLD;
+      if (lane >= T) cls = TEAM_CLS_SKIP;
+      // a group with no first-round row: its masked rows are all routed freely
+      bool has_first = false;
+      for (int v = 0; v < T; ++v) {
+        const int gv = __shfl_sync(0xffffffffu, f_group, v), cv = __shfl_sync(0xffffffffu, cls, v);
+        if (gv == f_group && cv == TEAM_CLS_FIRST) has_first = true;
+      }
+      if (cls == TEAM_CLS_COLD && !has_first) cls = TEAM_CLS_FIRST;
+      if (lane < kStRows) {
+        f_cls[lane] = (uint8_t)cls;
+        f_gslot[lane] = gslot;
+      }
+    }
+  }
   __syncthreads();
+
+  if constexpr (FUSED) {
+    // ---- router logits of this CTA's experts: fp32 dot products over the staged rows ----
+    const int E = d.E;
+    for (int e = blockIdx.x; e < E; e += gridDim.x) {
+      if (e != (int)blockIdx.x) load_router_row(e);
+      float acc[kStRows];
+#pragma unroll
+      for (int n = 0; n < kStRows; ++n) {
+        acc[n] = 0.f;
+        if (n < T) {
+          // RV bf16 elements of row n starting at h_lane: inside one 16-byte piece (RV divides 8)
+          const unsigned char* px = xs + (size_t)n * H * 2 + ((((h_lane >> 3) ^ n)) << 4) + (h_lane & 7) * 2;
+          if constexpr (RV == 4) {
+            const uint2 v = *reinterpret_cast<const uint2*>(px);
+            const float2 lo = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&v.x));
+            const float2 hi = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&v.y));
+            acc[n] = fmaf(rw[0], lo.x, acc[n]);
+            acc[n] = fmaf(rw[1], lo.y, acc[n]);
+            acc[n] = fmaf(rw[2], hi.x, acc[n]);
+            acc[n] = fmaf(rw[3], hi.y, acc[n]);
+          } else {
+            const uint32_t v = *reinterpret_cast<const uint32_t*>(px);
+            const float2 lo = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&v));
+            acc[n] = fmaf(rw[0], lo.x, acc[n]);
+            acc[n] = fmaf(rw[1], lo.y, acc[n]);
+          }
+        }
+        acc[n] = warp_sum(acc[n]);
+      }
+      if (lane == 0) {
+#pragma unroll
+        for (int n = 0; n < kStRows; ++n) f_part[warp * kStRows + n] = acc[n];
+      }
+      __syncthreads();
+      if (tid < T) {
+        float sum = 0.f;
+#pragma unroll
+        for (int w = 0; w < kStWarps; ++w) sum += f_part[w * kStRows + tid];      // fixed order
+        a.logits[(size_t)tid * E + e] = sum;
+      }
+      __syncthreads();
+    }
+    // ---- grid barrier: every CTA's logits (and zeroed output rows) are visible behind it ----
+    if (tid == 0) {
+      __threadfence();
+      const unsigned long long n = gridDim.x;
+      const unsigned long long old = atomicAdd(a.arrivals, 1ull);
+      const unsigned long long target = (old / n + 1ull) * n + (unsigned long long)a.extra_arrivals;
+      const long long t_begin = clock64();
+      while (st_ld_acquire(a.arrivals) < target) {
+        if (clock64() - t_begin > a.spin_cycles) {
+          *f_flag = 1;
+          break;
+        }
+        __nanosleep(32);
+      }
+    }
+    __syncthreads();
+    if (*f_flag) {
+      // the wait ran out: nothing of the step is computed, the status word says so
+      if (tid == 0) set_status(a.status, TEAM_ERR_TIMEOUT, 20);
+      return;
+    }
+    // ---- selection, repeated by every CTA: one warp per row, Algorithm 1's two rounds ----
+    float v[kMaxPerLane];
+    float row_max = 0.f, denom = 1.f;
+    const int k = d.k, ne = (E + 31) / 32;
+    const int my_cls = warp < T ? f_cls[warp] : TEAM_CLS_SKIP;
+    const bool exporter = blockIdx.x == 0;
+    if (warp < T) {
+      const int t = warp;
+      if (my_cls == TEAM_CLS_SKIP) {
+        if (lane < k) {
+          f_idx[t * k + lane] = -1;
+          f_wt[t * k + lane] = 0.f;
+        }
+        if (exporter) {
+          if (lane < k) {
+            a.r.topk_idx[t * k + lane] = -1;
+            a.r.topk_w[t * k + lane] = 0.f;
+            if (a.ex.topk_idx) a.ex.topk_idx[t * k + lane] = -1;
+            if (a.ex.topk_w) a.ex.topk_w[t * k + lane] = 0.f;
+          }
+          if (lane == 0) {
+            a.r.margin[t] = __builtin_huge_valf();
+            if (a.ex.margin) a.ex.margin[t] = __builtin_huge_valf();
+          }
+          if (a.ex.probs)
+            for (int e = lane; e < E; e += 32) a.ex.probs[(size_t)t * E + e] = 0.f;
+        }
+      } else {
+        float m = kNegInf;
+#pragma unroll
+        for (int i = 0; i < kMaxPerLane; ++i) {
+          const int e = i * 32 + lane;
+          v[i] = e < E ? __ldcg(a.logits + (size_t)t * E + e) : kNegInf;      // written by other SMs: read from L2
+          m = fmaxf(m, v[i]);
+        }
+        row_max = warp_max(m);
+        float se = 0.f;
+#pragma unroll
+        for (int i = 0; i < kMaxPerLane; ++i)
+          if (i * 32 + lane < E) se += expf(v[i] - row_max);
+        denom = warp_sum(se);
+        if (exporter && a.ex.probs) {
+#pragma unroll
+          for (int i = 0; i < kMaxPerLane; ++i) {
+            const int e = i * 32 + lane;
+            if (e < E) a.ex.probs[(size_t)t * E + e] = expf(v[i] - row_max) / denom;
+          }
+        }
+      }
+    }
+    for (int round = 1; round <= 2; ++round) {
+      if (warp < T && my_cls == (round == 1 ? TEAM_CLS_FIRST : TEAM_CLS_COLD)) {
+        const int t = warp, gs = f_gslot[t];
+        if (round == 2) {
+#pragma unroll
+          for (int i = 0; i < kMaxPerLane; ++i)
+            if (!((f_mask[gs * 8 + i] >> lane) & 1u)) v[i] = kNegInf;
+        }
+        const TopkResult tr = warp_topk(v, k, lane, ne);
+        const float w = routing_weight(tr, k, lane, row_max, denom, a.p.norm_topk);
+        if (lane < k) {
+          f_idx[t * k + lane] = tr.idx;
+          f_wt[t * k + lane] = w;
+          if (tr.idx < 0) {
+            if (exporter) set_status(a.status, TEAM_ERR_STATE, 3);
+          } else if (round == 1) {
+            atomicOr(&f_mask[gs * 8 + (tr.idx >> 5)], 1u << (tr.idx & 31));
+          }
+          if (exporter) {
+            a.r.topk_idx[t * k + lane] = tr.idx;
+            a.r.topk_w[t * k + lane] = w;
+            if (a.ex.topk_idx) a.ex.topk_idx[t * k + lane] = tr.idx;
+            if (a.ex.topk_w) a.ex.topk_w[t * k + lane] = w;
+          }
+        }
+        if (exporter && lane == 0) {
+          a.r.margin[t] = tr.margin;
+          if (a.ex.margin) a.ex.margin[t] = tr.margin;
+        }
+      }
+      __syncthreads();
+    }
+    if (exporter) {
+      if (tid < T) {
+        a.r.tok_class[tid] = f_cls[tid];
+        if (a.ex.tok_class) a.ex.tok_class[tid] = f_cls[tid];
+      }
+      // E_A of the groups that are present: written by the group's first row
+      const int n_words64 = (E + 63) / 64;
+      if (tid >= 32 && tid < 32 + T * n_words64) {
+        const int t = (tid - 32) / n_words64, wd = (tid - 32) % n_words64;
+        if (f_gslot[t] == t) {
+          const int g = min(max(a.st.group[t], 0), d.G - 1);
+          const uint64_t m = (uint64_t)f_mask[t * 8 + 2 * wd] | ((uint64_t)f_mask[t * 8 + 2 * wd + 1] << 32);
+          a.r.group_mask[(size_t)g * n_words64 + wd] = m;
+          if (a.ex.group_mask) a.ex.group_mask[(size_t)g * n_words64 + wd] = m;
+        }
+      }
+    }
+#pragma unroll
+    for (int b = 0; b < 4; ++b)
+      if (b * 32 + lane < T * k) e_slot[b] = f_idx[b * 32 + lane];
+  }
 
   // Resident mode needs no dispatch tables: with at most 8 rows every warp reads the rows' choices (T*k slots)
   // and forms the set of activated experts itself, word w of the bit set in lane w; activated expert number i
@@ -186,7 +495,7 @@ __global__ void __launch_bounds__(kStThreads, 1) k_experts_stream(StArgs a) {
       }
     }
     if (d.ns > 0) {     // shared experts are active as soon as one row is computed
-      const bool any = __ballot_sync(0xffffffffu, lane < T && a.tok_class[lane] != TEAM_CLS_SKIP) != 0u;
+      const bool any = __ballot_sync(0xffffffffu, lane < T && c_cls[lane] != TEAM_CLS_SKIP) != 0u;
       for (int sh = 0; sh < d.ns && any; ++sh)
         if (lane == ((d.E + sh) >> 5)) act_word |= 1u << ((d.E + sh) & 31);
     }
@@ -196,7 +505,7 @@ __global__ void __launch_bounds__(kStThreads, 1) k_experts_stream(StArgs a) {
   const int g_lo = (int)(n_groups * blockIdx.x / gridDim.x), g_hi = (int)(n_groups * (blockIdx.x + 1) / gridDim.x);
 
   // ---- this warp's ring and its fixed lane roles ----
-  const uint32_t ring = st_smem_u32(st_smem + (size_t)TOK * H * 2 + kStRedBytes + (size_t)warp * SLOTS * kStChunkBytes);
+  const uint32_t ring = st_smem_u32(st_smem + (size_t)TOK * H * 2 + RED_BYTES + (size_t)warp * SLOTS * kStChunkBytes);
   // phase-1 chunk: 16 rows x 128 bytes; lane copies one 16-byte piece of rows cp_row + 4j; piece p of row r sits at p ^ (r & 7)
   const int cp_row = lane >> 3, cp_piece = lane & 7;
   const uint32_t cp_off0 = cp_row * 128 + ((cp_piece ^ cp_row) << 4);          // rows cp_row, cp_row + 8 (+1024)
@@ -309,12 +618,12 @@ __global__ void __launch_bounds__(kStThreads, 1) k_experts_stream(StArgs a) {
         float wt = 0.f;
         if (lane < T) {
           if (e >= d.E) {
-            wt = a.tok_class[lane] != TEAM_CLS_SKIP ? 1.f : 0.f;      // a shared expert: every computed row, weight 1
+            wt = c_cls[lane] != TEAM_CLS_SKIP ? 1.f : 0.f;      // a shared expert: every computed row, weight 1
           } else {
             // all loads are independent of each other (no branch between them)
             for (int j = 0; j < d.k; ++j) {
-              const int ej = a.topk_idx[lane * d.k + j];
-              const float wj = a.topk_w[lane * d.k + j];
+              const int ej = c_idx[lane * d.k + j];
+              const float wj = c_wt[lane * d.k + j];
               wt = ej == e ? wj : wt;
             }
           }
@@ -463,17 +772,83 @@ static const void* stream_kernel(int hidden, int max_rows) {
   return two ? reinterpret_cast<const void*>(&k_experts_stream<2, true, 2>) : reinterpret_cast<const void*>(&k_experts_stream<2, true, 1>);
 }
 
+static const void* fused_kernel(int hidden) {
+  return hidden == 1024 ? reinterpret_cast<const void*>(&k_experts_stream<1, false, 1, true>)
+                        : reinterpret_cast<const void*>(&k_experts_stream<2, false, 1, true>);
+}
+
 cudaError_t configure_experts_stream(int hidden, int max_rows) {
   const void* fn = stream_kernel(hidden, max_rows);
   cudaError_t e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        (int)stream_smem_bytes(hidden, stream_token_tiles(max_rows)));
   if (e == cudaSuccess) e = cudaFuncSetAttribute(fn, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+  if (e == cudaSuccess && !experts_stream_gathers(max_rows)) {
+    fn = fused_kernel(hidden);
+    e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)stream_smem_bytes(hidden, 1, true));
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(fn, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+  }
   return e;
+}
+
+// The fused step can run when every CTA of the grid is resident at once (they meet at a barrier): one CTA per
+// SM fits by construction (launch bounds and shared memory allow exactly one), the occupancy query confirms it.
+bool step_fused_supported(int hidden, int max_rows, int n_experts, int grid) {
+  if (experts_stream_gathers(max_rows) || !(hidden == 1024 || hidden == 2048) || n_experts > TEAM_MAX_EXPERTS) return false;
+  int per_sm = 0;
+  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, fused_kernel(hidden), kStThreads,
+                                                    stream_smem_bytes(hidden, 1, true)) != cudaSuccess) {
+    cudaGetLastError();
+    return false;
+  }
+  int dev = 0, sms = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {
+    cudaGetLastError();
+    return false;
+  }
+  return per_sm >= 1 && grid <= per_sm * sms;
+}
+
+cudaError_t launch_step_fused(const void* x, const float* w_router, const void* w_gate, const void* w_up, const void* w_down,
+                              StepPtrs st, Workspace ws, RoutePtrs ex, float* y, Dims d, Policy p, int grid,
+                              long long spin_cycles, int extra_arrivals, cudaStream_t s) {
+  StArgs a = {};
+  a.x = static_cast<const __nv_bfloat16*>(x);
+  a.w_gate = static_cast<const __nv_bfloat16*>(w_gate);
+  a.w_up = static_cast<const __nv_bfloat16*>(w_up);
+  a.w_down = static_cast<const __nv_bfloat16*>(w_down);
+  a.y = y;
+  a.d = d;
+  a.w_router = w_router;
+  a.logits = ws.logits;
+  a.st = st;
+  a.p = p;
+  a.r = ws.r;
+  a.ex = ex;
+  a.arrivals = ws.arrivals;
+  a.status = ws.status;
+  a.spin_cycles = spin_cycles;
+  a.extra_arrivals = extra_arrivals;
+  // Cooperative: all CTAs are resident together, so the barrier's wait ends.  Programmatic serialization: the
+  // launch latency and the first router weight loads hide behind the tail of the preceding kernel.
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(grid);
+  cfg.blockDim = dim3(kStThreads);
+  cfg.dynamicSmemBytes = stream_smem_bytes(d.H, 1, true);
+  cfg.stream = s;
+  cudaLaunchAttribute attrs[2];
+  attrs[0].id = cudaLaunchAttributeCooperative;
+  attrs[0].val.cooperative = 1;
+  attrs[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attrs[1].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attrs;
+  cfg.numAttrs = 2;
+  void* params[1] = {&a};
+  return cudaLaunchKernelExC(&cfg, fused_kernel(d.H), params);
 }
 
 cudaError_t launch_experts_stream(const void* x, const void* w_gate, const void* w_up, const void* w_down, Workspace ws,
                                   float* y, Dims d, int max_rows, int grid, cudaStream_t s) {
-  StArgs a;
+  StArgs a = {};
   a.x = static_cast<const __nv_bfloat16*>(x);
   a.w_gate = static_cast<const __nv_bfloat16*>(w_gate);
   a.w_up = static_cast<const __nv_bfloat16*>(w_up);

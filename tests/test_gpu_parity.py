@@ -121,7 +121,7 @@ def test_c4_batch_sweep(seqs, weights_cache):
         P.run_schedule(shape, weights_cache(shape), steps, 0)
 
 
-def _run_stack(shape, n_layers, flags, weights_cache):
+def _run_stack(shape, n_layers, flags, weights_cache, tables=True):
     """MoE-only stack (config 5's structure): x <- x + layer(x) on computed rows, layer after layer, step after step.
 
     Every layer is checked teacher-forced (the oracle gets the activations the GPU stack actually fed into that
@@ -146,12 +146,16 @@ def _run_stack(shape, n_layers, flags, weights_cache):
             for li, layer in enumerate(layers):
                 x_in = x_dev.float().cpu().numpy()
                 out = B.alloc_routing(layer.cfg, T)
+                if not tables:
+                    out = {n: out[n] for n in P.CHOICE_TABLES}
                 y_before = y_dev.cpu().numpy()
                 B.team_moe_forward(layer.ctx, x_dev, st, out, y_dev)
                 B.team_residual_add(layer.ctx, x_dev, y_dev, T)
                 code, detail = B.team_read_status(layer.ctx)
                 assert code == B.TEAM_OK, (code, detail)
                 got = B.routing_to_host(out)
+                if not tables:
+                    got["n_rows_active"] = int((got["tok_class"] != O.CLS_SKIP).sum())
                 y_ref, ref = O.moe_forward(ocfg, layers_w[li], x_in, step["tok_state"], step["conf"], step["pos"],
                                            step["group"], step["branch"], y_prev=y_before)
                 what = f"{shape.name} stack step={si} layer={li}"
@@ -180,8 +184,9 @@ def test_c5_stack_small_shape(flags, weights_cache):
     _run_stack(W.MINI_WRAP, 8, flags, weights_cache)
 
 
-def test_c5_stack_sdar_shape_two_layers(weights_cache):
-    _run_stack(W.C2, 2, 3, weights_cache)
+@pytest.mark.parametrize("tables", [True, False], ids=["three_kernels", "one_kernel_step"])
+def test_c5_stack_sdar_shape_two_layers(weights_cache, tables):
+    _run_stack(W.C2, 2, 3, weights_cache, tables=tables)
 
 
 @pytest.mark.parametrize("side_stream", [False, True], ids=["default_stream", "own_stream_graph_replay"])
