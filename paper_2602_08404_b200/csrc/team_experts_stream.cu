@@ -251,28 +251,90 @@ __global__ void __launch_bounds__(kStThreads, 1) k_experts_stream(StArgs a) {
       *reinterpret_cast<uint4*>(xs + (size_t)n * H * 2 + ((ci ^ n) << 4)) = xv[i];
     }
   }
+  // fused step, thread 0: the barrier's target, from the arrival count as it stands before this CTA arrives.  The
+  // count is a multiple of the grid size between launches (every launch adds exactly one arrival per CTA), so
+  // whatever this launch's other CTAs have added already, rounding down gives the launch's base.
+  unsigned long long bar_target = 0ull;
   if constexpr (FUSED) {
+    if (tid == 0) {
+      const unsigned long long n = gridDim.x;
+      bar_target = (st_ld_acquire(a.arrivals) / n + 1ull) * n + (unsigned long long)a.extra_arrivals;
+    }
     // the output rows that will be accumulated into start from zero: the CTAs share the job
     {
+      const uint32_t skip_rows = (a.p.flags & TEAM_F_DCD) ? __ballot_sync(0xffffffffu, lane < T && f_state == TEAM_TOK_CACHED) : 0u;
       const int total4 = T * H / 4;
       for (int i = blockIdx.x * kStThreads + tid; i < total4; i += gridDim.x * kStThreads) {
         const int t = (i * 4) / H;
-        const bool skip = (a.p.flags & TEAM_F_DCD) && a.st.tok_state[t] == TEAM_TOK_CACHED;
-        if (!skip) reinterpret_cast<float4*>(a.y)[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (!((skip_rows >> t) & 1u)) reinterpret_cast<float4*>(a.y)[i] = make_float4(0.f, 0.f, 0.f, 0.f);
       }
     }
     if (tid < 64) f_mask[tid] = 0u;
     if (tid == 64) *f_flag = 0;
-    // E_A of groups nobody belongs to is empty: CTA 0 clears the tables before the present groups are filled in
-    if (blockIdx.x == 0) {
-      const int n_words64 = (d.E + 63) / 64;
-      for (int i = tid; i < d.G * n_words64; i += kStThreads) {
-        a.r.group_mask[i] = 0ull;
-        if (a.ex.group_mask) a.ex.group_mask[i] = 0ull;
+  }
+  __syncthreads();
+
+  // fused step: logits of the row this warp routes (warps 0 .. T-1), as order-preserving keys and as values
+  uint32_t f_key[kMaxPerLane];
+  float f_val[kMaxPerLane];
+  float f_margin = __builtin_huge_valf();
+  int f_mycls = TEAM_CLS_SKIP;
+  if constexpr (FUSED) {
+    // ---- router logits of this CTA's experts: fp32 dot products over the staged rows ----
+    const int E = d.E;
+    for (int e = blockIdx.x; e < E; e += gridDim.x) {
+      if (e != (int)blockIdx.x) load_router_row(e);
+      float acc[kStRows];
+#pragma unroll
+      for (int n = 0; n < kStRows; ++n) {
+        acc[n] = 0.f;
+        if (n < T) {
+          // RV bf16 elements of row n starting at h_lane: inside one 16-byte piece (RV divides 8)
+          const unsigned char* px = xs + (size_t)n * H * 2 + ((((h_lane >> 3) ^ n)) << 4) + (h_lane & 7) * 2;
+          if constexpr (RV == 4) {
+            const uint2 v = *reinterpret_cast<const uint2*>(px);
+            const float2 lo = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&v.x));
+            const float2 hi = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&v.y));
+            acc[n] = fmaf(rw[0], lo.x, acc[n]);
+            acc[n] = fmaf(rw[1], lo.y, acc[n]);
+            acc[n] = fmaf(rw[2], hi.x, acc[n]);
+            acc[n] = fmaf(rw[3], hi.y, acc[n]);
+          } else {
+            const uint32_t v = *reinterpret_cast<const uint32_t*>(px);
+            const float2 lo = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&v));
+            acc[n] = fmaf(rw[0], lo.x, acc[n]);
+            acc[n] = fmaf(rw[1], lo.y, acc[n]);
+          }
+          acc[n] = warp_sum(acc[n]);
+        }
+      }
+      if (lane == 0) {
+#pragma unroll
+        for (int n = 0; n < kStRows; ++n) f_part[warp * kStRows + n] = acc[n];
+      }
+      __syncthreads();
+      if (tid < T) {
+        float sum = 0.f;
+#pragma unroll
+        for (int w = 0; w < kStWarps; ++w) sum += f_part[w * kStRows + tid];      // fixed order
+        a.logits[(size_t)tid * E + e] = sum;
+      }
+      __syncthreads();
+    }
+    // ---- grid barrier: every CTA's logits (and zeroed output rows) are visible behind it.  Thread 0 arrives
+    //      and polls; meanwhile warp 1 classifies the rows (Eq. 4 needs no logits) and CTA 0 clears E_A's table ----
+    if (tid == 0) {
+      __threadfence();
+      atomicAdd(a.arrivals, 1ull);
+      const long long t_begin = clock64();
+      while (st_ld_acquire(a.arrivals) < bar_target) {
+        if (clock64() - t_begin > a.spin_cycles) {
+          *f_flag = 1;
+          break;
+        }
       }
     }
-    // ---- Eq. 4 classification (needs no logits): warp 0, lane u = row u ----
-    if (warp == 0) {
+    if (warp == 1) {
       if (lane < T && (f_group < 0 || f_group >= d.G || f_branch < 0 || f_branch > 255)) {
         if (blockIdx.x == 0) set_status(a.status, TEAM_ERR_STATE, 1);
         f_group = min(max(f_group, 0), d.G - 1);
@@ -308,64 +370,12 @@ __global__ void __launch_bounds__(kStThreads, 1) k_experts_stream(StArgs a) {
         f_gslot[lane] = gslot;
       }
     }
-  }
-  __syncthreads();
-
-  if constexpr (FUSED) {
-    // ---- router logits of this CTA's experts: fp32 dot products over the staged rows ----
-    const int E = d.E;
-    for (int e = blockIdx.x; e < E; e += gridDim.x) {
-      if (e != (int)blockIdx.x) load_router_row(e);
-      float acc[kStRows];
-#pragma unroll
-      for (int n = 0; n < kStRows; ++n) {
-        acc[n] = 0.f;
-        if (n < T) {
-          // RV bf16 elements of row n starting at h_lane: inside one 16-byte piece (RV divides 8)
-          const unsigned char* px = xs + (size_t)n * H * 2 + ((((h_lane >> 3) ^ n)) << 4) + (h_lane & 7) * 2;
-          if constexpr (RV == 4) {
-            const uint2 v = *reinterpret_cast<const uint2*>(px);
-            const float2 lo = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&v.x));
-            const float2 hi = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&v.y));
-            acc[n] = fmaf(rw[0], lo.x, acc[n]);
-            acc[n] = fmaf(rw[1], lo.y, acc[n]);
-            acc[n] = fmaf(rw[2], hi.x, acc[n]);
-            acc[n] = fmaf(rw[3], hi.y, acc[n]);
-          } else {
-            const uint32_t v = *reinterpret_cast<const uint32_t*>(px);
-            const float2 lo = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&v));
-            acc[n] = fmaf(rw[0], lo.x, acc[n]);
-            acc[n] = fmaf(rw[1], lo.y, acc[n]);
-          }
-        }
-        acc[n] = warp_sum(acc[n]);
-      }
-      if (lane == 0) {
-#pragma unroll
-        for (int n = 0; n < kStRows; ++n) f_part[warp * kStRows + n] = acc[n];
-      }
-      __syncthreads();
-      if (tid < T) {
-        float sum = 0.f;
-#pragma unroll
-        for (int w = 0; w < kStWarps; ++w) sum += f_part[w * kStRows + tid];      // fixed order
-        a.logits[(size_t)tid * E + e] = sum;
-      }
-      __syncthreads();
-    }
-    // ---- grid barrier: every CTA's logits (and zeroed output rows) are visible behind it ----
-    if (tid == 0) {
-      __threadfence();
-      const unsigned long long n = gridDim.x;
-      const unsigned long long old = atomicAdd(a.arrivals, 1ull);
-      const unsigned long long target = (old / n + 1ull) * n + (unsigned long long)a.extra_arrivals;
-      const long long t_begin = clock64();
-      while (st_ld_acquire(a.arrivals) < target) {
-        if (clock64() - t_begin > a.spin_cycles) {
-          *f_flag = 1;
-          break;
-        }
-        __nanosleep(32);
+    if (blockIdx.x == 0 && tid >= 64) {
+      // E_A of groups nobody belongs to is empty: the table is cleared before the present groups are filled in
+      const int n_words64 = (E + 63) / 64;
+      for (int i = tid - 64; i < d.G * n_words64; i += kStThreads - 64) {
+        a.r.group_mask[i] = 0ull;
+        if (a.ex.group_mask) a.ex.group_mask[i] = 0ull;
       }
     }
     __syncthreads();
@@ -374,108 +384,42 @@ __global__ void __launch_bounds__(kStThreads, 1) k_experts_stream(StArgs a) {
       if (tid == 0) set_status(a.status, TEAM_ERR_TIMEOUT, 20);
       return;
     }
-    // ---- selection, repeated by every CTA: one warp per row, Algorithm 1's two rounds ----
-    float v[kMaxPerLane];
-    float row_max = 0.f, denom = 1.f;
+    // ---- Algorithm 1, first round: one warp per row.  Only the picks are on the way to the first weight
+    //      bytes: the activated set is the union of the first-round choices (cold rows add nothing to it), so
+    //      the second round, the softmax and the routing weights wait until the first copies are in flight ----
     const int k = d.k, ne = (E + 31) / 32;
-    const int my_cls = warp < T ? f_cls[warp] : TEAM_CLS_SKIP;
-    const bool exporter = blockIdx.x == 0;
     if (warp < T) {
       const int t = warp;
-      if (my_cls == TEAM_CLS_SKIP) {
+      f_mycls = f_cls[t];
+      if (f_mycls == TEAM_CLS_SKIP) {
         if (lane < k) {
           f_idx[t * k + lane] = -1;
           f_wt[t * k + lane] = 0.f;
         }
-        if (exporter) {
-          if (lane < k) {
-            a.r.topk_idx[t * k + lane] = -1;
-            a.r.topk_w[t * k + lane] = 0.f;
-            if (a.ex.topk_idx) a.ex.topk_idx[t * k + lane] = -1;
-            if (a.ex.topk_w) a.ex.topk_w[t * k + lane] = 0.f;
-          }
-          if (lane == 0) {
-            a.r.margin[t] = __builtin_huge_valf();
-            if (a.ex.margin) a.ex.margin[t] = __builtin_huge_valf();
-          }
-          if (a.ex.probs)
-            for (int e = lane; e < E; e += 32) a.ex.probs[(size_t)t * E + e] = 0.f;
-        }
       } else {
-        float m = kNegInf;
 #pragma unroll
         for (int i = 0; i < kMaxPerLane; ++i) {
           const int e = i * 32 + lane;
-          v[i] = e < E ? __ldcg(a.logits + (size_t)t * E + e) : kNegInf;      // written by other SMs: read from L2
-          m = fmaxf(m, v[i]);
+          f_val[i] = (i < ne && e < E) ? __ldcg(a.logits + (size_t)t * E + e) : kNegInf;      // written by other SMs: read from L2
+          f_key[i] = float_key(f_val[i]);
         }
-        row_max = warp_max(m);
-        float se = 0.f;
-#pragma unroll
-        for (int i = 0; i < kMaxPerLane; ++i)
-          if (i * 32 + lane < E) se += expf(v[i] - row_max);
-        denom = warp_sum(se);
-        if (exporter && a.ex.probs) {
-#pragma unroll
-          for (int i = 0; i < kMaxPerLane; ++i) {
-            const int e = i * 32 + lane;
-            if (e < E) a.ex.probs[(size_t)t * E + e] = expf(v[i] - row_max) / denom;
+        if (f_mycls == TEAM_CLS_FIRST) {
+          const int gs = f_gslot[t];
+          const int n = warp_topk_picks(f_key, ne, k, lane,
+                                        [&](int j, int e, uint32_t key) {
+                                          f_idx[t * k + j] = e;
+                                          f_wt[t * k + j] = key_float(key);       // the logit; turned into the weight later
+                                          atomicOr(&f_mask[gs * 8 + (e >> 5)], 1u << (e & 31));
+                                        },
+                                        f_margin);
+          if (n < k) {
+            if (lane >= n && lane < k) f_idx[t * k + lane] = -1;
+            if (blockIdx.x == 0 && lane == 0) set_status(a.status, TEAM_ERR_STATE, 3);
           }
         }
       }
     }
-    for (int round = 1; round <= 2; ++round) {
-      if (warp < T && my_cls == (round == 1 ? TEAM_CLS_FIRST : TEAM_CLS_COLD)) {
-        const int t = warp, gs = f_gslot[t];
-        if (round == 2) {
-#pragma unroll
-          for (int i = 0; i < kMaxPerLane; ++i)
-            if (!((f_mask[gs * 8 + i] >> lane) & 1u)) v[i] = kNegInf;
-        }
-        const TopkResult tr = warp_topk(v, k, lane, ne);
-        const float w = routing_weight(tr, k, lane, row_max, denom, a.p.norm_topk);
-        if (lane < k) {
-          f_idx[t * k + lane] = tr.idx;
-          f_wt[t * k + lane] = w;
-          if (tr.idx < 0) {
-            if (exporter) set_status(a.status, TEAM_ERR_STATE, 3);
-          } else if (round == 1) {
-            atomicOr(&f_mask[gs * 8 + (tr.idx >> 5)], 1u << (tr.idx & 31));
-          }
-          if (exporter) {
-            a.r.topk_idx[t * k + lane] = tr.idx;
-            a.r.topk_w[t * k + lane] = w;
-            if (a.ex.topk_idx) a.ex.topk_idx[t * k + lane] = tr.idx;
-            if (a.ex.topk_w) a.ex.topk_w[t * k + lane] = w;
-          }
-        }
-        if (exporter && lane == 0) {
-          a.r.margin[t] = tr.margin;
-          if (a.ex.margin) a.ex.margin[t] = tr.margin;
-        }
-      }
-      __syncthreads();
-    }
-    if (exporter) {
-      if (tid < T) {
-        a.r.tok_class[tid] = f_cls[tid];
-        if (a.ex.tok_class) a.ex.tok_class[tid] = f_cls[tid];
-      }
-      // E_A of the groups that are present: written by the group's first row
-      const int n_words64 = (E + 63) / 64;
-      if (tid >= 32 && tid < 32 + T * n_words64) {
-        const int t = (tid - 32) / n_words64, wd = (tid - 32) % n_words64;
-        if (f_gslot[t] == t) {
-          const int g = min(max(a.st.group[t], 0), d.G - 1);
-          const uint64_t m = (uint64_t)f_mask[t * 8 + 2 * wd] | ((uint64_t)f_mask[t * 8 + 2 * wd + 1] << 32);
-          a.r.group_mask[(size_t)g * n_words64 + wd] = m;
-          if (a.ex.group_mask) a.ex.group_mask[(size_t)g * n_words64 + wd] = m;
-        }
-      }
-    }
-#pragma unroll
-    for (int b = 0; b < 4; ++b)
-      if (b * 32 + lane < T * k) e_slot[b] = f_idx[b * 32 + lane];
+    __syncthreads();
   }
 
   // Resident mode needs no dispatch tables: with at most 8 rows every warp reads the rows' choices (T*k slots)
@@ -485,13 +429,21 @@ __global__ void __launch_bounds__(kStThreads, 1) k_experts_stream(StArgs a) {
   uint32_t act_word = 0u;
   const int n_words = (d.E + d.ns + 31) >> 5;
   if (!GATHER) {
+    if constexpr (FUSED) {
+      // the union of the groups' necessary sets, straight from shared memory: word w in lane w
+      if (lane < 8) {
 #pragma unroll
-    for (int b = 0; b < 4; ++b) {
-      if (b * 32 >= T * d.k) break;
-      const int e = e_slot[b];
-      for (int w = 0; w < n_words; ++w) {
-        const uint32_t m = __reduce_or_sync(0xffffffffu, (e >= 0 && (e >> 5) == w) ? 1u << (e & 31) : 0u);
-        if (lane == w) act_word |= m;
+        for (int gs = 0; gs < kStRows; ++gs) act_word |= f_mask[gs * 8 + lane];
+      }
+    } else {
+#pragma unroll
+      for (int b = 0; b < 4; ++b) {
+        if (b * 32 >= T * d.k) break;
+        const int e = e_slot[b];
+        for (int w = 0; w < n_words; ++w) {
+          const uint32_t m = __reduce_or_sync(0xffffffffu, (e >= 0 && (e >> 5) == w) ? 1u << (e & 31) : 0u);
+          if (lane == w) act_word |= m;
+        }
       }
     }
     if (d.ns > 0) {     // shared experts are active as soon as one row is computed
@@ -523,6 +475,88 @@ __global__ void __launch_bounds__(kStThreads, 1) k_experts_stream(StArgs a) {
   const __nv_bfloat16* wmat = tile ? a.w_up : a.w_gate;
   const uint64_t pol = st_stream_policy();
 
+  // fused step: what the selection still owes once the activated set is known -- the second routing round (cold
+  // rows inside E_A), the softmax denominators and routing weights, and CTA 0's exports.  Run once per CTA by
+  // warps 0 .. T-1, in the shadow of the first weight copies' latency (or after the loop if this CTA has no
+  // group at all); the routing weights are first read after the barrier that ends phase 1.
+  bool late_done = false;
+  auto late_select = [&]() {
+    if constexpr (FUSED) {
+      if (warp < T) {
+        const int t = warp, k = d.k, E = d.E, ne = (E + 31) / 32;
+        const bool exporter = blockIdx.x == 0;
+        float row_max = 0.f, denom = 1.f, w = 0.f;
+        if (f_mycls == TEAM_CLS_COLD) {
+          const int gs = f_gslot[t];
+#pragma unroll
+          for (int i = 0; i < kMaxPerLane; ++i)
+            if (!((f_mask[gs * 8 + i] >> lane) & 1u)) f_key[i] = 0x007fffffu;      // outside E_A: no candidate
+          const int n = warp_topk_picks(f_key, ne, k, lane,
+                                        [&](int j, int e, uint32_t key) {
+                                          f_idx[t * k + j] = e;
+                                          f_wt[t * k + j] = key_float(key);
+                                        },
+                                        f_margin);
+          if (n < k) {
+            if (lane >= n && lane < k) f_idx[t * k + lane] = -1;
+            if (exporter && lane == 0) set_status(a.status, TEAM_ERR_STATE, 3);
+          }
+        }
+        __syncwarp();
+        if (f_mycls != TEAM_CLS_SKIP) {
+          float m = kNegInf;
+#pragma unroll
+          for (int i = 0; i < kMaxPerLane; ++i) m = fmaxf(m, f_val[i]);
+          row_max = warp_max(m);
+          float se = 0.f;
+#pragma unroll
+          for (int i = 0; i < kMaxPerLane; ++i)
+            if (i * 32 + lane < E) se += expf(f_val[i] - row_max);
+          denom = warp_sum(se);
+          TopkResult tr;
+          tr.idx = lane < k ? f_idx[t * k + lane] : -1;
+          tr.val = lane < k ? f_wt[t * k + lane] : kNegInf;
+          tr.margin = f_margin;
+          tr.top = row_max;
+          w = routing_weight(tr, k, lane, row_max, denom, a.p.norm_topk);
+          if (tr.idx < 0) w = 0.f;
+          __syncwarp();
+          if (lane < k) f_wt[t * k + lane] = w;
+        }
+        if (exporter) {
+          if (lane < k) {
+            const int e = f_idx[t * k + lane];
+            a.r.topk_idx[t * k + lane] = e;
+            a.r.topk_w[t * k + lane] = w;
+            if (a.ex.topk_idx) a.ex.topk_idx[t * k + lane] = e;
+            if (a.ex.topk_w) a.ex.topk_w[t * k + lane] = w;
+          }
+          if (lane == 0) {
+            a.r.margin[t] = f_margin;
+            if (a.ex.margin) a.ex.margin[t] = f_margin;
+            a.r.tok_class[t] = (uint8_t)f_mycls;
+            if (a.ex.tok_class) a.ex.tok_class[t] = (uint8_t)f_mycls;
+          }
+          if (a.ex.probs) {
+#pragma unroll
+            for (int i = 0; i < kMaxPerLane; ++i) {
+              const int e = i * 32 + lane;
+              if (e < E) a.ex.probs[(size_t)t * E + e] = f_mycls != TEAM_CLS_SKIP ? expf(f_val[i] - row_max) / denom : 0.f;
+            }
+          }
+          // E_A of the groups that are present: written by the group's first row
+          const int n_words64 = (E + 63) / 64;
+          const int g = min(max(__shfl_sync(0xffffffffu, f_group, t), 0), d.G - 1);
+          if (f_gslot[t] == t && lane < n_words64) {
+            const uint64_t mk = (uint64_t)f_mask[t * 8 + 2 * lane] | ((uint64_t)f_mask[t * 8 + 2 * lane + 1] << 32);
+            a.r.group_mask[(size_t)g * n_words64 + lane] = mk;
+            if (a.ex.group_mask) a.ex.group_mask[(size_t)g * n_words64 + lane] = mk;
+          }
+        }
+      }
+    }
+  };
+
   int cur_item = -1;
   for (int s_lo = g_lo, s_hi; s_lo < g_hi; s_lo = s_hi) {
     s_hi = min(g_hi, s_lo + PASS);
@@ -546,6 +580,28 @@ __global__ void __launch_bounds__(kStThreads, 1) k_experts_stream(StArgs a) {
         left = left >= c ? left - c : -1;
       }
     }
+    // ---- routing weights of the pass's experts, per group and token (read in phase 2, after the barriers):
+    //      warp q < ng looks group q's expert up in the rows' choices ----
+    auto pass_weights = [&]() {
+      const int item = __shfl_sync(0xffffffffu, my_item, warp), e = __shfl_sync(0xffffffffu, my_e, warp);
+      if (lane == 0) s_item[warp] = item;
+      if (lane < kStRows) {
+        float wt = 0.f;
+        if (lane < T) {
+          if (e >= d.E) {
+            wt = c_cls[lane] != TEAM_CLS_SKIP ? 1.f : 0.f;      // a shared expert: every computed row, weight 1
+          } else {
+            // all loads are independent of each other (no branch between them)
+            for (int j = 0; j < d.k; ++j) {
+              const int ej = c_idx[lane * d.k + j];
+              const float wj = c_wt[lane * d.k + j];
+              wt = ej == e ? wj : wt;
+            }
+          }
+        }
+        s_w[warp][lane] = wt;
+      }
+    };
     // ---- issue side: phase-1 chunks, then phase-2 chunks, then empty groups ----
     const int n1 = ng * NCH, n2 = ng * CPG;
     int n_issued = 0, iq = 0, icc = 0;
@@ -610,26 +666,12 @@ __global__ void __launch_bounds__(kStThreads, 1) k_experts_stream(StArgs a) {
         __syncthreads();
         cur_item = item0;
       }
-    } else if (warp < ng) {
-      // ---- routing weights of the pass's experts, per group and token (read in phase 2, after the barriers) ----
-      const int item = __shfl_sync(0xffffffffu, my_item, warp), e = __shfl_sync(0xffffffffu, my_e, warp);
-      if (lane == 0) s_item[warp] = item;
-      if (lane < kStRows) {
-        float wt = 0.f;
-        if (lane < T) {
-          if (e >= d.E) {
-            wt = c_cls[lane] != TEAM_CLS_SKIP ? 1.f : 0.f;      // a shared expert: every computed row, weight 1
-          } else {
-            // all loads are independent of each other (no branch between them)
-            for (int j = 0; j < d.k; ++j) {
-              const int ej = c_idx[lane * d.k + j];
-              const float wj = c_wt[lane * d.k + j];
-              wt = ej == e ? wj : wt;
-            }
-          }
-        }
-        s_w[warp][lane] = wt;
-      }
+    } else if (!FUSED && warp < ng) {
+      pass_weights();
+    }
+    if (FUSED && !late_done) {
+      late_select();
+      late_done = true;
     }
 
     // ---- phase 1 ----
@@ -677,6 +719,7 @@ __global__ void __launch_bounds__(kStThreads, 1) k_experts_stream(StArgs a) {
       }
     }
     __syncthreads();
+    if (FUSED && warp < ng) pass_weights();      // the routing weights are complete by now (late selection)
     // ---- sum the slices, SwiGLU ----
     for (int idx = tid; idx < ng * 16 * TOK; idx += kStThreads) {
       const int qq = idx / (16 * TOK), r = (idx / TOK) & 15, n = idx % TOK;
@@ -747,6 +790,7 @@ __global__ void __launch_bounds__(kStThreads, 1) k_experts_stream(StArgs a) {
     st_wait_group<0>();     // only empty groups can be pending here
     __syncthreads();        // s_act, s_w and the partial sums are free for the next pass
   }
+  if (FUSED && !late_done) late_select();      // a CTA without any group still owes its part (CTA 0: the exports)
 }
 
 // Few rows: all rows resident.  Up to kStGatherMaxRows rows: work items whose rows are gathered per item, of

@@ -28,52 +28,104 @@ __device__ __forceinline__ float key_float(uint32_t k) {
   return __uint_as_float((k & 0x80000000u) ? (k & 0x7fffffffu) : ~k);
 }
 
+// Core of the selection.  key[i] is the key of expert i*32+lane (float_key(-inf) for a non-candidate); only the
+// first ne = ceil(E / 32) entries are looked at.  Picks the k largest keys in descending order, ties to the
+// lower expert id, and calls on_pick(j, expert, key) for the j-th pick ON THE LANE THAT HOLDS IT (nothing is
+// broadcast).  Picked keys are retired in place.  Returns the number of picks made (< k only if fewer than k
+// candidates exist); margin_out (all lanes) = logit of the last pick minus the best logit left (+inf if none).
+//
+// One pick is a short dependent chain: warp-wide maximum of the lanes' current best keys (one redux), a ballot
+// of who holds it, and only the holder updates its state; two or more holders (equal logits in different
+// lanes) take a second redux for the lowest expert id.
+template <typename OnPick>
+__device__ __forceinline__ int warp_topk_picks(uint32_t (&key)[kMaxPerLane], int ne, int k, int lane, OnPick&& on_pick,
+                                               float& margin_out) {
+  const uint32_t key_neg_inf = 0x007fffffu;            // float_key(-inf)
+  uint32_t bk = key_neg_inf;
+  int bi = 0;
+  auto local_best = [&]() {
+    bk = key_neg_inf;
+    bi = 0;
+#pragma unroll
+    for (int i = 0; i < kMaxPerLane; ++i) {
+      // ascending expert id within the lane, strict '>' keeps the lower id on ties
+      if (i < ne && key[i] > bk) {
+        bk = key[i];
+        bi = i;
+      }
+    }
+  };
+  local_best();
+  float last = kNegInf;
+  margin_out = __builtin_huge_valf();
+  int n = 0;
+  for (int j = 0; j <= k; ++j) {
+    const uint32_t wk = __reduce_max_sync(0xffffffffu, bk);
+    if (wk == key_neg_inf) break;                       // no candidate left
+    if (j == k) {
+      margin_out = last - key_float(wk);
+      break;
+    }
+    const uint32_t holders = __ballot_sync(0xffffffffu, bk == wk);
+    int win_lane = __ffs(holders) - 1;
+    if (holders & (holders - 1u)) {
+      const uint32_t wi = __reduce_min_sync(0xffffffffu, bk == wk ? (uint32_t)(bi * 32 + lane) : 0x7fffffffu);
+      win_lane = (int)(wi & 31u);
+    }
+    if (lane == win_lane) {
+      on_pick(j, bi * 32 + lane, wk);
+#pragma unroll
+      for (int i = 0; i < kMaxPerLane; ++i)
+        if (i == bi) key[i] = key_neg_inf;
+      local_best();
+    }
+    last = key_float(wk);
+    n = j + 1;
+  }
+  return n;
+}
+
 // v[i] is the logit of expert i*32+lane, or -inf if that expert is not a candidate
 // (beyond E, or outside the allowed set); only the first ne = ceil(E / 32) entries are looked at.
-// The logits are turned into keys once.  Each of the k+1 rounds takes the warp-wide maximum key and
-// then the lowest expert id among the lanes that hold it, and retires that key.
+// Lane j < k receives the j-th choice.
 __device__ __forceinline__ TopkResult warp_topk(const float (&v)[kMaxPerLane], int k, int lane, int ne = kMaxPerLane) {
   TopkResult r;
   r.idx = -1;
   r.val = kNegInf;
   r.top = kNegInf;
-  r.margin = __builtin_huge_valf();
-  float last = kNegInf;
-  const uint32_t key_neg_inf = float_key(kNegInf);
   uint32_t key[kMaxPerLane];
 #pragma unroll
-  for (int i = 0; i < kMaxPerLane; ++i) key[i] = i < ne ? float_key(v[i]) : key_neg_inf;
-  for (int j = 0; j <= k; ++j) {
-    uint32_t bk = key_neg_inf;
-    int bi = 0;
+  for (int i = 0; i < kMaxPerLane; ++i) key[i] = i < ne ? float_key(v[i]) : 0x007fffffu;
+  // the holder of a pick remembers it; afterwards pick j moves to lane j (one shuffle per pick, off the picks'
+  // dependent chain)
+  int order[kMaxPerLane];             // this lane's key i was picked as pick number order[i] (-1: not picked)
 #pragma unroll
-    for (int i = 0; i < kMaxPerLane; ++i) {
-      if (i >= ne) break;
-      // ascending expert id within the lane, strict '>' keeps the lower id on ties
-      if (key[i] > bk) {
-        bk = key[i];
-        bi = i;
-      }
-    }
-    const uint32_t wk = __reduce_max_sync(0xffffffffu, bk);
-    const bool none = wk == key_neg_inf;
-    const int wi = (int)__reduce_min_sync(0xffffffffu, (bk == wk && !none) ? (uint32_t)(bi * 32 + lane) : 0x7fffffffu);
-    const float bv = none ? kNegInf : key_float(wk);
-    if (j == 0) r.top = bv;
-    if (j < k) {
-      if (lane == j) {
-        r.idx = none ? -1 : wi;
-        r.val = bv;
-      }
-      last = bv;
-      if (!none && (wi & 31) == lane) {
+  for (int i = 0; i < kMaxPerLane; ++i) order[i] = -1;
+  const int n = warp_topk_picks(key, ne, k, lane,
+                                [&](int j, int e, uint32_t) {
 #pragma unroll
-        for (int i = 0; i < kMaxPerLane; ++i)
-          if (i == (wi >> 5)) key[i] = key_neg_inf;
+                                  for (int i = 0; i < kMaxPerLane; ++i)
+                                    if (i == (e >> 5)) order[i] = j;
+                                },
+                                r.margin);
+  for (int j = 0; j < n; ++j) {
+    int slot = -1;
+    float mine_val = 0.f;
+#pragma unroll
+    for (int i = 0; i < kMaxPerLane; ++i)
+      if (order[i] == j) {
+        slot = i;
+        mine_val = v[i];
       }
-    } else {
-      r.margin = none ? __builtin_huge_valf() : last - bv;
+    const uint32_t holder = __ballot_sync(0xffffffffu, slot >= 0);
+    const int src = __ffs(holder) - 1;
+    const int e = __shfl_sync(0xffffffffu, slot * 32 + lane, src);
+    const float val = __shfl_sync(0xffffffffu, mine_val, src);
+    if (lane == j) {
+      r.idx = e;
+      r.val = val;
     }
+    if (j == 0) r.top = val;
   }
   return r;
 }
