@@ -56,6 +56,8 @@ def parse_args(argv=None):
                          "branches x 4; paper: c2 shape, block 32 x 4 branches in one group; c5: stack of c2 layers, block loop")
     ap.add_argument("--seqs", type=int, default=1, help="sequences of the c4 batch sweep")
     ap.add_argument("--blocks", type=int, default=64, help="decoding blocks of the c5 stack run")
+    ap.add_argument("--expert-kernel", default="auto", choices=["auto", "stream", "tile"],
+                    help="auto: the library's choice by rows per call; stream: weight-streaming kernel; tile: tcgen05 grouped GEMMs")
     return ap.parse_args(argv)
 
 
@@ -233,17 +235,27 @@ def run_layer(args):
     R = args.layers or 8
 
     # R independent layers, generated on the device (seeded); layer 0 also goes to the host for the oracle leg
-    layers, packed = [], []
+    layers, packed, tiles = [], [], []
+    want_tiles = args.expert_kernel == "tile" or (args.expert_kernel == "auto" and T >= 64)
+    want_classic = not want_tiles or args.expert_kernel == "stream"
     for r in range(R):
         wr, wg, wu, wd = W.device_layer_weights(shape, 1000 + r, dev)
-        layers.append((wr, wg, wu, wd if r == 0 else None))
-        packed.append(B.team_pack_w_down(wd))      # the layout the library reads; row-major kept for the oracle leg
+        # the layouts the library reads; layer 0's row-major copies are kept for the oracle leg
+        tiles.append(B.team_pack_w_tiles(wg, wu, wd) if want_tiles else (None, None))
+        packed.append(B.team_pack_w_down(wd) if want_classic else None)
+        keep = r == 0 or want_classic
+        layers.append((wr, wg if keep else None, wu if keep else None, wd if r == 0 else None))
     cfg = B.make_config(H, E, k, I, ns, max_rows=T, max_groups=shape.seqs, dtype=B.TEAM_DTYPE_BF16, flags=args.flags,
                         tau_hot=shape.tau_hot, L_hot=shape.L_hot)
     ctxs = []
     for r in range(R):
         c = B.team_create(cfg)
-        B.team_set_weights(c, *layers[r][:3], packed[r])
+        if want_classic:
+            B.team_set_weights(c, *layers[r][:3], packed[r], *tiles[r])
+        else:
+            B.team_set_weights(c, layers[r][0], None, None, None, *tiles[r])
+        if args.expert_kernel != "auto":
+            B.team_debug_knob(c, B.TEAM_KNOB_EXPERT_KERNEL, 1 if args.expert_kernel == "stream" else 2)
         ctxs.append(c)
 
     x_dev = [B.to_device(s["x"], B.TEAM_DTYPE_BF16, dev) for s in steps_host]

@@ -88,8 +88,11 @@ typedef struct {
   int32_t inter;       /* I; multiple of 64 for bf16, of 16 for fp32                     */
   int32_t n_shared;    /* always-on experts appended after the routed ones              */
   int32_t max_rows;    /* largest n_rows of any call on this context; it also picks the
-                          expert kernel's mode (bf16, H 1024 or 2048): <= 8 rows all
-                          resident, <= 64 items of 8 token-slots, above items of 16     */
+                          expert kernel (bf16).  Hidden size 1024 or 2048 and fewer than 64
+                          rows: the weight-streaming kernel on the row-major / slab layout
+                          (<= 8 rows all resident, else work items of 8 token-slots).
+                          Otherwise: the tensor-memory (tcgen05) grouped GEMMs on the
+                          tile-major layout of team_pack_w_tiles()                      */
   int32_t max_groups;  /* group ids are in [0, max_groups), <= TEAM_MAX_GROUPS; branch ids in [0, 256) */
   int32_t dtype;       /* TEAM_DTYPE_F32: x and expert weights fp32 (plain FMA kernels);
                           TEAM_DTYPE_BF16: x and expert weights bf16, fp32 accumulation
@@ -104,10 +107,14 @@ typedef struct {
 
 typedef struct {
   const void *w_router; /* fp32 [E, H] row-major                                          */
+  /* Expert weights come in two layouts; a context needs the one its expert kernel reads (see max_rows in
+     team_config) and accepts both.  Set the pointers of a layout you do not provide to NULL. */
   const void *w_gate;   /* [E + n_shared, I, H] row-major, dtype per config               */
   const void *w_up;     /* [E + n_shared, I, H]                                           */
   const void *w_down;   /* [E + n_shared, I/16, H, 16]: Eq. 1's W_down [H, I] of every expert
                            stored in slabs of 16 columns, as team_pack_w_down() writes it */
+  const void *w_gu_tiles;   /* bf16 only: gate and up projections as 16 KB tensor-core tiles, */
+  const void *w_down_tiles; /* and the down projection likewise, as team_pack_w_tiles() writes them */
 } team_weights;
 
 /* State carried from the previous denoising step (Algorithm 1 inputs D, M; Eq. 4). */
@@ -147,7 +154,9 @@ int team_create(const team_config *cfg, team_ctx **out);
 int team_destroy(team_ctx *ctx);
 
 /* Borrow the layer's weights (device pointers, 16-byte aligned; bf16 expert
- * weights 128-byte aligned).  May be called again to switch layers; the switch
+ * weights 128-byte aligned).  w_router is required, and at least one complete
+ * layout of the expert weights; a call whose expert kernel needs a layout that
+ * was not given returns TEAM_ERR_ARG.  May be called again to switch layers; the switch
  * takes effect for calls issued afterwards (pointers are passed by value at
  * launch). */
 int team_set_weights(team_ctx *ctx, const team_weights *w);
@@ -164,6 +173,21 @@ int team_set_weights(team_ctx *ctx, const team_weights *w);
  * Errors: TEAM_ERR_ARG, TEAM_ERR_SHAPE, TEAM_ERR_CUDA. */
 int team_pack_w_down(const void *src, void *dst, int n_experts_total, int hidden,
                      int inter, int dtype, void *stream);
+
+/* Tile-major copy of a layer's expert weights for the tensor-memory kernels (bf16): Eq. 1's three projections
+ * cut into [128 rows x 64 k] tiles of 16 KB, each contiguous and already in the 128-byte-swizzled K-major layout
+ * the tensor core reads, so that a pipeline stage is one bulk copy.
+ *   gu_tiles   [n_experts_total][I/64][H/64][128][64]: tile row blk*32 + m*16 + i holds row (u*64 + blk*16 + i) of
+ *              W_gate (m = 0) or W_up (m = 1), k-block kb; 16-byte piece p of tile row r is stored at p ^ (r & 7).
+ *   down_tiles [n_experts_total][H/128][I/64][128][64]: tile row r holds row ht*128 + r of W_down [H, I], columns
+ *              kb*64 ...; same piece swizzle.
+ * Sources are row-major device tensors ([.., I, H], [.., I, H], [.., H, I]), 16-byte aligned; destinations are
+ * device buffers of the same total size (gu_tiles: both matrices), 128-byte aligned, not overlapping the
+ * sources; all stay owned by the caller, who may free the row-major copies afterwards.  hidden must be a
+ * multiple of 128, inter of 64.  Asynchronous on `stream`; needs no context.
+ * Errors: TEAM_ERR_ARG, TEAM_ERR_SHAPE, TEAM_ERR_CUDA. */
+int team_pack_w_tiles(const void *w_gate, const void *w_up, const void *w_down, void *gu_tiles, void *down_tiles,
+                      int n_experts_total, int hidden, int inter, void *stream);
 
 /* Change flags / tau_hot / L_hot / hot_dist_inclusive / prefix_decoded /
  * norm_topk of an existing context (shapes and dtype must be unchanged). */
@@ -272,8 +296,11 @@ int team_debug_force_simt(team_ctx *ctx, int on);
  *   TEAM_KNOB_EXTRA_ARRIVALS (0/1): 1 makes that barrier wait for one arrival that never comes, so that the
  *     give-up path can be exercised (with a short limit) without any kernel hanging; y is then left unspecified
  *     for the computed rows of that call.
+ *   TEAM_KNOB_EXPERT_KERNEL (0/1/2): 0 lets max_rows choose the expert kernel of a bf16 context, 1 asks for the
+ *     weight-streaming kernel, 2 for the tensor-memory kernels (ignored where the shape does not allow the kernel);
+ *     the weight layout that kernel reads must have been given.
  * Errors: TEAM_ERR_ARG. */
-enum { TEAM_KNOB_NO_FUSE = 1, TEAM_KNOB_EXTRA_ARRIVALS = 2, TEAM_KNOB_WAIT_LIMIT_US = 3 };
+enum { TEAM_KNOB_NO_FUSE = 1, TEAM_KNOB_EXTRA_ARRIVALS = 2, TEAM_KNOB_WAIT_LIMIT_US = 3, TEAM_KNOB_EXPERT_KERNEL = 4 };
 int team_debug_knob(team_ctx *ctx, int knob, long long value);
 
 const char *team_strerror(int code);

@@ -23,7 +23,7 @@ TEAM_F_DCD, TEAM_F_LAC = 1, 2
 TEAM_DTYPE_F32, TEAM_DTYPE_BF16 = 0, 1
 
 EXPORTS = ["team_create", "team_destroy", "team_set_weights", "team_set_policy", "team_route",
-           "team_route_static", "team_pack_w_down", "team_select_experts", "team_moe_forward", "team_moe_forward_host", "team_residual_add", "team_read_status",
+           "team_route_static", "team_pack_w_down", "team_pack_w_tiles", "team_select_experts", "team_moe_forward", "team_moe_forward_host", "team_residual_add", "team_read_status",
            "team_last_launch_count", "team_expert_kernel_name", "team_expert_timing", "team_debug_force_simt", "team_debug_knob", "team_strerror",
            "team_last_cuda_error", "team_version"]
 
@@ -38,7 +38,7 @@ class team_config(ctypes.Structure):
 
 class team_weights(ctypes.Structure):
     _fields_ = [("w_router", ctypes.c_void_p), ("w_gate", ctypes.c_void_p), ("w_up", ctypes.c_void_p),
-                ("w_down", ctypes.c_void_p)]
+                ("w_down", ctypes.c_void_p), ("w_gu_tiles", ctypes.c_void_p), ("w_down_tiles", ctypes.c_void_p)]
 
 
 class team_step_state(ctypes.Structure):
@@ -69,6 +69,7 @@ def lib():
         L.team_set_policy.argtypes = [vp, ctypes.POINTER(team_config)]
         L.team_route.argtypes = [vp, vp, ctypes.POINTER(team_step_state), ctypes.POINTER(team_routing), vp]
         L.team_pack_w_down.argtypes = [vp, vp, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int, vp]
+        L.team_pack_w_tiles.argtypes = [vp, vp, vp, vp, vp, ctypes.c_int, ctypes.c_int, ctypes.c_int, vp]
         L.team_route_static.argtypes = [ctypes.POINTER(team_config), vp, vp, ctypes.POINTER(team_step_state),
                                         ctypes.POINTER(team_routing), vp]
         L.team_select_experts.argtypes = [vp, ctypes.POINTER(team_step_state), ctypes.POINTER(team_routing), vp]
@@ -136,9 +137,20 @@ def team_destroy(ctx):
     _check(lib().team_destroy(ctx))
 
 
-def team_set_weights(ctx, w_router, w_gate, w_up, w_down):
-    w = team_weights(_ptr(w_router), _ptr(w_gate), _ptr(w_up), _ptr(w_down))
+def team_set_weights(ctx, w_router, w_gate=None, w_up=None, w_down=None, w_gu_tiles=None, w_down_tiles=None):
+    """w_gate / w_up / w_down: the row-major / slab layout; w_gu_tiles / w_down_tiles: the tile-major layout."""
+    w = team_weights(_ptr(w_router), _ptr(w_gate), _ptr(w_up), _ptr(w_down), _ptr(w_gu_tiles), _ptr(w_down_tiles))
     _check(lib().team_set_weights(ctx, ctypes.byref(w)), ctx)
+
+
+def team_pack_w_tiles(w_gate, w_up, w_down):
+    """Row-major bf16 device tensors [n, I, H], [n, I, H], [n, H, I] -> (gu_tiles, down_tiles) in the tile-major layout."""
+    n, I, H = w_gate.shape
+    gu = torch.empty((2 * n * I * H,), dtype=torch.bfloat16, device=w_gate.device)
+    dt = torch.empty((n * I * H,), dtype=torch.bfloat16, device=w_gate.device)
+    _check(lib().team_pack_w_tiles(_ptr(w_gate.contiguous()), _ptr(w_up.contiguous()), _ptr(w_down.contiguous()), _ptr(gu),
+                                   _ptr(dt), n, H, I, _stream()))
+    return gu, dt
 
 
 def team_pack_w_down(w_down):
@@ -229,7 +241,7 @@ def team_expert_timing(ctx, enable):
     return ms.value, n.value
 
 
-TEAM_KNOB_NO_FUSE, TEAM_KNOB_EXTRA_ARRIVALS, TEAM_KNOB_WAIT_LIMIT_US = 1, 2, 3
+TEAM_KNOB_NO_FUSE, TEAM_KNOB_EXTRA_ARRIVALS, TEAM_KNOB_WAIT_LIMIT_US, TEAM_KNOB_EXPERT_KERNEL = 1, 2, 3, 4
 
 
 def team_debug_knob(ctx, knob, value):

@@ -7,11 +7,6 @@
 
 #include "team_common.cuh"
 
-namespace team {
-cudaError_t launch_experts_tc(int item_tile, const void* x, const void* w_gate, const void* w_up, const void* w_down,
-                              Workspace ws, float* y, Dims d, int grid, cudaStream_t s);
-}  // namespace team
-
 struct team_ctx {
   team_config cfg;
   team::Workspace ws;
@@ -24,7 +19,10 @@ struct team_ctx {
   int item_tile;
   int last_launches;
   int force_simt;
-  bool stream_path;   // few rows: the weight-streaming expert kernel instead of the tensor-memory one
+  bool stream_path;   // bf16: the weight-streaming expert kernel runs this context's calls (else the tensor-memory kernels)
+  bool can_stream, can_tile;   // what the shape allows
+  int prefer;         // diagnostic knob: 0 = choose by max_rows, 1 = streaming kernel, 2 = tensor-memory kernels
+  int stream_item_tile, tile_item_tile;
   bool fused_ok;      // at most 8 rows: the whole step can run as one kernel (router and selection in its prologue)
   int no_fuse;        // diagnostic knob: keep the three-kernel sequence
   int extra_arrivals; // diagnostic knob: arrivals the fused step's barrier waits for beyond the grid's own
@@ -37,6 +35,7 @@ struct team_ctx {
   // ... and the step (copy in, kernels, copy out) recorded once as a graph, replayed while nothing it bakes in changes
   cudaGraphExec_t hs_graph;
   int hs_graph_rows;
+  int hs_graph_launches;   // kernels in the recorded step
   bool hs_graph_off;     // recording failed once: plain launches from then on
   char cuda_err[256];
   // expert-kernel timing
@@ -130,7 +129,16 @@ cudaError_t timing_events(team_ctx* ctx, cudaEvent_t* e0, cudaEvent_t* e1) {
 
 bool use_tensor_path(const team_ctx* ctx) { return ctx->cfg.dtype == TEAM_DTYPE_BF16 && !ctx->force_simt; }
 
-int pick_item_tile(const team_config& c) { return team::experts_tc_item_tile(c.max_rows); }
+// Calls of fewer rows than this run the weight-streaming kernel when the shape allows both (measured crossover).
+constexpr int kTileMinRows = 64;
+
+void choose_expert_kernel(team_ctx* ctx) {
+  bool stream = ctx->can_stream && (!ctx->can_tile || ctx->cfg.max_rows < kTileMinRows);
+  if (ctx->prefer == 1 && ctx->can_stream) stream = true;
+  if (ctx->prefer == 2 && ctx->can_tile) stream = false;
+  ctx->stream_path = stream;
+  ctx->item_tile = stream ? ctx->stream_item_tile : ctx->tile_item_tile;
+}
 
 }  // namespace
 
@@ -174,6 +182,7 @@ int team_create(const team_config* cfg, team_ctx** out) {
   ctx->hs_pin = nullptr;
   ctx->hs_graph = nullptr;
   ctx->hs_graph_rows = 0;
+  ctx->hs_graph_launches = 0;
   ctx->hs_graph_off = false;
   ctx->cuda_err[0] = 0;
   ctx->timing = false;
@@ -188,19 +197,27 @@ int team_create(const team_config* cfg, team_ctx** out) {
     delete ctx;
     return TEAM_ERR_CUDA;
   }
-  ctx->item_tile = pick_item_tile(*cfg);
-  ctx->stream_path = cfg->dtype == TEAM_DTYPE_BF16 && team::experts_stream_supported(cfg->max_rows, cfg->hidden, cfg->inter);
-  // the few-rows kernel's gather mode takes work items of 8 or 16 token-slots
-  if (ctx->stream_path && team::experts_stream_gathers(cfg->max_rows)) ctx->item_tile = team::experts_stream_item_tile(cfg->max_rows);
+  const bool bf16 = cfg->dtype == TEAM_DTYPE_BF16;
+  ctx->can_stream = bf16 && team::experts_stream_supported(cfg->max_rows, cfg->hidden, cfg->inter);
+  ctx->can_tile = bf16 && team::experts_tile_supported(cfg->hidden, cfg->inter);
+  if (bf16 && !ctx->can_stream && !ctx->can_tile) {
+    delete ctx;
+    return TEAM_ERR_SHAPE;
+  }
+  ctx->prefer = 0;
+  // work items: the streaming kernel's gather mode takes 8 or 16 token-slots, the tensor-memory kernels up to 128
+  ctx->stream_item_tile = ctx->can_stream && team::experts_stream_gathers(cfg->max_rows) ? team::experts_stream_item_tile(cfg->max_rows) : 8;
+  ctx->tile_item_tile = team::experts_tile_chunk();
+  choose_expert_kernel(ctx);
   e = team::configure_router(cfg->dtype, cfg->hidden);
   if (e == cudaSuccess) e = team::configure_select(dims_of(*cfg, cfg->max_rows));
-  if (e == cudaSuccess && cfg->dtype == TEAM_DTYPE_BF16 && !ctx->stream_path) e = team::configure_experts_tc(ctx->item_tile);
-  if (e == cudaSuccess && ctx->stream_path) e = team::configure_experts_stream(cfg->hidden, cfg->max_rows);
+  if (e == cudaSuccess && ctx->can_tile) e = team::configure_experts_tile();
+  if (e == cudaSuccess && ctx->can_stream) e = team::configure_experts_stream(cfg->hidden, cfg->max_rows);
   if (e != cudaSuccess) {
     delete ctx;
     return TEAM_ERR_CUDA;
   }
-  ctx->fused_ok = ctx->stream_path && team::step_fused_supported(cfg->hidden, cfg->max_rows, cfg->n_experts, ctx->n_sms);
+  ctx->fused_ok = ctx->can_stream && team::step_fused_supported(cfg->hidden, cfg->max_rows, cfg->n_experts, ctx->n_sms);
 
   const size_t T = cfg->max_rows, E = cfg->n_experts, k = cfg->top_k, ns = cfg->n_shared, EN = E + ns;
   const size_t S = T * (k + ns);
@@ -215,13 +232,11 @@ int team_create(const team_config* cfg, team_ctx** out) {
   const size_t o_cnt = take(EN * 4), o_off = take((EN + 1) * 4), o_perm = take(S * 4), o_act_list = take(EN * 4);
   const size_t o_scal = take(64), o_items = take((EN + S / 8 + 2) * sizeof(team::WorkItem));
   const size_t o_act = take(cfg->dtype == TEAM_DTYPE_F32 ? S * cfg->inter * 4 : 256);
-  const bool bf16 = cfg->dtype == TEAM_DTYPE_BF16;
-  const size_t max_items = EN + S / ctx->item_tile + 2;
-  // the exchange scratch and its counters belong to the tensor-memory expert kernel only
-  const bool exchange = bf16 && !ctx->stream_path;
-  const size_t n_flags = exchange ? max_items * (cfg->inter / 64) : 0;
-  const size_t o_flags = take(n_flags * 4 + 4);
-  const size_t o_actg = take(exchange ? max_items * ctx->item_tile * cfg->inter * 2 : 256);
+  // the tensor-memory kernels' gathered token tiles, activation tiles and per-slot tables
+  const size_t tile_items = EN + S / ctx->tile_item_tile + 2;
+  const size_t tile_rows = ctx->can_tile ? team::experts_tile_rows(S, tile_items) : 0;
+  const size_t o_trow = take(tile_rows * 4 + 4), o_tw = take(tile_rows * 4 + 4);
+  const size_t o_tx = take(tile_rows * cfg->hidden * 2 + 256), o_tact = take(tile_rows * cfg->inter * 2 + 256);
   ctx->ws_bytes = off;
   e = cudaMalloc(&ctx->ws_base, ctx->ws_bytes);
   if (e != cudaSuccess) {
@@ -250,9 +265,10 @@ int team_create(const team_config* cfg, team_ctx** out) {
   ws.arrivals = reinterpret_cast<unsigned long long*>(scal + 8);
   ws.items = reinterpret_cast<team::WorkItem*>(b + o_items);
   ws.act = reinterpret_cast<float*>(b + o_act);
-  ws.win_flags = reinterpret_cast<int32_t*>(b + o_flags);
-  ws.n_flags = (int32_t)n_flags;
-  ws.act_g = reinterpret_cast<__nv_bfloat16*>(b + o_actg);
+  ws.tile_row = reinterpret_cast<int32_t*>(b + o_trow);
+  ws.tile_w = reinterpret_cast<float*>(b + o_tw);
+  ws.tile_x = reinterpret_cast<__nv_bfloat16*>(b + o_tx);
+  ws.tile_act = reinterpret_cast<__nv_bfloat16*>(b + o_tact);
   *out = ctx;
   return TEAM_OK;
 }
@@ -271,11 +287,17 @@ int team_destroy(team_ctx* ctx) {
 
 int team_set_weights(team_ctx* ctx, const team_weights* w) {
   if (ctx == nullptr || w == nullptr) return TEAM_ERR_ARG;
-  if (!w->w_router || !w->w_gate || !w->w_up || !w->w_down) return TEAM_ERR_ARG;
+  if (!w->w_router || ((uintptr_t)w->w_router & 15)) return TEAM_ERR_ARG;
+  // expert weights: the row-major / slab set, the tile-major set, or both; each set is all or nothing
+  const bool classic = w->w_gate || w->w_up || w->w_down, tiles = w->w_gu_tiles || w->w_down_tiles;
+  if (classic && !(w->w_gate && w->w_up && w->w_down)) return TEAM_ERR_ARG;
+  if (tiles && !(w->w_gu_tiles && w->w_down_tiles)) return TEAM_ERR_ARG;
+  if (!classic && !tiles) return TEAM_ERR_ARG;
   const uintptr_t align = ctx->cfg.dtype == TEAM_DTYPE_BF16 ? 127 : 15;
-  if (((uintptr_t)w->w_router & 15) || ((uintptr_t)w->w_gate & align) || ((uintptr_t)w->w_up & align) ||
-      ((uintptr_t)w->w_down & align))
+  if (classic && (((uintptr_t)w->w_gate & align) || ((uintptr_t)w->w_up & align) || ((uintptr_t)w->w_down & align)))
     return TEAM_ERR_ARG;
+  if (tiles && (((uintptr_t)w->w_gu_tiles & 127) || ((uintptr_t)w->w_down_tiles & 127))) return TEAM_ERR_ARG;
+  if (tiles && ctx->cfg.dtype != TEAM_DTYPE_BF16) return TEAM_ERR_ARG;
   ctx->w = *w;
   ctx->has_weights = true;
   drop_host_graph(ctx);
@@ -348,6 +370,10 @@ int team_moe_forward(team_ctx* ctx, const void* x, const team_step_state* st, te
   const team::Dims d = dims_of(ctx->cfg, st->n_rows);
   const bool tc = use_tensor_path(ctx);
   ctx->last_launches = 0;
+  // the weight layout the expert kernel of this context reads must have been given
+  if (tc && ctx->stream_path && !ctx->w.w_gate) return TEAM_ERR_ARG;
+  if (tc && !ctx->stream_path && !ctx->w.w_gu_tiles) return TEAM_ERR_ARG;
+  if (!tc && !ctx->w.w_gate) return TEAM_ERR_ARG;
   // The resident few-rows expert kernel reads the rows' choices directly; the dispatch tables are built only
   // when the caller asked for one of them.
   const bool wants_tables = out != nullptr && (out->expert_count || out->expert_offset || out->perm || out->active ||
@@ -384,9 +410,9 @@ int team_moe_forward(team_ctx* ctx, const void* x, const team_step_state* st, te
       e = team::launch_experts_stream(x, ctx->w.w_gate, ctx->w.w_up, ctx->w.w_down, ctx->ws, y, d, ctx->cfg.max_rows,
                                       ctx->n_sms, s);
     else
-      e = team::launch_experts_tc(ctx->item_tile, x, ctx->w.w_gate, ctx->w.w_up, ctx->w.w_down, ctx->ws, y, d, ctx->n_sms, s);
+      e = team::launch_experts_tile(x, ctx->w.w_gu_tiles, ctx->w.w_down_tiles, ctx->ws, y, d, ctx->n_sms, s);
     if (e != cudaSuccess) return fail_cuda(ctx, e, "expert kernel");
-    ++ctx->last_launches;
+    ctx->last_launches += ctx->stream_path ? 1 : 3;
   } else {
     e = team::launch_experts_simt(x, ctx->cfg.dtype, ctx->w.w_gate, ctx->w.w_up, ctx->w.w_down, ctx->ws, y, d, s);
     if (e != cudaSuccess) return fail_cuda(ctx, e, "expert kernels (fp32)");
@@ -471,6 +497,7 @@ int team_moe_forward_host(team_ctx* ctx, const void* x_host, const team_step_sta
     if (g) cudaGraphDestroy(g);
     if (good) {
       ctx->hs_graph_rows = (int)T;
+      ctx->hs_graph_launches = ctx->last_launches;
     } else {
       cudaGetLastError();
       ctx->hs_graph = nullptr;
@@ -481,7 +508,7 @@ int team_moe_forward_host(team_ctx* ctx, const void* x_host, const team_step_sta
   if (replay) {
     const cudaError_t e = cudaGraphLaunch(ctx->hs_graph, s);
     if (e != cudaSuccess) return fail_cuda(ctx, e, "graph launch");
-    ctx->last_launches = 2 + team::select_launches(dims_of(ctx->cfg, st_host->n_rows));
+    ctx->last_launches = ctx->hs_graph_launches;
   } else {
     rc = issue();
     if (rc != TEAM_OK) return rc;
@@ -518,7 +545,7 @@ int team_last_launch_count(const team_ctx* ctx) { return ctx ? ctx->last_launche
 const char* team_expert_kernel_name(const team_ctx* ctx) {
   if (ctx == nullptr) return "";
   if (!use_tensor_path(ctx)) return "k_gate_up + k_down";
-  if (!ctx->stream_path) return "k_experts_tc";
+  if (!ctx->stream_path) return "k_grouped_gemm (tcgen05: gate/up + SwiGLU, then down + combine)";
   const bool fused = ctx->fused_ok && !ctx->no_fuse && !team::experts_stream_gathers(ctx->cfg.max_rows);
   return fused ? "k_experts_stream (fused step: router, selection and experts in one launch)" : "k_experts_stream";
 }
@@ -527,6 +554,11 @@ int team_debug_knob(team_ctx* ctx, int knob, long long value) {
   if (ctx == nullptr) return TEAM_ERR_ARG;
   switch (knob) {
     case TEAM_KNOB_NO_FUSE: ctx->no_fuse = value != 0; break;
+    case TEAM_KNOB_EXPERT_KERNEL:
+      if (value < 0 || value > 2) return TEAM_ERR_ARG;
+      ctx->prefer = (int)value;
+      choose_expert_kernel(ctx);
+      break;
     case TEAM_KNOB_EXTRA_ARRIVALS:
       if (value < 0 || value > 1) return TEAM_ERR_ARG;
       ctx->extra_arrivals = (int)value;

@@ -70,9 +70,11 @@ struct Workspace {
   int32_t* n_items;     // [1]
   float* act;           // fp32 path: [max_rows*(k+ns), I] SwiGLU activations
   int32_t* status;      // [2] code, detail
-  __nv_bfloat16* act_g; // bf16 path: [items][item_tile][I] activations published between CTAs
-  int32_t* win_flags;   // bf16 path: [n_flags] groups published per 64-column window, zeroed per step
-  int32_t n_flags;
+  // tensor-memory expert kernels: gathered token tiles, SwiGLU activation tiles, per-slot (row, weight) tables
+  __nv_bfloat16* tile_x;    // [padded slot rows][H] as per-chunk [kb][rows][64] tiles
+  __nv_bfloat16* tile_act;  // [padded slot rows][I] likewise
+  int32_t* tile_row;        // [padded slot rows]
+  float* tile_w;            // [padded slot rows]
   unsigned long long* arrivals;   // fused step: CTA arrivals at the grid barrier, counted over all launches
 };
 
@@ -98,8 +100,14 @@ __device__ __forceinline__ void slot_row_weight(int slot, int T, int k, const fl
 cudaError_t configure_router(int dtype, int hidden);
 int router_smem_bytes(int hidden);   // dynamic shared memory the logits kernels are opted in to for this hidden size
 cudaError_t configure_select(Dims max_dims);
-cudaError_t configure_experts_tc(int item_tile);
-int experts_tc_item_tile(int max_rows);
+bool experts_tile_supported(int hidden, int inter);
+int experts_tile_chunk();
+size_t experts_tile_rows(size_t slots, size_t max_items);
+cudaError_t configure_experts_tile();
+cudaError_t launch_experts_tile(const void* x, const void* gu_tiles, const void* d_tiles, Workspace ws, float* y, Dims d,
+                                int grid, cudaStream_t s);
+cudaError_t launch_pack_w_tiles(const void* w_gate, const void* w_up, const void* w_down, void* gu, void* dt, int n_exp,
+                                int H, int I, cudaStream_t s);
 bool experts_stream_supported(int max_rows, int hidden, int inter);
 bool experts_stream_gathers(int max_rows);
 int experts_stream_item_tile(int max_rows);

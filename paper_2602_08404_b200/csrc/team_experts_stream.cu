@@ -274,8 +274,28 @@ __global__ void __launch_bounds__(kStThreads, 1) k_experts_stream(StArgs a) {
   }
   __syncthreads();
 
+  // ---- this warp's ring and its fixed lane roles (nothing here depends on the selection: set up ahead of it) ----
+  const uint32_t ring = st_smem_u32(st_smem + (size_t)TOK * H * 2 + RED_BYTES + (size_t)warp * SLOTS * kStChunkBytes);
+  // phase-1 chunk: 16 rows x 128 bytes; lane copies one 16-byte piece of rows cp_row + 4j; piece p of row r sits at p ^ (r & 7)
+  const int cp_row = lane >> 3, cp_piece = lane & 7;
+  const uint32_t cp_off0 = cp_row * 128 + ((cp_piece ^ cp_row) << 4);          // rows cp_row, cp_row + 8 (+1024)
+  const uint32_t cp_off1 = (cp_row + 4) * 128 + ((cp_piece ^ (cp_row + 4)) << 4);
+  // phase-2 chunk: 64 slab rows x 32 bytes, contiguous in memory; lane copies pieces lane + 32j; half p of row r sits at p ^ bit 2 of r
+  const uint32_t cq_off = (lane >> 1) * 32 + (((lane & 1) ^ ((lane >> 3) & 1)) << 4);
+  // ldmatrix lane roles: A tile row and k half (low / high 8), B token row and k piece
+  const int a_row = (lane & 7) + ((lane >> 3) & 1) * 8, a_hi = lane >> 4;
+  const uint32_t a1_base = a_row * 128;
+  const int a1_swz = a_row & 7;
+  const uint32_t a2_off = a_row * 32 + ((a_hi ^ ((a_row >> 2) & 1)) << 4);
+  const int b_tok = lane & 7, b_m = lane >> 3;
+  const uint32_t xs_lane = st_smem_u32(xs) + (uint32_t)b_tok * H * 2;
+  const int tile = warp & 1, ks = warp >> 1;     // phase 1: this warp's 16-row tile (gate | up) and hidden slice
+  const __nv_bfloat16* wmat = tile ? a.w_up : a.w_gate;
+  const uint64_t pol = st_stream_policy();
+
   // fused step: logits of the row this warp routes (warps 0 .. T-1), as order-preserving keys and as values
   uint32_t f_key[kMaxPerLane];
+  int f_slot[kMaxPerLane];
   float f_val[kMaxPerLane];
   float f_margin = __builtin_huge_valf();
   int f_mycls = TEAM_CLS_SKIP;
@@ -402,10 +422,12 @@ __global__ void __launch_bounds__(kStThreads, 1) k_experts_stream(StArgs a) {
           const int e = i * 32 + lane;
           f_val[i] = (i < ne && e < E) ? __ldcg(a.logits + (size_t)t * E + e) : kNegInf;      // written by other SMs: read from L2
           f_key[i] = float_key(f_val[i]);
+          f_slot[i] = i;
         }
         if (f_mycls == TEAM_CLS_FIRST) {
           const int gs = f_gslot[t];
-          const int n = warp_topk_picks(f_key, ne, k, lane,
+          sort_lane_keys(f_key, f_slot);
+          const int n = warp_topk_picks(f_key, f_slot, k, lane,
                                         [&](int j, int e, uint32_t key) {
                                           f_idx[t * k + j] = e;
                                           f_wt[t * k + j] = key_float(key);       // the logit; turned into the weight later
@@ -453,27 +475,18 @@ __global__ void __launch_bounds__(kStThreads, 1) k_experts_stream(StArgs a) {
     }
     n_act = __reduce_add_sync(0xffffffffu, __popc(act_word));
   }
-  const long long n_groups = (long long)(GATHER ? *a.n_items : n_act) * NG;
-  const int g_lo = (int)(n_groups * blockIdx.x / gridDim.x), g_hi = (int)(n_groups * (blockIdx.x + 1) / gridDim.x);
-
-  // ---- this warp's ring and its fixed lane roles ----
-  const uint32_t ring = st_smem_u32(st_smem + (size_t)TOK * H * 2 + RED_BYTES + (size_t)warp * SLOTS * kStChunkBytes);
-  // phase-1 chunk: 16 rows x 128 bytes; lane copies one 16-byte piece of rows cp_row + 4j; piece p of row r sits at p ^ (r & 7)
-  const int cp_row = lane >> 3, cp_piece = lane & 7;
-  const uint32_t cp_off0 = cp_row * 128 + ((cp_piece ^ cp_row) << 4);          // rows cp_row, cp_row + 8 (+1024)
-  const uint32_t cp_off1 = (cp_row + 4) * 128 + ((cp_piece ^ (cp_row + 4)) << 4);
-  // phase-2 chunk: 64 slab rows x 32 bytes, contiguous in memory; lane copies pieces lane + 32j; half p of row r sits at p ^ bit 2 of r
-  const uint32_t cq_off = (lane >> 1) * 32 + (((lane & 1) ^ ((lane >> 3) & 1)) << 4);
-  // ldmatrix lane roles: A tile row and k half (low / high 8), B token row and k piece
-  const int a_row = (lane & 7) + ((lane >> 3) & 1) * 8, a_hi = lane >> 4;
-  const uint32_t a1_base = a_row * 128;
-  const int a1_swz = a_row & 7;
-  const uint32_t a2_off = a_row * 32 + ((a_hi ^ ((a_row >> 2) & 1)) << 4);
-  const int b_tok = lane & 7, b_m = lane >> 3;
-  const uint32_t xs_lane = st_smem_u32(xs) + (uint32_t)b_tok * H * 2;
-  const int tile = warp & 1, ks = warp >> 1;     // phase 1: this warp's 16-row tile (gate | up) and hidden slice
-  const __nv_bfloat16* wmat = tile ? a.w_up : a.w_gate;
-  const uint64_t pol = st_stream_policy();
+  // at most (2048 * 20 + 260) items x 64 groups: the products below stay far inside 64 bits and, for the resident
+  // modes (at most 260 experts x 64 groups x a grid of a few hundred), inside 32
+  int g_lo, g_hi;
+  if (GATHER) {
+    const long long n_groups = (long long)(*a.n_items) * NG;
+    g_lo = (int)(n_groups * blockIdx.x / gridDim.x);
+    g_hi = (int)(n_groups * (blockIdx.x + 1) / gridDim.x);
+  } else {
+    const unsigned n_groups = (unsigned)(n_act * NG);
+    g_lo = (int)(n_groups * blockIdx.x / gridDim.x);
+    g_hi = (int)(n_groups * (blockIdx.x + 1u) / gridDim.x);
+  }
 
   // fused step: what the selection still owes once the activated set is known -- the second routing round (cold
   // rows inside E_A), the softmax denominators and routing weights, and CTA 0's exports.  Run once per CTA by
@@ -483,15 +496,16 @@ __global__ void __launch_bounds__(kStThreads, 1) k_experts_stream(StArgs a) {
   auto late_select = [&]() {
     if constexpr (FUSED) {
       if (warp < T) {
-        const int t = warp, k = d.k, E = d.E, ne = (E + 31) / 32;
+        const int t = warp, k = d.k, E = d.E;
         const bool exporter = blockIdx.x == 0;
         float row_max = 0.f, denom = 1.f, w = 0.f;
         if (f_mycls == TEAM_CLS_COLD) {
           const int gs = f_gslot[t];
 #pragma unroll
           for (int i = 0; i < kMaxPerLane; ++i)
-            if (!((f_mask[gs * 8 + i] >> lane) & 1u)) f_key[i] = 0x007fffffu;      // outside E_A: no candidate
-          const int n = warp_topk_picks(f_key, ne, k, lane,
+            if (!((f_mask[gs * 8 + i] >> lane) & 1u)) f_key[i] = kKeyNegInf;      // outside E_A: no candidate
+          sort_lane_keys(f_key, f_slot);
+          const int n = warp_topk_picks(f_key, f_slot, k, lane,
                                         [&](int j, int e, uint32_t key) {
                                           f_idx[t * k + j] = e;
                                           f_wt[t * k + j] = key_float(key);

@@ -41,3 +41,16 @@ extern "C" int team_pack_w_down(const void* src, void* dst, int n_experts_total,
       static_cast<const uint4*>(src), static_cast<uint4*>(dst), n_pieces, hidden, pieces_per_row, pieces_per_group);
   return cudaGetLastError() == cudaSuccess ? TEAM_OK : TEAM_ERR_CUDA;
 }
+
+extern "C" int team_pack_w_tiles(const void* w_gate, const void* w_up, const void* w_down, void* gu_tiles, void* down_tiles,
+                                 int n_experts_total, int hidden, int inter, void* stream) {
+  if (!w_gate || !w_up || !w_down || !gu_tiles || !down_tiles) return TEAM_ERR_ARG;
+  if (gu_tiles == w_gate || gu_tiles == w_up || down_tiles == w_down || gu_tiles == down_tiles) return TEAM_ERR_ARG;
+  if (((uintptr_t)w_gate & 15) || ((uintptr_t)w_up & 15) || ((uintptr_t)w_down & 15) || ((uintptr_t)gu_tiles & 127) ||
+      ((uintptr_t)down_tiles & 127))
+    return TEAM_ERR_ARG;
+  if (n_experts_total <= 0 || hidden <= 0 || inter <= 0 || hidden % 128 || inter % 64) return TEAM_ERR_SHAPE;
+  const cudaError_t e = team::launch_pack_w_tiles(w_gate, w_up, w_down, gu_tiles, down_tiles, n_experts_total, hidden, inter,
+                                                  static_cast<cudaStream_t>(stream));
+  return e == cudaSuccess ? TEAM_OK : TEAM_ERR_CUDA;
+}

@@ -117,9 +117,6 @@ k_select(const float* __restrict__ logits, StepPtrs st, Workspace ws, RoutePtrs 
   for (int i = tid; i < d.G * n_words32; i += kSelThreads) s.mask[i] = 0u;
   for (int i = tid; i < d.G; i += kSelThreads) s.has_first[i] = 0;
   for (int i = tid; i < nw * EN; i += kSelThreads) s.hist[i] = 0;
-  // per-window publication counters of the expert kernel start every step from zero
-  if (mode != kSelDispatch)
-    for (int i = cta * kSelThreads + tid; i < ws.n_flags; i += nb * kSelThreads) ws.win_flags[i] = 0;
   float conf_r[TEAM_MAX_ROWS / kSelThreads];     // confidences of the rows this thread classifies, fetched with the rest
 #pragma unroll
   for (int i = 0; i < TEAM_MAX_ROWS / kSelThreads; ++i) {

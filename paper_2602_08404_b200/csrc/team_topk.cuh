@@ -28,40 +28,49 @@ __device__ __forceinline__ float key_float(uint32_t k) {
   return __uint_as_float((k & 0x80000000u) ? (k & 0x7fffffffu) : ~k);
 }
 
-// Core of the selection.  key[i] is the key of expert i*32+lane (float_key(-inf) for a non-candidate); only the
-// first ne = ceil(E / 32) entries are looked at.  Picks the k largest keys in descending order, ties to the
+constexpr uint32_t kKeyNegInf = 0x007fffffu;            // float_key(-inf): "not a candidate"
+
+// Sorts a lane's eight (key, slot) pairs: key descending, equal keys by ascending slot (slot i stands for expert
+// i*32+lane, so this is "ties to the lower expert id" inside the lane).  A 19-comparator network, all indices
+// compile-time constants: everything stays in registers.
+__device__ __forceinline__ void sort_lane_keys(uint32_t (&key)[kMaxPerLane], int (&slot)[kMaxPerLane]) {
+  static_assert(kMaxPerLane == 8, "the network below sorts eight entries");
+#define TEAM_CE(i, j)                                                                        \
+  {                                                                                          \
+    const bool sw = key[j] > key[i] || (key[j] == key[i] && slot[j] < slot[i]);              \
+    const uint32_t ka = sw ? key[j] : key[i], kb = sw ? key[i] : key[j];                     \
+    const int sa = sw ? slot[j] : slot[i], sb = sw ? slot[i] : slot[j];                      \
+    key[i] = ka; key[j] = kb; slot[i] = sa; slot[j] = sb;                                    \
+  }
+  TEAM_CE(0, 1) TEAM_CE(2, 3) TEAM_CE(4, 5) TEAM_CE(6, 7)
+  TEAM_CE(0, 2) TEAM_CE(1, 3) TEAM_CE(4, 6) TEAM_CE(5, 7)
+  TEAM_CE(1, 2) TEAM_CE(5, 6) TEAM_CE(0, 4) TEAM_CE(3, 7)
+  TEAM_CE(1, 5) TEAM_CE(2, 6)
+  TEAM_CE(1, 4) TEAM_CE(3, 6)
+  TEAM_CE(2, 4) TEAM_CE(3, 5)
+  TEAM_CE(3, 4)
+#undef TEAM_CE
+}
+
+// Core of the selection.  key[] / slot[] are the lane's candidates as sort_lane_keys leaves them (non-candidates
+// carry kKeyNegInf and sort to the end).  Picks the k largest keys of the warp in descending order, ties to the
 // lower expert id, and calls on_pick(j, expert, key) for the j-th pick ON THE LANE THAT HOLDS IT (nothing is
-// broadcast).  Picked keys are retired in place.  Returns the number of picks made (< k only if fewer than k
+// broadcast).  Picked entries are shifted out.  Returns the number of picks made (< k only if fewer than k
 // candidates exist); margin_out (all lanes) = logit of the last pick minus the best logit left (+inf if none).
 //
-// One pick is a short dependent chain: warp-wide maximum of the lanes' current best keys (one redux), a ballot
-// of who holds it, and only the holder updates its state; two or more holders (equal logits in different
-// lanes) take a second redux for the lowest expert id.
+// One pick is a short dependent chain: the warp-wide maximum of the lanes' heads (one redux), a ballot of who
+// holds it, and the holder shifts its list by one; two or more holders (equal logits in different lanes) take a
+// second redux for the lowest expert id.
 template <typename OnPick>
-__device__ __forceinline__ int warp_topk_picks(uint32_t (&key)[kMaxPerLane], int ne, int k, int lane, OnPick&& on_pick,
-                                               float& margin_out) {
-  const uint32_t key_neg_inf = 0x007fffffu;            // float_key(-inf)
-  uint32_t bk = key_neg_inf;
-  int bi = 0;
-  auto local_best = [&]() {
-    bk = key_neg_inf;
-    bi = 0;
-#pragma unroll
-    for (int i = 0; i < kMaxPerLane; ++i) {
-      // ascending expert id within the lane, strict '>' keeps the lower id on ties
-      if (i < ne && key[i] > bk) {
-        bk = key[i];
-        bi = i;
-      }
-    }
-  };
-  local_best();
+__device__ __forceinline__ int warp_topk_picks(uint32_t (&key)[kMaxPerLane], int (&slot)[kMaxPerLane], int k, int lane,
+                                               OnPick&& on_pick, float& margin_out) {
   float last = kNegInf;
   margin_out = __builtin_huge_valf();
   int n = 0;
   for (int j = 0; j <= k; ++j) {
+    const uint32_t bk = key[0];
     const uint32_t wk = __reduce_max_sync(0xffffffffu, bk);
-    if (wk == key_neg_inf) break;                       // no candidate left
+    if (wk == kKeyNegInf) break;                        // no candidate left
     if (j == k) {
       margin_out = last - key_float(wk);
       break;
@@ -69,15 +78,17 @@ __device__ __forceinline__ int warp_topk_picks(uint32_t (&key)[kMaxPerLane], int
     const uint32_t holders = __ballot_sync(0xffffffffu, bk == wk);
     int win_lane = __ffs(holders) - 1;
     if (holders & (holders - 1u)) {
-      const uint32_t wi = __reduce_min_sync(0xffffffffu, bk == wk ? (uint32_t)(bi * 32 + lane) : 0x7fffffffu);
+      const uint32_t wi = __reduce_min_sync(0xffffffffu, bk == wk ? (uint32_t)(slot[0] * 32 + lane) : 0x7fffffffu);
       win_lane = (int)(wi & 31u);
     }
     if (lane == win_lane) {
-      on_pick(j, bi * 32 + lane, wk);
+      on_pick(j, slot[0] * 32 + lane, wk);
 #pragma unroll
-      for (int i = 0; i < kMaxPerLane; ++i)
-        if (i == bi) key[i] = key_neg_inf;
-      local_best();
+      for (int i = 0; i + 1 < kMaxPerLane; ++i) {
+        key[i] = key[i + 1];
+        slot[i] = slot[i + 1];
+      }
+      key[kMaxPerLane - 1] = kKeyNegInf;
     }
     last = key_float(wk);
     n = j + 1;
@@ -94,14 +105,19 @@ __device__ __forceinline__ TopkResult warp_topk(const float (&v)[kMaxPerLane], i
   r.val = kNegInf;
   r.top = kNegInf;
   uint32_t key[kMaxPerLane];
+  int slot[kMaxPerLane];
 #pragma unroll
-  for (int i = 0; i < kMaxPerLane; ++i) key[i] = i < ne ? float_key(v[i]) : 0x007fffffu;
+  for (int i = 0; i < kMaxPerLane; ++i) {
+    key[i] = i < ne ? float_key(v[i]) : kKeyNegInf;
+    slot[i] = i;
+  }
+  sort_lane_keys(key, slot);
   // the holder of a pick remembers it; afterwards pick j moves to lane j (one shuffle per pick, off the picks'
   // dependent chain)
   int order[kMaxPerLane];             // this lane's key i was picked as pick number order[i] (-1: not picked)
 #pragma unroll
   for (int i = 0; i < kMaxPerLane; ++i) order[i] = -1;
-  const int n = warp_topk_picks(key, ne, k, lane,
+  const int n = warp_topk_picks(key, slot, k, lane,
                                 [&](int j, int e, uint32_t) {
 #pragma unroll
                                   for (int i = 0; i < kMaxPerLane; ++i)

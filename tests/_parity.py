@@ -34,8 +34,11 @@ class Layer:
         self.shape, self.cfg = shape, lib_config(shape, flags, **kw)
         self.ctx = B.team_create(self.cfg)
         dc = dtype_code(shape)
+        w_down = B.to_device(weights["w_down"], dc)
         self.w = [torch.as_tensor(weights["w_router"]).cuda().contiguous(), B.to_device(weights["w_gate"], dc),
-                  B.to_device(weights["w_up"], dc), B.team_pack_w_down(B.to_device(weights["w_down"], dc))]
+                  B.to_device(weights["w_up"], dc), B.team_pack_w_down(w_down)]
+        if shape.dtype == "bf16":        # both layouts: whichever expert kernel the context picks finds its own
+            self.w += list(B.team_pack_w_tiles(self.w[1], self.w[2], w_down))
         B.team_set_weights(self.ctx, *self.w)
 
     def close(self):

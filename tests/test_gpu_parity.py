@@ -48,9 +48,9 @@ def test_c1_tiny_fp32_all_steps(flags, weights_cache):
 @pytest.mark.parametrize("shape", [W.MINI_BF16, W.MINI_SHARED, W.MINI_WRAP], ids=lambda s: s.name)
 def test_mini_bf16_tensor_path(shape, flags, weights_cache):
     stats = P.run_schedule(shape, weights_cache(shape), W.make_schedule(shape), flags)
-    # router, selection, experts; the selection is two launches (rounds per group, then dispatch) for several
-    # groups with more than 32 rows
-    assert all(s["launches"] == (4 if shape.seqs > 1 and shape.rows > 32 else 3) for s in stats)
+    # router, selection, then gather + the two grouped GEMMs; the selection is two launches (rounds per group, then
+    # dispatch) for several groups with more than 32 rows
+    assert all(s["launches"] == (6 if shape.seqs > 1 and shape.rows > 32 else 5) for s in stats)
 
 
 @pytest.mark.parametrize("shape", [W.MINI_BF16, W.MINI_SHARED], ids=lambda s: s.name)
@@ -93,7 +93,8 @@ def test_few_rows_kernel_gather_mode_with_split_items(flags, weights_cache):
 @pytest.mark.parametrize("flags", [0, 3])
 def test_few_rows_kernel_gather_mode_items_of_16_slots(flags, weights_cache):
     shape = W.STREAM_GATHER16                    # 80 rows in 2 groups: items of 16 slots, the shared expert has five
-    stats = P.run_schedule(shape, weights_cache(shape), W.make_schedule(shape), flags)
+    stats = P.run_schedule(shape, weights_cache(shape), W.make_schedule(shape), flags,
+                           knobs=[(B.TEAM_KNOB_EXPERT_KERNEL, 1)])      # (64 rows and more default to the tensor-memory kernels)
     # 40 rows per group are more than a CTA routes at once: the selection is one launch of a 2-CTA cluster
     assert len(stats) == 4 and all(s["launches"] == 3 for s in stats)
 
@@ -104,21 +105,68 @@ def test_c3_llada_shape_with_shared_expert(flags, weights_cache):
     assert len(stats) == 8
 
 
-def test_paper_operating_point_block32_four_branches_one_group(weights_cache):
-    shape = W.paper_point()                      # 128 rows, one group: single-CTA selection, gathered expert items
+KERNELS = {"default": [], "streaming": [(B.TEAM_KNOB_EXPERT_KERNEL, 1)], "tensor_memory": [(B.TEAM_KNOB_EXPERT_KERNEL, 2)]}
+
+
+@pytest.mark.parametrize("kernel", ["streaming", "tensor_memory"])
+def test_paper_operating_point_block32_four_branches_one_group(weights_cache, kernel):
+    shape = W.paper_point()                      # 128 rows, one group: cluster selection, one expert sees up to 108 slots
     steps = W.make_schedule(shape)[1:4]
-    P.run_schedule(shape, weights_cache(shape), steps, 3)
+    P.run_schedule(shape, weights_cache(shape), steps, 3, knobs=KERNELS[kernel])
 
 
+@pytest.mark.parametrize("kernel", ["streaming", "tensor_memory"])
 @pytest.mark.parametrize("seqs", [1, 4, 16, 64])
-def test_c4_batch_sweep(seqs, weights_cache):
+def test_c4_batch_sweep(seqs, weights_cache, kernel):
     shape = W.c4(seqs)
     steps = W.make_schedule(shape)
     # all four steps for the small batches, two for the large ones (the oracle takes seconds per step there)
     steps = steps if seqs <= 4 else steps[1:3]
-    P.run_schedule(shape, weights_cache(shape), steps, 3)
+    stats = P.run_schedule(shape, weights_cache(shape), steps, 3, knobs=KERNELS[kernel])
+    assert all(s["launches"] >= (5 if kernel == "tensor_memory" else 3) for s in stats)
     if seqs <= 4:
-        P.run_schedule(shape, weights_cache(shape), steps, 0)
+        P.run_schedule(shape, weights_cache(shape), steps, 0, knobs=KERNELS[kernel])
+
+
+@pytest.mark.parametrize("flags", [0, 3])
+def test_c3_llada_shape_on_the_tensor_memory_kernels(flags, weights_cache):
+    stats = P.run_schedule(W.C3, weights_cache(W.C3), W.make_schedule(W.C3)[:4], flags, knobs=KERNELS["tensor_memory"])
+    assert all(s["launches"] == 5 for s in stats)
+
+
+def test_tensor_memory_kernels_with_more_slots_than_a_chunk_holds(weights_cache):
+    """An expert chosen by more than 128 token-slots is split into several chunks (its weights are then streamed
+    once per chunk): 160 rows with a shared expert that every row uses."""
+    import dataclasses
+    shape = dataclasses.replace(W.STREAM_GATHER16, name="tile_split_chunks", block=40, seqs=4, seed=21)
+    steps = W.make_schedule(shape)[:2]
+    P.run_schedule(shape, weights_cache(shape), steps, 0, knobs=KERNELS["tensor_memory"])
+
+
+def test_pack_w_tiles_is_the_stated_permutation():
+    n, H, I = 2, 256, 128
+    gen = torch.Generator().manual_seed(6)
+    wg, wu = [torch.randn((n, I, H), generator=gen).to(torch.bfloat16) for _ in range(2)]
+    wd = torch.randn((n, H, I), generator=gen).to(torch.bfloat16)
+    gu, dt = B.team_pack_w_tiles(wg.cuda(), wu.cuda(), wd.cuda())
+    torch.cuda.synchronize()
+    gu = gu.cpu().view(torch.int16).numpy().reshape(n, I // 64, H // 64, 128, 8, 8)
+    dt = dt.cpu().view(torch.int16).numpy().reshape(n, H // 128, I // 64, 128, 8, 8)
+    g16, u16, d16 = (t.view(torch.int16).numpy() for t in (wg, wu, wd))
+    for e in range(n):
+        for u in range(I // 64):
+            for kb in range(H // 64):
+                for r in range(128):
+                    blk, m, i = r // 32, (r // 16) % 2, r % 16
+                    src = (u16 if m else g16)[e, u * 64 + blk * 16 + i, kb * 64:(kb + 1) * 64].reshape(8, 8)
+                    for p in range(8):
+                        np.testing.assert_array_equal(gu[e, u, kb, r, p ^ (r & 7)], src[p])
+        for ht in range(H // 128):
+            for kb in range(I // 64):
+                for r in range(128):
+                    src = d16[e, ht * 128 + r, kb * 64:(kb + 1) * 64].reshape(8, 8)
+                    for p in range(8):
+                        np.testing.assert_array_equal(dt[e, ht, kb, r, p ^ (r & 7)], src[p])
 
 
 def _run_stack(shape, n_layers, flags, weights_cache, tables=True):
