@@ -236,7 +236,7 @@ def run_layer(args):
 
     # R independent layers, generated on the device (seeded); layer 0 also goes to the host for the oracle leg
     layers, packed, tiles = [], [], []
-    want_tiles = args.expert_kernel == "tile" or (args.expert_kernel == "auto" and T >= 64)
+    want_tiles = args.expert_kernel == "tile" or (args.expert_kernel == "auto" and T >= 96)
     want_classic = not want_tiles or args.expert_kernel == "stream"
     for r in range(R):
         wr, wg, wu, wd = W.device_layer_weights(shape, 1000 + r, dev)

@@ -88,7 +88,7 @@ typedef struct {
   int32_t inter;       /* I; multiple of 64 for bf16, of 16 for fp32                     */
   int32_t n_shared;    /* always-on experts appended after the routed ones              */
   int32_t max_rows;    /* largest n_rows of any call on this context; it also picks the
-                          expert kernel (bf16).  Hidden size 1024 or 2048 and fewer than 64
+                          expert kernel (bf16).  Hidden size 1024 or 2048 and fewer than 96
                           rows: the weight-streaming kernel on the row-major / slab layout
                           (<= 8 rows all resident, else work items of 8 token-slots).
                           Otherwise: the tensor-memory (tcgen05) grouped GEMMs on the
@@ -103,6 +103,9 @@ typedef struct {
   int32_t hot_dist_inclusive; /* 1: |k-j| <= L_hot (Sec. 5.1 wording), 0: < (Eq. 4 as printed) */
   int32_t prefix_decoded;     /* 1: position -1 (previous block) counts as decoded      */
   int32_t norm_topk;          /* 1: routing weights renormalised over the k chosen      */
+  int32_t refresh_every;      /* Sec. 4.1 / Table 3 (Refresh-4, Refresh-8): N > 0 recomputes every token on the
+                                 steps with step_index % N == 0 (cached tokens are treated as newly accepted
+                                 there); 0 = never, the paper's refresh-free choice                        */
 } team_config;
 
 typedef struct {
@@ -125,6 +128,7 @@ typedef struct {
   const int32_t *pos;       /* [T] position in the block                                  */
   const int32_t *group;     /* [T] scope of E_A                                           */
   const int32_t *branch;    /* [T] speculative branch id (scope of "decoded" in Eq. 4)    */
+  int32_t step_index;       /* denoising step inside the block, 0-based (read only when refresh_every > 0) */
 } team_step_state;
 
 /* Optional outputs; any pointer may be NULL.  team_route fills probs, topk_idx,
@@ -190,7 +194,7 @@ int team_pack_w_tiles(const void *w_gate, const void *w_up, const void *w_down, 
                       int n_experts_total, int hidden, int inter, void *stream);
 
 /* Change flags / tau_hot / L_hot / hot_dist_inclusive / prefix_decoded /
- * norm_topk of an existing context (shapes and dtype must be unchanged). */
+ * norm_topk / refresh_every of an existing context (shapes and dtype must be unchanged). */
 int team_set_policy(team_ctx *ctx, const team_config *cfg);
 
 /* Router (Algorithm 1 "Router", Sec. 4.1 row selection): logits = x W_r^T in

@@ -47,6 +47,9 @@ stated where it is applied):
   * With DCD off, every decoded row (new or old) is computed and is a
     first-round row.
   * Shared experts (if any) are applied to every computed row with weight 1.
+  * Periodic refresh (Sec. 4.1, second paragraph; Table 3, Refresh-4 / Refresh-8): with refresh_every = N > 0
+    every N-th denoising step of a block (step_index 0, N, 2N, ...) recomputes all tokens -- on such a step a
+    cached token is treated like a newly accepted one.  N = 0 is the paper's own choice, refresh-free.
 
 Parity pins live in tests/test_oracle_*.py; every function below is pinned by
 at least one of them.
@@ -75,6 +78,7 @@ class Config:
     prefix_decoded: int = 1
     norm_topk: int = 1
     max_groups: int = 1
+    refresh_every: int = 0
 
 
 # ----------------------------------------------------------------------------
@@ -86,6 +90,21 @@ def active_rows(tok_state, flags):
     if flags & F_DCD:
         return np.flatnonzero(tok_state != TOK_CACHED)
     return np.arange(tok_state.shape[0])
+
+
+# ----------------------------------------------------------------------------
+# Sec. 4.1, second paragraph / Table 3 -- periodic refresh: every N-th step all
+# tokens are recomputed, i.e. cached tokens count as newly accepted on that step.
+# ----------------------------------------------------------------------------
+def is_refresh_step(cfg, step_index):
+    return cfg.refresh_every > 0 and step_index % cfg.refresh_every == 0
+
+
+def refreshed_states(cfg, tok_state, step_index):
+    tok_state = np.array(tok_state, dtype=np.uint8)
+    if is_refresh_step(cfg, step_index):
+        tok_state[tok_state == TOK_CACHED] = TOK_NEW
+    return tok_state
 
 
 # ----------------------------------------------------------------------------
@@ -249,7 +268,8 @@ def expert_ffn(x_rows, w_gate_e, w_up_e, w_down_e):
 # recomputed (cached tokens keep the output of the step that last computed them).
 # weights: dict with w_router [E,H], w_gate/w_up [E+ns,I,H], w_down [E+ns,H,I].
 # ----------------------------------------------------------------------------
-def moe_forward(cfg, weights, x, tok_state, conf, pos, group, branch, y_prev=None):
+def moe_forward(cfg, weights, x, tok_state, conf, pos, group, branch, y_prev=None, step_index=0):
+    tok_state = refreshed_states(cfg, tok_state, step_index)
     T = len(tok_state)
     logits32, probs = router(x, weights["w_router"])
     r = select_experts(cfg, logits32, probs, tok_state, conf, pos, group, branch)

@@ -33,7 +33,7 @@ class team_config(ctypes.Structure):
                 ("inter", ctypes.c_int32), ("n_shared", ctypes.c_int32), ("max_rows", ctypes.c_int32),
                 ("max_groups", ctypes.c_int32), ("dtype", ctypes.c_int32), ("flags", ctypes.c_int32),
                 ("tau_hot", ctypes.c_float), ("L_hot", ctypes.c_int32), ("hot_dist_inclusive", ctypes.c_int32),
-                ("prefix_decoded", ctypes.c_int32), ("norm_topk", ctypes.c_int32)]
+                ("prefix_decoded", ctypes.c_int32), ("norm_topk", ctypes.c_int32), ("refresh_every", ctypes.c_int32)]
 
 
 class team_weights(ctypes.Structure):
@@ -43,7 +43,8 @@ class team_weights(ctypes.Structure):
 
 class team_step_state(ctypes.Structure):
     _fields_ = [("n_rows", ctypes.c_int32), ("tok_state", ctypes.c_void_p), ("conf", ctypes.c_void_p),
-                ("pos", ctypes.c_void_p), ("group", ctypes.c_void_p), ("branch", ctypes.c_void_p)]
+                ("pos", ctypes.c_void_p), ("group", ctypes.c_void_p), ("branch", ctypes.c_void_p),
+                ("step_index", ctypes.c_int32)]
 
 
 class team_routing(ctypes.Structure):
@@ -119,9 +120,9 @@ def _stream():
 
 
 def make_config(hidden, n_experts, top_k, inter, n_shared=0, max_rows=64, max_groups=1, dtype=TEAM_DTYPE_BF16,
-                flags=0, tau_hot=0.7, L_hot=3, hot_dist_inclusive=1, prefix_decoded=1, norm_topk=1):
+                flags=0, tau_hot=0.7, L_hot=3, hot_dist_inclusive=1, prefix_decoded=1, norm_topk=1, refresh_every=0):
     return team_config(hidden, n_experts, top_k, inter, n_shared, max_rows, max_groups, dtype, flags, tau_hot,
-                       L_hot, hot_dist_inclusive, prefix_decoded, norm_topk)
+                       L_hot, hot_dist_inclusive, prefix_decoded, norm_topk, refresh_every)
 
 
 # ---- the C entry points, same names, torch tensors for device memory ---------------------------------
@@ -169,7 +170,7 @@ def team_set_policy(ctx, cfg):
 
 def _state(st):
     return team_step_state(int(st["tok_state"].shape[0]), _ptr(st["tok_state"]), _ptr(st["conf"]), _ptr(st["pos"]),
-                           _ptr(st["group"]), _ptr(st["branch"]))
+                           _ptr(st["group"]), _ptr(st["branch"]), int(st.get("step_index", 0)))
 
 
 def _routing(out):
@@ -211,7 +212,8 @@ def _hptr(t):
 def team_moe_forward_host(ctx, x_host, st_host, out, y_host):
     """x_host, the step state and y_host are CPU tensors; `out` (optional) holds device tensors. Blocks until y_host is filled."""
     st = team_step_state(int(st_host["tok_state"].shape[0]), _hptr(st_host["tok_state"]), _hptr(st_host["conf"]),
-                         _hptr(st_host["pos"]), _hptr(st_host["group"]), _hptr(st_host["branch"]))
+                         _hptr(st_host["pos"]), _hptr(st_host["group"]), _hptr(st_host["branch"]),
+                         int(st_host.get("step_index", 0)))
     r = _routing(out)
     _check(lib().team_moe_forward_host(ctx, _hptr(x_host), ctypes.byref(st), ctypes.byref(r) if r is not None else None,
                                        _hptr(y_host), _stream()), ctx)

@@ -36,6 +36,7 @@ struct team_ctx {
   cudaGraphExec_t hs_graph;
   int hs_graph_rows;
   int hs_graph_launches;   // kernels in the recorded step
+  int hs_graph_flags;      // flags of the recorded step (a refresh step runs with other flags)
   bool hs_graph_off;     // recording failed once: plain launches from then on
   char cuda_err[256];
   // expert-kernel timing
@@ -57,9 +58,16 @@ team::Dims dims_of(const team_config& c, int T) {
   return d;
 }
 
-team::Policy policy_of(const team_config& c) {
+// Sec. 4.1 / Table 3: on a refresh step every token is recomputed -- cached tokens count as newly accepted, which
+// is what the kernels do when delayed caching is off for that call.
+int step_flags(const team_config& c, const team_step_state* st) {
+  const bool refresh = c.refresh_every > 0 && st != nullptr && st->step_index % c.refresh_every == 0;
+  return refresh ? (c.flags & ~TEAM_F_DCD) : c.flags;
+}
+
+team::Policy policy_of(const team_config& c, const team_step_state* st) {
   team::Policy p;
-  p.flags = c.flags; p.tau_hot = c.tau_hot; p.L_hot = c.L_hot; p.inclusive = c.hot_dist_inclusive;
+  p.flags = step_flags(c, st); p.tau_hot = c.tau_hot; p.L_hot = c.L_hot; p.inclusive = c.hot_dist_inclusive;
   p.prefix_decoded = c.prefix_decoded; p.norm_topk = c.norm_topk;
   return p;
 }
@@ -78,7 +86,7 @@ int check_config(const team_config* c) {
   } else {
     return TEAM_ERR_SHAPE;
   }
-  if (c->L_hot < 0) return TEAM_ERR_ARG;
+  if (c->L_hot < 0 || c->refresh_every < 0) return TEAM_ERR_ARG;
   return TEAM_OK;
 }
 
@@ -130,7 +138,7 @@ cudaError_t timing_events(team_ctx* ctx, cudaEvent_t* e0, cudaEvent_t* e1) {
 bool use_tensor_path(const team_ctx* ctx) { return ctx->cfg.dtype == TEAM_DTYPE_BF16 && !ctx->force_simt; }
 
 // Calls of fewer rows than this run the weight-streaming kernel when the shape allows both (measured crossover).
-constexpr int kTileMinRows = 64;
+constexpr int kTileMinRows = 96;
 
 void choose_expert_kernel(team_ctx* ctx) {
   bool stream = ctx->can_stream && (!ctx->can_tile || ctx->cfg.max_rows < kTileMinRows);
@@ -311,7 +319,7 @@ int team_set_policy(team_ctx* ctx, const team_config* cfg) {
       cfg->n_shared != c.n_shared || cfg->max_rows != c.max_rows || cfg->max_groups != c.max_groups ||
       cfg->dtype != c.dtype)
     return TEAM_ERR_SHAPE;
-  if (cfg->L_hot < 0) return TEAM_ERR_ARG;
+  if (cfg->L_hot < 0 || cfg->refresh_every < 0) return TEAM_ERR_ARG;
   ctx->cfg = *cfg;
   drop_host_graph(ctx);
   return TEAM_OK;
@@ -338,10 +346,10 @@ int team_route(team_ctx* ctx, const void* x, const team_step_state* st, team_rou
   const team::Dims d = dims_of(ctx->cfg, st->n_rows);
   ctx->last_launches = 0;
   cudaError_t e = team::launch_router_logits(x, ctx->cfg.dtype, static_cast<const float*>(ctx->w.w_router),
-                                             st->tok_state, ctx->ws.logits, nullptr, d, ctx->cfg.flags, s);
+                                             st->tok_state, ctx->ws.logits, nullptr, d, step_flags(ctx->cfg, st), s);
   if (e != cudaSuccess) return fail_cuda(ctx, e, "router logits");
   ++ctx->last_launches;
-  e = team::launch_router_topk(ctx->ws.logits, st->tok_state, export_ptrs(out), d, policy_of(ctx->cfg), s);
+  e = team::launch_router_topk(ctx->ws.logits, st->tok_state, export_ptrs(out), d, policy_of(ctx->cfg, st), s);
   if (e != cudaSuccess) return fail_cuda(ctx, e, "router top-k");
   ++ctx->last_launches;
   return TEAM_OK;
@@ -354,7 +362,7 @@ int team_select_experts(team_ctx* ctx, const team_step_state* st, team_routing* 
   const team::Dims d = dims_of(ctx->cfg, st->n_rows);
   ctx->last_launches = 0;
   cudaError_t e = team::launch_select(ctx->ws.logits, step_ptrs(st), ctx->ws, export_ptrs(out), d,
-                                      policy_of(ctx->cfg), ctx->item_tile, true, s);
+                                      policy_of(ctx->cfg, st), ctx->item_tile, true, s);
   if (e != cudaSuccess) return fail_cuda(ctx, e, "select");
   ctx->last_launches += team::select_launches(d);
   return TEAM_OK;
@@ -386,7 +394,7 @@ int team_moe_forward(team_ctx* ctx, const void* x, const team_step_state* st, te
     if (ctx->timing && (e = timing_events(ctx, &ev0, &ev1)) != cudaSuccess) return fail_cuda(ctx, e, "event create");
     if (ev0) cudaEventRecord(ev0, s);
     e = team::launch_step_fused(x, static_cast<const float*>(ctx->w.w_router), ctx->w.w_gate, ctx->w.w_up, ctx->w.w_down,
-                                step_ptrs(st), ctx->ws, export_ptrs(out), y, d, policy_of(ctx->cfg), ctx->n_sms,
+                                step_ptrs(st), ctx->ws, export_ptrs(out), y, d, policy_of(ctx->cfg, st), ctx->n_sms,
                                 ctx->spin_cycles, ctx->extra_arrivals, s);
     if (e != cudaSuccess) return fail_cuda(ctx, e, "fused step");
     if (ev1) cudaEventRecord(ev1, s);
@@ -394,10 +402,10 @@ int team_moe_forward(team_ctx* ctx, const void* x, const team_step_state* st, te
     return TEAM_OK;
   }
   e = team::launch_router_logits(x, ctx->cfg.dtype, static_cast<const float*>(ctx->w.w_router), st->tok_state,
-                                 ctx->ws.logits, tc ? y : nullptr, d, ctx->cfg.flags, s);
+                                 ctx->ws.logits, tc ? y : nullptr, d, step_flags(ctx->cfg, st), s);
   if (e != cudaSuccess) return fail_cuda(ctx, e, "router logits");
   ++ctx->last_launches;
-  e = team::launch_select(ctx->ws.logits, step_ptrs(st), ctx->ws, export_ptrs(out), d, policy_of(ctx->cfg),
+  e = team::launch_select(ctx->ws.logits, step_ptrs(st), ctx->ws, export_ptrs(out), d, policy_of(ctx->cfg, st),
                           ctx->item_tile, wants_tables || !resident, s);
   if (e != cudaSuccess) return fail_cuda(ctx, e, "select");
   ctx->last_launches += team::select_launches(d);
@@ -484,7 +492,7 @@ int team_moe_forward_host(team_ctx* ctx, const void* x_host, const team_step_sta
       replay = false;
     }
   }
-  if (replay && (ctx->hs_graph == nullptr || ctx->hs_graph_rows != (int)T)) {
+  if (replay && (ctx->hs_graph == nullptr || ctx->hs_graph_rows != (int)T || ctx->hs_graph_flags != step_flags(ctx->cfg, st_host))) {
     drop_host_graph(ctx);
     cudaGraph_t g = nullptr;
     bool good = cudaStreamBeginCapture(s, cudaStreamCaptureModeThreadLocal) == cudaSuccess;
@@ -498,6 +506,7 @@ int team_moe_forward_host(team_ctx* ctx, const void* x_host, const team_step_sta
     if (good) {
       ctx->hs_graph_rows = (int)T;
       ctx->hs_graph_launches = ctx->last_launches;
+      ctx->hs_graph_flags = step_flags(ctx->cfg, st_host);
     } else {
       cudaGetLastError();
       ctx->hs_graph = nullptr;

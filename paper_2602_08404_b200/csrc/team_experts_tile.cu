@@ -113,11 +113,13 @@ __global__ void __launch_bounds__(256) k_gather_tiles(GatherArgs a) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int H = a.d.H, n_items = *a.n_items;
   const int pieces = H / 8;                                      // 16-byte pieces per row
-  for (int c = blockIdx.x; c < n_items; c += gridDim.x) {
+  // four CTAs share a chunk: CTA slice s takes the rows n with (n / 8) % 4 == s, its warp w those with n % 8 == w
+  const int slice = blockIdx.x & 3;
+  for (int c = blockIdx.x >> 2; c < n_items; c += gridDim.x >> 2) {
     const WorkItem it = a.items[c];
     const int np = pad16(it.n), r0 = chunk_row0(it, c);
     __nv_bfloat16* base = a.xg + (size_t)r0 * H;
-    for (int n = warp; n < np; n += 8) {
+    for (int n = slice * 8 + warp; n < np; n += 32) {
       int row = -1;
       float wt = 0.f;
       if (n < it.n) slot_row_weight(a.perm[it.begin + n], a.d.T, a.d.k, a.topk_w, row, wt);
@@ -380,7 +382,7 @@ cudaError_t launch_experts_tile(const void* x, const void* gu_tiles, const void*
   g.row_of = ws.tile_row;
   g.w_of = ws.tile_w;
   g.d = d;
-  cudaError_t e = launch_pdl(reinterpret_cast<const void*>(&k_gather_tiles), dim3(2 * grid), dim3(256), 0, s, &g);
+  cudaError_t e = launch_pdl(reinterpret_cast<const void*>(&k_gather_tiles), dim3(4 * grid), dim3(256), 0, s, &g);
   if (e != cudaSuccess) return e;
   TileArgs a = {};
   a.items = ws.items;

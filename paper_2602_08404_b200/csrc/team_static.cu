@@ -85,7 +85,7 @@ extern "C" int team_route_static(const team_config* cfg, const void* x, const vo
   d.T = st->n_rows; d.H = cfg->hidden; d.E = cfg->n_experts; d.k = cfg->top_k; d.I = cfg->inter; d.ns = cfg->n_shared;
   d.G = cfg->max_groups;
   team::Policy p;
-  p.flags = cfg->flags; p.tau_hot = cfg->tau_hot; p.L_hot = cfg->L_hot; p.inclusive = cfg->hot_dist_inclusive;
+  p.flags = (cfg->refresh_every > 0 && st->step_index % cfg->refresh_every == 0) ? (cfg->flags & ~TEAM_F_DCD) : cfg->flags; p.tau_hot = cfg->tau_hot; p.L_hot = cfg->L_hot; p.inclusive = cfg->hot_dist_inclusive;
   p.prefix_decoded = cfg->prefix_decoded; p.norm_topk = cfg->norm_topk;
   team::RoutePtrs e;
   memset(&e, 0, sizeof(e));
@@ -95,7 +95,7 @@ extern "C" int team_route_static(const team_config* cfg, const void* x, const vo
   // Every computed row's logits are rewritten by the first kernel and skipped rows are never read by the
   // second, so nothing in the shared scratch has to be cleared between calls.
   cudaError_t ce = team::launch_router_logits(x, cfg->dtype, static_cast<const float*>(w_router), st->tok_state, logits,
-                                              nullptr, d, cfg->flags, s);
+                                              nullptr, d, p.flags, s);
   if (ce == cudaSuccess) ce = team::launch_router_topk(logits, st->tok_state, e, d, p, s);
   return ce == cudaSuccess ? TEAM_OK : TEAM_ERR_CUDA;
 }

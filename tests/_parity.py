@@ -248,6 +248,7 @@ def run_schedule(shape, weights, steps, flags, force_simt=False, policy_switch=N
                 B.team_set_policy(layer.ctx, layer.cfg)
             x_dev = B.to_device(step["x"], dtype_code(shape))
             st = B.state_to_device(step)
+            st["step_index"] = si
             out = B.alloc_routing(layer.cfg, T)
             if not tables:
                 out = {n: out[n] for n in CHOICE_TABLES}
@@ -262,7 +263,7 @@ def run_schedule(shape, weights, steps, flags, force_simt=False, policy_switch=N
                 chosen = set(got["topk_idx"][comp].ravel().tolist())
                 got["n_active"] = len(chosen) + (shape.n_shared if comp.any() else 0)
             y_ref, ref = O.moe_forward(ocfg, weights, step["x"], step["tok_state"], step["conf"], step["pos"],
-                                       step["group"], step["branch"], y_prev=y_ref)
+                                       step["group"], step["branch"], y_prev=y_ref, step_index=si)
             what = f"{shape.name} flags={ocfg.flags} step={si}"
             exact, pin = compare_routing(ocfg, ref, got, step["group"], what, return_pin=True)
             got_y = y_dev.cpu().numpy()

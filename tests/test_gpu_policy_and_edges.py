@@ -114,6 +114,19 @@ def test_policy_switch_between_steps_of_one_context(switch):
             assert all(s["rows"] == shape.rows for s in stats[2:])
 
 
+@pytest.mark.parametrize("tables", [True, False], ids=["with_tables", "choices_only"])
+@pytest.mark.parametrize("shape", [W.C2, W.MINI_SHARED, W.C1], ids=lambda s: s.name)
+def test_periodic_refresh(shape, tables):
+    """Refresh-N (Sec. 4.1, second paragraph; Table 3): every N-th step recomputes all tokens, the others run with
+    delayed caching.  With N = 2 the steps 0, 2, 4 compute every row."""
+    steps = W.make_schedule(shape)
+    stats = P.run_schedule(shape, _weights(shape), steps, TEAM, tables=tables, refresh_every=2)
+    plain = P.run_schedule(shape, _weights(shape), steps, TEAM, tables=tables)
+    for s, q in zip(stats, plain):
+        assert s["rows"] == (shape.rows if s["step"] % 2 == 0 else q["rows"])
+    assert any(s["rows"] > q["rows"] for s, q in zip(stats, plain))       # the schedule does have cached rows to refresh
+
+
 def _plain_topk_reference(ocfg, logits32, probs, cls_computed):
     """Plain (unrestricted) top-k, weights and margin of every computed row, from the oracle's pieces."""
     T = logits32.shape[0]

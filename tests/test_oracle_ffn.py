@@ -199,6 +199,41 @@ def test_stack_with_single_expert_layers_is_a_residual_mlp_stack_with_rounding()
     np.testing.assert_array_equal(out, x.astype(np.float64))
 
 
+def test_periodic_refresh_recomputes_everything_every_nth_step():
+    """Sec. 4.1 (second paragraph) / Table 3: Refresh-N recomputes all tokens every N steps.  Pins: the computed-row
+    counts over an 8-step schedule follow by hand; a refresh step equals the same step with delayed caching off
+    (cached tokens are first-round rows there too); every other step equals plain delayed caching."""
+    rng = np.random.default_rng(12)
+    T, E, k, H, I = 4, 6, 2, 8, 4
+    w = _weights(rng, E, H, I)
+    x = rng.standard_normal((T, H)).astype(np.float32)
+    _, conf, pos, grp, br = _state(T)
+    # tokens 0..3 are accepted after steps 0, 2, 4, 6: NEW on the next step, cached from the one after
+    sched = []
+    for s in range(8):
+        st = np.zeros(T, np.uint8)
+        for p in range(T):
+            if s == 2 * p + 1:
+                st[p] = O.TOK_NEW
+            elif s > 2 * p + 1:
+                st[p] = O.TOK_CACHED
+        sched.append(st)
+    want = {0: [4, 4, 3, 3, 2, 2, 1, 1], 4: [4, 4, 3, 3, 4, 2, 1, 1], 8: [4, 4, 3, 3, 2, 2, 1, 1], 2: [4, 4, 4, 3, 4, 2, 4, 1]}
+    for n, rows in want.items():
+        cfg = O.Config(hidden=H, n_experts=E, top_k=k, inter=I, flags=O.F_DCD | O.F_LAC, L_hot=1, refresh_every=n)
+        plain = O.Config(hidden=H, n_experts=E, top_k=k, inter=I, flags=O.F_DCD | O.F_LAC, L_hot=1)
+        nodcd = O.Config(hidden=H, n_experts=E, top_k=k, inter=I, flags=O.F_LAC, L_hot=1)
+        got = []
+        for s, st in enumerate(sched):
+            y, r = O.moe_forward(cfg, w, x, st, conf, pos, grp, br, step_index=s)
+            got.append(r["n_rows_active"])
+            same_as = nodcd if (n > 0 and s % n == 0) else plain
+            y2, r2 = O.moe_forward(same_as, w, x, st, conf, pos, grp, br)
+            np.testing.assert_array_equal(y, y2)
+            np.testing.assert_array_equal(r["tok_class"], r2["tok_class"])
+        assert got == rows, (n, got)
+
+
 # --- planted mistakes: each must be caught by at least one pin ---------------------
 def _fails(pins, mod):
     for pin in pins:
