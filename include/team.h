@@ -292,6 +292,38 @@ const char *team_expert_kernel_name(const team_ctx *ctx);
  * Meant for triage of a parity failure, not for production. */
 int team_debug_force_simt(team_ctx *ctx, int on);
 
+/* Decode-loop glue of a block (Eq. 2-3; Sec. 4.2 "Speculative Exploration for Hot Tokens"; Sec. 5.4 "Aligned Token
+ * Candidates in SEH"): from the outputs of one forward pass over the block's branches -- predicted token and
+ * confidence per branch and position -- accept the confident positions (c > tau), verify the speculative branches
+ * in a chain, pick the next two candidates, and lay out the rows of the next forward pass for team_moe_forward.
+ *
+ * Branches (n_branches = 4; Sec. 5.1): 0 = base, 1 = base + 1st-confidence candidate accepted, 2 = base + 2nd,
+ * 3 = base + both.  A candidate is confirmed in a branch when that branch predicts the speculated token at its
+ * position with c > tau.  The base branch is always trusted; branch 1 after it if the 1st candidate is confirmed in
+ * the base branch, then branch 3 if the 2nd is confirmed in branch 1; else branch 2 if the 2nd is confirmed in the
+ * base branch, then branch 3 if the 1st is confirmed in branch 2.  Every masked position with c > tau in a trusted
+ * branch is accepted with the prediction of the first trusted branch that accepts it; confirmed candidates are
+ * accepted with their speculated tokens.  Accepted tokens are TEAM_TOK_NEW at the next step, the previous NEW ones
+ * TEAM_TOK_CACHED (Sec. 4.1).  The next candidates are the two masked positions with the highest confidences in the
+ * last trusted ("adopted") branch, ties to the lower position.  n_branches = 1 is plain threshold decoding (Eq. 3).
+ *
+ * All pointers are device memory owned by the caller.  team_seh_state persists over the steps of a block:
+ *   token [S, L] int32 (-1 while masked), state [S, L] uint8 TEAM_TOK_*, spec_pos / spec_tok [S, 2] int32 (the
+ *   candidates the given forward pass was run with; rewritten with the next ones), counters [S, 2] int32 (forward
+ *   passes, accepted tokens; optional).
+ * pred int32 / conf fp32 [S, n_branches, L]: the forward pass's outputs; both NULL begins a block (everything masked,
+ *   no candidates, counters zeroed).
+ * team_seh_rows: the next forward pass's step state, [S * n_branches * L] each, rows ordered [sequence][branch]
+ *   [position], group = sequence; conf is the adopted branch's for masked positions and 1 for decoded ones.
+ * adopted_out [S] int32 (optional): the adopted branch.  block <= TEAM_MAX_BLOCK, S * n_branches * block <=
+ * TEAM_MAX_ROWS.  Asynchronous on `stream`; needs no context.
+ * Errors: TEAM_ERR_ARG, TEAM_ERR_SHAPE, TEAM_ERR_CUDA. */
+typedef struct { int32_t n_seqs, block, n_branches; float tau; } team_seh_config;
+typedef struct { int32_t *token; uint8_t *state; int32_t *spec_pos; int32_t *spec_tok; int32_t *counters; } team_seh_state;
+typedef struct { uint8_t *tok_state; float *conf; int32_t *pos; int32_t *group; int32_t *branch; } team_seh_rows;
+int team_seh_step(const team_seh_config *cfg, const team_seh_state *state, const int32_t *pred, const float *conf,
+                  const team_seh_rows *rows, int32_t *adopted_out, void *stream);
+
 /* Diagnostic knobs of a context (not for production use).
  *   TEAM_KNOB_NO_FUSE (value 0/1): with at most 8 rows and no dispatch table asked for, team_moe_forward runs the
  *     whole step as one kernel; 1 keeps the three-kernel sequence (router, selection, experts) instead.

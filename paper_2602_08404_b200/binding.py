@@ -23,7 +23,7 @@ TEAM_F_DCD, TEAM_F_LAC = 1, 2
 TEAM_DTYPE_F32, TEAM_DTYPE_BF16 = 0, 1
 
 EXPORTS = ["team_create", "team_destroy", "team_set_weights", "team_set_policy", "team_route",
-           "team_route_static", "team_pack_w_down", "team_pack_w_tiles", "team_select_experts", "team_moe_forward", "team_moe_forward_host", "team_residual_add", "team_read_status",
+           "team_route_static", "team_pack_w_down", "team_pack_w_tiles", "team_seh_step", "team_select_experts", "team_moe_forward", "team_moe_forward_host", "team_residual_add", "team_read_status",
            "team_last_launch_count", "team_expert_kernel_name", "team_expert_timing", "team_debug_force_simt", "team_debug_knob", "team_strerror",
            "team_last_cuda_error", "team_version"]
 
@@ -45,6 +45,19 @@ class team_step_state(ctypes.Structure):
     _fields_ = [("n_rows", ctypes.c_int32), ("tok_state", ctypes.c_void_p), ("conf", ctypes.c_void_p),
                 ("pos", ctypes.c_void_p), ("group", ctypes.c_void_p), ("branch", ctypes.c_void_p),
                 ("step_index", ctypes.c_int32)]
+
+
+class team_seh_config(ctypes.Structure):
+    _fields_ = [("n_seqs", ctypes.c_int32), ("block", ctypes.c_int32), ("n_branches", ctypes.c_int32),
+                ("tau", ctypes.c_float)]
+
+
+class team_seh_state(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_void_p) for n in ("token", "state", "spec_pos", "spec_tok", "counters")]
+
+
+class team_seh_rows(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_void_p) for n in ("tok_state", "conf", "pos", "group", "branch")]
 
 
 class team_routing(ctypes.Structure):
@@ -71,6 +84,8 @@ def lib():
         L.team_route.argtypes = [vp, vp, ctypes.POINTER(team_step_state), ctypes.POINTER(team_routing), vp]
         L.team_pack_w_down.argtypes = [vp, vp, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int, vp]
         L.team_pack_w_tiles.argtypes = [vp, vp, vp, vp, vp, ctypes.c_int, ctypes.c_int, ctypes.c_int, vp]
+        L.team_seh_step.argtypes = [ctypes.POINTER(team_seh_config), ctypes.POINTER(team_seh_state), vp, vp,
+                                    ctypes.POINTER(team_seh_rows), vp, vp]
         L.team_route_static.argtypes = [ctypes.POINTER(team_config), vp, vp, ctypes.POINTER(team_step_state),
                                         ctypes.POINTER(team_routing), vp]
         L.team_select_experts.argtypes = [vp, ctypes.POINTER(team_step_state), ctypes.POINTER(team_routing), vp]
@@ -190,6 +205,26 @@ def team_route_static(cfg, x, w_router, st, out):
     r = _routing(out)
     return lib().team_route_static(ctypes.byref(cfg), _ptr(x), _ptr(w_router), ctypes.byref(_state(st)), ctypes.byref(r),
                                    _stream())
+
+
+def seh_alloc(n_seqs, block, n_branches=4, device="cuda"):
+    """Device buffers of the decode-loop glue: (state dict, rows dict) as team_seh_step takes them."""
+    z = lambda shape, dt: torch.zeros(shape, dtype=dt, device=device)
+    T = n_seqs * n_branches * block
+    state = dict(token=z((n_seqs, block), torch.int32), state=z((n_seqs, block), torch.uint8),
+                 spec_pos=z((n_seqs, 2), torch.int32), spec_tok=z((n_seqs, 2), torch.int32), counters=z((n_seqs, 2), torch.int32))
+    rows = dict(tok_state=z((T,), torch.uint8), conf=z((T,), torch.float32), pos=z((T,), torch.int32),
+                group=z((T,), torch.int32), branch=z((T,), torch.int32))
+    return state, rows
+
+
+def team_seh_step(n_seqs, block, n_branches, tau, state, pred, conf, rows, adopted=None):
+    """pred / conf: device tensors [S, n_branches, L] (both None: begin a block)."""
+    cfg = team_seh_config(n_seqs, block, n_branches, tau)
+    st = team_seh_state(*[_ptr(state[n]) for n, _ in team_seh_state._fields_])
+    rw = team_seh_rows(*[_ptr(rows[n]) for n, _ in team_seh_rows._fields_])
+    _check(lib().team_seh_step(ctypes.byref(cfg), ctypes.byref(st), _ptr(pred), _ptr(conf), ctypes.byref(rw), _ptr(adopted),
+                               _stream()))
 
 
 def team_select_experts(ctx, st, out):

@@ -144,6 +144,29 @@ def device_layer_weights(shape, layer_seed, device, std=0.02):
     return wr, wg, wu, wd
 
 
+def make_decode_script(n_seqs, block, n_steps, seed, n_branches=4, vocab=1000, rise=1.8, slope=0.5, boost=2.5):
+    """Scripted outputs of a language-model head for a decode loop: pred int32 and conf fp32 [steps][S][branches][L].
+
+    Stands in for the model's predictions (Eq. 2), which need a trained checkpoint.  The script does not depend on
+    the decoding state: it gives every position a prediction and a confidence at every step, and the decode loop
+    reads the ones it needs.  Confidence follows sigmoid(rise * (step + 1) - slope * position + boost * [branch has
+    extra accepted tokens] + noise): it grows from step to step, falls from left to right (tokens are accepted in a
+    near-autoregressive order, Sec. 3) and is a little higher in branches that carry speculated tokens.  The
+    prediction is the sequence's fixed target token, except that an unconfident position sometimes predicts
+    another token."""
+    rng = np.random.Generator(np.random.Philox(seed))
+    truth = rng.integers(0, vocab, size=(n_seqs, 1, block))
+    steps = np.arange(n_steps).reshape(n_steps, 1, 1, 1)
+    pos = np.arange(block).reshape(1, 1, 1, block)
+    extra = np.array([0, 1, 1, 2][:n_branches], dtype=np.float64).reshape(1, 1, n_branches, 1)
+    z = rise * (steps + 1) - slope * pos + boost * extra + rng.normal(0.0, 0.7, size=(n_steps, n_seqs, n_branches, block))
+    conf = (1.0 / (1.0 + np.exp(-z))).astype(np.float32)
+    other = rng.integers(0, vocab, size=conf.shape)
+    wrong = rng.random(conf.shape) > 0.4 + 0.6 * conf
+    pred = np.where(wrong, other, np.broadcast_to(truth[None], conf.shape)).astype(np.int32)
+    return pred, conf
+
+
 def _accept_step(shape, p):
     """Step at whose end position p is accepted (it is NEW at the following step)."""
     return (p // shape.unmask_per_step + 1) * shape.unmask_every - 1
