@@ -102,6 +102,96 @@ k_router_logits(const XT* __restrict__ x, const float* __restrict__ w_router, co
 }
 
 
+// Many rows (bf16 activations): a register-tiled fp32 FMA kernel.  A CTA takes 16 rows x 32 experts; the rows sit in
+// shared memory as bf16 (widened exactly on use); warp w takes experts 4w .. 4w+3 of the tile, its lanes stride
+// the hidden dimension four elements at a time (128-bit weight loads, 512 contiguous bytes per warp and expert)
+// and keep 4 x 16 accumulators each, so that one weight load feeds 16 rows and one row load feeds 4 experts.  The
+// 64 per-lane partial sums of a warp are reduced with a transposing butterfly (62 shuffles instead of 320).
+constexpr int kTiledRows = 16;
+constexpr int kTiledExperts = 32;      // per CTA: 8 warps x 4
+
+__device__ __forceinline__ void butterfly32(float (&v)[32], int lane) {
+  // after the five steps lane l holds the warp-wide sum of entry l
+#pragma unroll
+  for (int half = 16; half >= 1; half >>= 1) {
+    const bool upper = (lane & half) != 0;
+#pragma unroll
+    for (int i = 0; i < half; ++i) {
+      const float keep = upper ? v[i + half] : v[i];
+      const float send = upper ? v[i] : v[i + half];
+      v[i] = keep + __shfl_xor_sync(0xffffffffu, send, half);
+    }
+  }
+}
+
+__global__ void __launch_bounds__(256)
+k_router_logits_tiled(const __nv_bfloat16* __restrict__ x, const float* __restrict__ w_router,
+                      const uint8_t* __restrict__ tok_state, float* __restrict__ logits, float* __restrict__ y_zero,
+                      Dims d, int flags) {
+  extern __shared__ __align__(16) unsigned char s_xb[];   // [kTiledRows][H] bf16
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int H = d.H, T = d.T, E = d.E;
+  const int t0 = blockIdx.y * kTiledRows, nt = min(kTiledRows, T - t0);
+  const int e0 = blockIdx.x * kTiledExperts + warp * 4;
+  // stage the rows (16-byte pieces; rows beyond T are zero)
+  {
+    const uint4* src = reinterpret_cast<const uint4*>(x + (size_t)t0 * H);
+    uint4* dst = reinterpret_cast<uint4*>(s_xb);
+    const int n16 = nt * H / 8, all16 = kTiledRows * H / 8;
+    for (int i = tid; i < all16; i += 256) dst[i] = i < n16 ? __ldg(src + i) : make_uint4(0u, 0u, 0u, 0u);
+  }
+  if (y_zero != nullptr) {
+    for (int r = 0; r < nt; ++r) {
+      const bool skip = (flags & TEAM_F_DCD) && tok_state[t0 + r] == TEAM_TOK_CACHED;
+      if (!skip)
+        for (int i = blockIdx.x * 256 + tid; i < H; i += gridDim.x * 256) y_zero[(size_t)(t0 + r) * H + i] = 0.f;
+    }
+  }
+  __syncthreads();
+  float acc[2][32];                    // [pair of experts][expert-in-pair * 16 + row]
+#pragma unroll
+  for (int g = 0; g < 2; ++g)
+#pragma unroll
+    for (int i = 0; i < 32; ++i) acc[g][i] = 0.f;
+  const float4* wrow[4];
+#pragma unroll
+  for (int q = 0; q < 4; ++q) wrow[q] = reinterpret_cast<const float4*>(w_router + (size_t)min(e0 + q, E - 1) * H);
+  const int n4 = H >> 2;
+  float4 wv[4];
+#pragma unroll
+  for (int q = 0; q < 4; ++q) wv[q] = __ldg(wrow[q] + lane);
+  for (int c = lane; c < n4; c += 32) {
+    float4 wn[4];
+    const int cn = c + 32 < n4 ? c + 32 : c;             // next step's weights are requested before this step's math
+#pragma unroll
+    for (int q = 0; q < 4; ++q) wn[q] = __ldg(wrow[q] + cn);
+#pragma unroll
+    for (int r = 0; r < kTiledRows; ++r) {
+      const uint2 xb = *reinterpret_cast<const uint2*>(s_xb + ((size_t)r * H + c * 4) * 2);
+      const float2 lo = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&xb.x));
+      const float2 hi = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&xb.y));
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        float a = acc[q >> 1][(q & 1) * 16 + r];
+        a = fmaf(wv[q].x, lo.x, a);
+        a = fmaf(wv[q].y, lo.y, a);
+        a = fmaf(wv[q].z, hi.x, a);
+        a = fmaf(wv[q].w, hi.y, a);
+        acc[q >> 1][(q & 1) * 16 + r] = a;
+      }
+    }
+#pragma unroll
+    for (int q = 0; q < 4; ++q) wv[q] = wn[q];
+  }
+#pragma unroll
+  for (int g = 0; g < 2; ++g) {
+    butterfly32(acc[g], lane);
+    const int e = e0 + g * 2 + (lane >> 4), r = lane & 15;
+    if (e < E && r < nt) logits[(size_t)(t0 + r) * E + e] = acc[g][0];
+  }
+}
+
 // Few rows (T <= kRowTile): the whole job is one pass over the 4*E*H bytes of router weights, so it
 // is spread as widely as possible -- two experts per CTA, four warps per expert, each lane issuing all
 // of its 128-bit weight loads before anything else -- and the activations are staged once per CTA.
@@ -270,6 +360,7 @@ cudaError_t configure_router(int dtype, int hidden) {
   } else {
     e = prepare_kernel(k_router_logits<__nv_bfloat16>, smem);
     if (e == cudaSuccess) e = prepare_kernel(k_router_logits_small<__nv_bfloat16>, smem);
+    if (e == cudaSuccess) e = prepare_kernel(k_router_logits_tiled, smem);
   }
   if (e == cudaSuccess)
     e = cudaFuncSetAttribute(k_router_topk, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
@@ -288,6 +379,14 @@ cudaError_t launch_router_logits(const void* x, int dtype, const float* w_router
     else
       k_router_logits_small<__nv_bfloat16><<<grid, block, smem, s>>>(static_cast<const __nv_bfloat16*>(x), w_router,
                                                                      tok_state, logits, y_zero, d, flags);
+    return cudaGetLastError();
+  }
+  // the register-tiled kernel pays off once its 16-row x 32-expert tiles fill the SMs; smaller calls keep more,
+  // smaller CTAs in flight with the 8 x 8 kernel below
+  if (dtype == TEAM_DTYPE_BF16 && ((d.T + kTiledRows - 1) / kTiledRows) * ((d.E + kTiledExperts - 1) / kTiledExperts) >= 128) {
+    dim3 grid((d.E + kTiledExperts - 1) / kTiledExperts, (d.T + kTiledRows - 1) / kTiledRows);
+    k_router_logits_tiled<<<grid, 256, (size_t)kTiledRows * d.H * 2, s>>>(static_cast<const __nv_bfloat16*>(x), w_router,
+                                                                        tok_state, logits, y_zero, d, flags);
     return cudaGetLastError();
   }
   dim3 grid((d.E + kExpertsPerCta - 1) / kExpertsPerCta, (d.T + kRowTile - 1) / kRowTile);

@@ -534,7 +534,7 @@ cudaError_t launch_select(const float* logits, StepPtrs st, Workspace ws, RouteP
   cfg.numAttrs = 1;
   // Several groups and more rows than one CTA routes at once (one row per warp): the routing rounds run as
   // one CTA per group (up to 32), the dispatch as a second single-CTA launch.
-  const int group_ctas = d.G < 32 ? d.G : 32;
+  const int group_ctas = d.G < 128 ? d.G : 128;
   if (d.T > kSelWarps && (d.G == 1 || d.T / group_ctas > kSelWarps)) {
     // one group, or groups of more rows than a CTA routes at once: one cluster, rows split over its CTAs
     const int c = d.T > 64 ? 8 : 4;        // 16 rows or fewer per CTA up to 128 rows
@@ -560,7 +560,7 @@ cudaError_t launch_select(const float* logits, StepPtrs st, Workspace ws, RouteP
 }
 
 int select_launches(Dims d) {
-  const int group_ctas = d.G < 32 ? d.G : 32;
+  const int group_ctas = d.G < 128 ? d.G : 128;
   if (d.T > kSelWarps && (d.G == 1 || d.T / group_ctas > kSelWarps)) return 1;
   return d.G > 1 && d.T > kSelWarps ? 2 : 1;
 }
