@@ -106,6 +106,14 @@ typedef struct {
   int32_t refresh_every;      /* Sec. 4.1 / Table 3 (Refresh-4, Refresh-8): N > 0 recomputes every token on the
                                  steps with step_index % N == 0 (cached tokens are treated as newly accepted
                                  there); 0 = never, the paper's refresh-free choice                        */
+  int32_t ep_rank;            /* expert parallelism: this context computes the experts                    */
+  int32_t ep_world;           /* [ep_rank * E / ep_world, (ep_rank + 1) * E / ep_world) only; 0 or 1 = all.  With
+                                 ep_world > 1: n_experts must be a multiple of ep_world, n_shared must be 0, the
+                                 expert-weight tensors given to team_set_weights hold the context's OWN experts
+                                 only (E / ep_world of them, in order), router weights and routing are complete
+                                 and identical on every rank, and y receives this rank's PARTIAL sums for the
+                                 computed rows: the layer output is the sum over the ranks (an all-reduce of
+                                 the computed rows of y, which is the caller's to run)                     */
 } team_config;
 
 typedef struct {
@@ -335,8 +343,14 @@ int team_seh_step(const team_seh_config *cfg, const team_seh_state *state, const
  *   TEAM_KNOB_EXPERT_KERNEL (0/1/2): 0 lets max_rows choose the expert kernel of a bf16 context, 1 asks for the
  *     weight-streaming kernel, 2 for the tensor-memory kernels (ignored where the shape does not allow the kernel);
  *     the weight layout that kernel reads must have been given.
- * Errors: TEAM_ERR_ARG. */
-enum { TEAM_KNOB_NO_FUSE = 1, TEAM_KNOB_EXTRA_ARRIVALS = 2, TEAM_KNOB_WAIT_LIMIT_US = 3, TEAM_KNOB_EXPERT_KERNEL = 4 };
+ *   TEAM_KNOB_ORDERED_COMBINE (0/1): the weighted combine normally adds the experts' contributions into y with fp32
+ *     reductions, whose order (hence the last bits of y) varies from run to run.  1 makes the one-kernel step keep
+ *     one partial output per CTA and sum them in CTA order behind a second grid barrier: two runs are then identical
+ *     bit for bit, which tells a race from a rounding difference.  Allocates n_SMs x max_rows x H floats on first
+ *     use; only for contexts of at most 8 rows on hidden size 1024 or 2048 (else TEAM_ERR_SHAPE); a few us slower.
+ * Errors: TEAM_ERR_ARG, TEAM_ERR_SHAPE, TEAM_ERR_CUDA. */
+enum { TEAM_KNOB_NO_FUSE = 1, TEAM_KNOB_EXTRA_ARRIVALS = 2, TEAM_KNOB_WAIT_LIMIT_US = 3, TEAM_KNOB_EXPERT_KERNEL = 4,
+       TEAM_KNOB_ORDERED_COMBINE = 5 };
 int team_debug_knob(team_ctx *ctx, int knob, long long value);
 
 const char *team_strerror(int code);

@@ -33,7 +33,8 @@ class team_config(ctypes.Structure):
                 ("inter", ctypes.c_int32), ("n_shared", ctypes.c_int32), ("max_rows", ctypes.c_int32),
                 ("max_groups", ctypes.c_int32), ("dtype", ctypes.c_int32), ("flags", ctypes.c_int32),
                 ("tau_hot", ctypes.c_float), ("L_hot", ctypes.c_int32), ("hot_dist_inclusive", ctypes.c_int32),
-                ("prefix_decoded", ctypes.c_int32), ("norm_topk", ctypes.c_int32), ("refresh_every", ctypes.c_int32)]
+                ("prefix_decoded", ctypes.c_int32), ("norm_topk", ctypes.c_int32), ("refresh_every", ctypes.c_int32),
+                ("ep_rank", ctypes.c_int32), ("ep_world", ctypes.c_int32)]
 
 
 class team_weights(ctypes.Structure):
@@ -135,9 +136,9 @@ def _stream():
 
 
 def make_config(hidden, n_experts, top_k, inter, n_shared=0, max_rows=64, max_groups=1, dtype=TEAM_DTYPE_BF16,
-                flags=0, tau_hot=0.7, L_hot=3, hot_dist_inclusive=1, prefix_decoded=1, norm_topk=1, refresh_every=0):
+                flags=0, tau_hot=0.7, L_hot=3, hot_dist_inclusive=1, prefix_decoded=1, norm_topk=1, refresh_every=0, ep_rank=0, ep_world=1):
     return team_config(hidden, n_experts, top_k, inter, n_shared, max_rows, max_groups, dtype, flags, tau_hot,
-                       L_hot, hot_dist_inclusive, prefix_decoded, norm_topk, refresh_every)
+                       L_hot, hot_dist_inclusive, prefix_decoded, norm_topk, refresh_every, ep_rank, ep_world)
 
 
 # ---- the C entry points, same names, torch tensors for device memory ---------------------------------
@@ -279,6 +280,7 @@ def team_expert_timing(ctx, enable):
 
 
 TEAM_KNOB_NO_FUSE, TEAM_KNOB_EXTRA_ARRIVALS, TEAM_KNOB_WAIT_LIMIT_US, TEAM_KNOB_EXPERT_KERNEL = 1, 2, 3, 4
+TEAM_KNOB_ORDERED_COMBINE = 5
 
 
 def team_debug_knob(ctx, knob, value):

@@ -27,6 +27,7 @@ struct team_ctx {
   int no_fuse;        // diagnostic knob: keep the three-kernel sequence
   int extra_arrivals; // diagnostic knob: arrivals the fused step's barrier waits for beyond the grid's own
   long long spin_cycles;   // limit of device-side waits, in SM clock cycles
+  float* ordered;          // ordered combine of the one-kernel step: [SMs][max_rows][H] partial outputs (null: off)
   void* simt_act;   // diagnostic fp32-FMA path on bf16 weights: activation scratch
   // team_moe_forward_host: one device block and its pinned host mirror, [inputs | y]
   unsigned char* hs_dev;
@@ -55,6 +56,9 @@ int fail_cuda(team_ctx* ctx, cudaError_t e, const char* what) {
 team::Dims dims_of(const team_config& c, int T) {
   team::Dims d;
   d.T = T; d.H = c.hidden; d.E = c.n_experts; d.k = c.top_k; d.I = c.inter; d.ns = c.n_shared; d.G = c.max_groups;
+  const int world = c.ep_world > 1 ? c.ep_world : 1, per = c.n_experts / world;
+  d.elo = world > 1 ? c.ep_rank * per : 0;
+  d.ehi = world > 1 ? d.elo + per : c.n_experts;
   return d;
 }
 
@@ -87,6 +91,10 @@ int check_config(const team_config* c) {
     return TEAM_ERR_SHAPE;
   }
   if (c->L_hot < 0 || c->refresh_every < 0) return TEAM_ERR_ARG;
+  if (c->ep_world > 1) {
+    if (c->ep_rank < 0 || c->ep_rank >= c->ep_world) return TEAM_ERR_ARG;
+    if (c->n_experts % c->ep_world || c->n_shared != 0 || c->n_experts / c->ep_world < 1) return TEAM_ERR_SHAPE;
+  }
   return TEAM_OK;
 }
 
@@ -119,6 +127,22 @@ void drop_host_graph(team_ctx* ctx) {
   if (ctx->hs_graph) cudaGraphExecDestroy(ctx->hs_graph);
   ctx->hs_graph = nullptr;
   ctx->hs_graph_rows = 0;
+}
+
+// Expert parallelism: the context holds its own experts' weights only; the kernels index experts by their global
+// id, so every expert-weight pointer is moved back by the first local expert's offset (plain address arithmetic:
+// the kernels only ever touch the experts of the local range).
+const void* expert_base(const void* p, const team_ctx* ctx, const team::Dims& d) {
+  if (p == nullptr || d.elo == 0) return p;
+  const size_t elt = ctx->cfg.dtype == TEAM_DTYPE_F32 ? 4 : 2;
+  const size_t per_expert = (size_t)d.I * d.H * elt;
+  return reinterpret_cast<const void*>(reinterpret_cast<uintptr_t>(p) - (uintptr_t)d.elo * per_expert);
+}
+
+const void* gu_tiles_base(const team_ctx* ctx, const team::Dims& d) {      // gate and up tiles: two matrices per expert
+  const void* p = ctx->w.w_gu_tiles;
+  if (p == nullptr || d.elo == 0) return p;
+  return reinterpret_cast<const void*>(reinterpret_cast<uintptr_t>(p) - (uintptr_t)d.elo * ((size_t)2 * d.I * d.H * 2));
 }
 
 // The next pair of timing events of the context (created on demand).
@@ -199,6 +223,7 @@ int team_create(const team_config* cfg, team_ctx** out) {
   ctx->no_fuse = 0;
   ctx->extra_arrivals = 0;
   ctx->spin_cycles = 2000000000ll;      // about a second
+  ctx->ordered = nullptr;
   cudaError_t e = cudaGetDevice(&ctx->device);
   if (e == cudaSuccess) e = cudaDeviceGetAttribute(&ctx->n_sms, cudaDevAttrMultiProcessorCount, ctx->device);
   if (e != cudaSuccess) {
@@ -286,6 +311,7 @@ int team_destroy(team_ctx* ctx) {
   for (cudaEvent_t e : ctx->ev) cudaEventDestroy(e);
   cudaFree(ctx->ws_base);
   if (ctx->simt_act) cudaFree(ctx->simt_act);
+  if (ctx->ordered) cudaFree(ctx->ordered);
   if (ctx->hs_dev) cudaFree(ctx->hs_dev);
   if (ctx->hs_pin) cudaFreeHost(ctx->hs_pin);
   if (ctx->hs_graph) cudaGraphExecDestroy(ctx->hs_graph);
@@ -317,7 +343,7 @@ int team_set_policy(team_ctx* ctx, const team_config* cfg) {
   const team_config& c = ctx->cfg;
   if (cfg->hidden != c.hidden || cfg->n_experts != c.n_experts || cfg->top_k != c.top_k || cfg->inter != c.inter ||
       cfg->n_shared != c.n_shared || cfg->max_rows != c.max_rows || cfg->max_groups != c.max_groups ||
-      cfg->dtype != c.dtype)
+      cfg->dtype != c.dtype || cfg->ep_rank != c.ep_rank || cfg->ep_world != c.ep_world)
     return TEAM_ERR_SHAPE;
   if (cfg->L_hot < 0 || cfg->refresh_every < 0) return TEAM_ERR_ARG;
   ctx->cfg = *cfg;
@@ -393,9 +419,10 @@ int team_moe_forward(team_ctx* ctx, const void* x, const team_step_state* st, te
     // at most 8 rows and no dispatch table asked for: the whole step is one kernel
     if (ctx->timing && (e = timing_events(ctx, &ev0, &ev1)) != cudaSuccess) return fail_cuda(ctx, e, "event create");
     if (ev0) cudaEventRecord(ev0, s);
-    e = team::launch_step_fused(x, static_cast<const float*>(ctx->w.w_router), ctx->w.w_gate, ctx->w.w_up, ctx->w.w_down,
+    e = team::launch_step_fused(x, static_cast<const float*>(ctx->w.w_router), expert_base(ctx->w.w_gate, ctx, d),
+                                expert_base(ctx->w.w_up, ctx, d), expert_base(ctx->w.w_down, ctx, d),
                                 step_ptrs(st), ctx->ws, export_ptrs(out), y, d, policy_of(ctx->cfg, st), ctx->n_sms,
-                                ctx->spin_cycles, ctx->extra_arrivals, s);
+                                ctx->spin_cycles, ctx->extra_arrivals, ctx->ordered, s);
     if (e != cudaSuccess) return fail_cuda(ctx, e, "fused step");
     if (ev1) cudaEventRecord(ev1, s);
     ctx->last_launches = 1;
@@ -415,14 +442,16 @@ int team_moe_forward(team_ctx* ctx, const void* x, const team_step_state* st, te
   }
   if (tc) {
     if (ctx->stream_path)
-      e = team::launch_experts_stream(x, ctx->w.w_gate, ctx->w.w_up, ctx->w.w_down, ctx->ws, y, d, ctx->cfg.max_rows,
-                                      ctx->n_sms, s);
+      e = team::launch_experts_stream(x, expert_base(ctx->w.w_gate, ctx, d), expert_base(ctx->w.w_up, ctx, d),
+                                      expert_base(ctx->w.w_down, ctx, d), ctx->ws, y, d, ctx->cfg.max_rows, ctx->n_sms, s);
     else
-      e = team::launch_experts_tile(x, ctx->w.w_gu_tiles, ctx->w.w_down_tiles, ctx->ws, y, d, ctx->n_sms, s);
+      e = team::launch_experts_tile(x, gu_tiles_base(ctx, d), expert_base(ctx->w.w_down_tiles, ctx, d), ctx->ws, y, d,
+                                    ctx->n_sms, s);
     if (e != cudaSuccess) return fail_cuda(ctx, e, "expert kernel");
     ctx->last_launches += ctx->stream_path ? 1 : 3;
   } else {
-    e = team::launch_experts_simt(x, ctx->cfg.dtype, ctx->w.w_gate, ctx->w.w_up, ctx->w.w_down, ctx->ws, y, d, s);
+    e = team::launch_experts_simt(x, ctx->cfg.dtype, expert_base(ctx->w.w_gate, ctx, d), expert_base(ctx->w.w_up, ctx, d),
+                                  expert_base(ctx->w.w_down, ctx, d), ctx->ws, y, d, s);
     if (e != cudaSuccess) return fail_cuda(ctx, e, "expert kernels (fp32)");
     ctx->last_launches += 2;
   }
@@ -563,6 +592,18 @@ int team_debug_knob(team_ctx* ctx, int knob, long long value) {
   if (ctx == nullptr) return TEAM_ERR_ARG;
   switch (knob) {
     case TEAM_KNOB_NO_FUSE: ctx->no_fuse = value != 0; break;
+    case TEAM_KNOB_ORDERED_COMBINE:
+      // only the one-kernel step has the ordered mode (its CTAs meet at a grid barrier anyway)
+      if (!ctx->fused_ok || team::experts_stream_gathers(ctx->cfg.max_rows)) return TEAM_ERR_SHAPE;
+      if (value != 0 && ctx->ordered == nullptr) {
+        const cudaError_t e = cudaMalloc(reinterpret_cast<void**>(&ctx->ordered),
+                                         (size_t)ctx->n_sms * ctx->cfg.max_rows * ctx->cfg.hidden * sizeof(float));
+        if (e != cudaSuccess) return fail_cuda(ctx, e, "ordered-combine scratch");
+      } else if (value == 0 && ctx->ordered != nullptr) {
+        cudaFree(ctx->ordered);
+        ctx->ordered = nullptr;
+      }
+      break;
     case TEAM_KNOB_EXPERT_KERNEL:
       if (value < 0 || value > 2) return TEAM_ERR_ARG;
       ctx->prefer = (int)value;

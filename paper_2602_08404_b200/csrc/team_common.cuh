@@ -18,6 +18,7 @@ struct Dims {
   int I;   // expert intermediate
   int ns;  // shared experts
   int G;   // max groups
+  int elo, ehi;   // expert parallelism: this call computes the routed experts [elo, ehi) only (0, E without it)
 };
 
 // Eq. 4 / Algorithm 1 policy knobs.
@@ -117,7 +118,7 @@ cudaError_t launch_experts_stream(const void* x, const void* w_gate, const void*
 bool step_fused_supported(int hidden, int max_rows, int n_experts, int grid);
 cudaError_t launch_step_fused(const void* x, const float* w_router, const void* w_gate, const void* w_up, const void* w_down,
                               StepPtrs st, Workspace ws, RoutePtrs ex, float* y, Dims d, Policy p, int grid,
-                              long long spin_cycles, int extra_arrivals, cudaStream_t s);
+                              long long spin_cycles, int extra_arrivals, float* ordered, cudaStream_t s);
 cudaError_t launch_router_logits(const void* x, int dtype, const float* w_router, const uint8_t* tok_state,
                                  float* logits, float* y_zero, Dims d, int flags, cudaStream_t s);
 cudaError_t launch_router_topk(const float* logits, const uint8_t* tok_state, RoutePtrs out, Dims d, Policy p,

@@ -70,7 +70,7 @@ k_gate_up(const WT* __restrict__ x, const WT* __restrict__ w_gate, const WT* __r
   const int slot = blockIdx.y;
   int e, t;
   slot_expert_row(slot, d, topk_idx, tok_class, e, t);
-  if (e < 0) return;
+  if (e < 0 || (e < d.E && (e < d.elo || e >= d.ehi))) return;      // not computed, or another rank's expert
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int i = blockIdx.x * 8 + warp;
   if (i >= d.I) return;
@@ -103,7 +103,7 @@ k_down(const WT* __restrict__ w_down, const float* __restrict__ act, const int32
       e = d.E + (j - d.k);
       w = 1.f;
     }
-    if (e < 0) continue;
+    if (e < 0 || (e < d.E && (e < d.elo || e >= d.ehi))) continue;
     // W_down is stored in slabs of 16 columns: element (e, h, c) sits at (((e * I/16 + c/16) * H + h) * 16 + c%16)
     const WT* wr = w_down + ((size_t)e * (d.I / 16) * d.H + h) * 16;
     const float* ar = act + (size_t)slot * d.I;

@@ -73,6 +73,7 @@ struct StArgs {
   int32_t* status;
   long long spin_cycles;        // limit of the barrier's wait
   int extra_arrivals;           // diagnostic: arrivals the barrier waits for beyond the grid's own (0 in normal use)
+  float* ordered;               // ordered combine: [grid][T][H] per-CTA partial outputs (null: fp32 reductions into y)
 };
 
 __device__ __forceinline__ uint32_t st_smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -268,6 +269,10 @@ __global__ void __launch_bounds__(kStThreads, 1) k_experts_stream(StArgs a) {
         const int t = (i * 4) / H;
         if (!((skip_rows >> t) & 1u)) reinterpret_cast<float4*>(a.y)[i] = make_float4(0.f, 0.f, 0.f, 0.f);
       }
+    }
+    if (a.ordered != nullptr) {
+      float4* mine = reinterpret_cast<float4*>(a.ordered + (size_t)blockIdx.x * T * H);
+      for (int i = tid; i < T * H / 4; i += kStThreads) mine[i] = make_float4(0.f, 0.f, 0.f, 0.f);
     }
     if (tid < 64) f_mask[tid] = 0u;
     if (tid == 64) *f_flag = 0;
@@ -472,6 +477,16 @@ __global__ void __launch_bounds__(kStThreads, 1) k_experts_stream(StArgs a) {
       const bool any = __ballot_sync(0xffffffffu, lane < T && c_cls[lane] != TEAM_CLS_SKIP) != 0u;
       for (int sh = 0; sh < d.ns && any; ++sh)
         if (lane == ((d.E + sh) >> 5)) act_word |= 1u << ((d.E + sh) & 31);
+    }
+    if (d.elo > 0 || d.ehi < d.E) {
+      // expert parallelism: only this rank's routed experts [elo, ehi) are computed here
+      const int lo = lane * 32, hi = lo + 32;
+      uint32_t keep = 0u;
+      if (hi > d.elo && lo < d.ehi) {
+        const int a0 = max(d.elo, lo) - lo, a1 = min(d.ehi, hi) - lo;       // bits [a0, a1)
+        keep = (a1 - a0 == 32) ? 0xffffffffu : (((1u << (a1 - a0)) - 1u) << a0);
+      }
+      act_word &= keep;
     }
     n_act = __reduce_add_sync(0xffffffffu, __popc(act_word));
   }
@@ -777,7 +792,10 @@ __global__ void __launch_bounds__(kStThreads, 1) k_experts_stream(StArgs a) {
         __syncwarp();
         // the expert's groups in this pass are summed: scale by the routing weights and add to y
         if (q == ng - 1 || s_item[q + 1] != s_item[q]) {
-          float* y0 = a.y + warp * HW + ch * 64 + g;
+          // ordered combine (one-kernel step only): the CTA's own partial output, every element owned by one thread,
+          // summed over the CTAs in index order at the end of the kernel; otherwise fp32 reductions into y
+          const bool ordered = FUSED && a.ordered != nullptr;
+          float* y0 = (ordered ? a.ordered + (size_t)blockIdx.x * T * H : a.y) + warp * HW + ch * 64 + g;
 #pragma unroll
           for (int nt = 0; nt < NTL; ++nt) {
             const int cA = nt * 8 + 2 * c, cB = cA + 1;          // this thread's two token columns
@@ -787,13 +805,24 @@ __global__ void __launch_bounds__(kStThreads, 1) k_experts_stream(StArgs a) {
             float* yB = y0 + (size_t)max(rB, 0) * H;
 #pragma unroll
             for (int u = 0; u < 4; ++u) {
-              if (wA != 0.f) {
-                atomicAdd(yA + u * 16, wA * acc[u][nt][0]);
-                atomicAdd(yA + u * 16 + 8, wA * acc[u][nt][2]);
-              }
-              if (wB != 0.f) {
-                atomicAdd(yB + u * 16, wB * acc[u][nt][1]);
-                atomicAdd(yB + u * 16 + 8, wB * acc[u][nt][3]);
+              if (ordered) {
+                if (wA != 0.f) {
+                  yA[u * 16] += wA * acc[u][nt][0];
+                  yA[u * 16 + 8] += wA * acc[u][nt][2];
+                }
+                if (wB != 0.f) {
+                  yB[u * 16] += wB * acc[u][nt][1];
+                  yB[u * 16 + 8] += wB * acc[u][nt][3];
+                }
+              } else {
+                if (wA != 0.f) {
+                  atomicAdd(yA + u * 16, wA * acc[u][nt][0]);
+                  atomicAdd(yA + u * 16 + 8, wA * acc[u][nt][2]);
+                }
+                if (wB != 0.f) {
+                  atomicAdd(yB + u * 16, wB * acc[u][nt][1]);
+                  atomicAdd(yB + u * 16 + 8, wB * acc[u][nt][3]);
+                }
               }
               acc[u][nt][0] = acc[u][nt][1] = acc[u][nt][2] = acc[u][nt][3] = 0.f;
             }
@@ -805,6 +834,40 @@ __global__ void __launch_bounds__(kStThreads, 1) k_experts_stream(StArgs a) {
     __syncthreads();        // s_act, s_w and the partial sums are free for the next pass
   }
   if (FUSED && !late_done) late_select();      // a CTA without any group still owes its part (CTA 0: the exports)
+  if constexpr (FUSED) {
+    if (a.ordered != nullptr) {
+      // ---- ordered combine: a second grid barrier, then y = sum over the CTAs' partial outputs in index order ----
+      __syncthreads();
+      if (tid == 0) {
+        __threadfence();
+        atomicAdd(a.arrivals, 1ull);
+        const unsigned long long target = bar_target - (unsigned long long)a.extra_arrivals + gridDim.x;
+        const long long t_begin = clock64();
+        while (st_ld_acquire(a.arrivals) < target) {
+          if (clock64() - t_begin > a.spin_cycles) {
+            *f_flag = 1;
+            break;
+          }
+        }
+      }
+      __syncthreads();
+      if (*f_flag) {
+        if (tid == 0) set_status(a.status, TEAM_ERR_TIMEOUT, 21);
+        return;
+      }
+      const int total4 = T * H / 4, n_cta = gridDim.x;
+      for (int i = blockIdx.x * kStThreads + tid; i < total4; i += n_cta * kStThreads) {
+        const int t = (i * 4) / H;
+        if (c_cls[t] == TEAM_CLS_SKIP) continue;
+        float4 sum = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int cta = 0; cta < n_cta; ++cta) {
+          const float4 v = __ldcg(reinterpret_cast<const float4*>(a.ordered + (size_t)cta * T * H) + i);
+          sum.x += v.x; sum.y += v.y; sum.z += v.z; sum.w += v.w;
+        }
+        reinterpret_cast<float4*>(a.y)[i] = sum;
+      }
+    }
+  }
 }
 
 // Few rows: all rows resident.  Up to kStGatherMaxRows rows: work items whose rows are gathered per item, of
@@ -868,8 +931,9 @@ bool step_fused_supported(int hidden, int max_rows, int n_experts, int grid) {
 
 cudaError_t launch_step_fused(const void* x, const float* w_router, const void* w_gate, const void* w_up, const void* w_down,
                               StepPtrs st, Workspace ws, RoutePtrs ex, float* y, Dims d, Policy p, int grid,
-                              long long spin_cycles, int extra_arrivals, cudaStream_t s) {
+                              long long spin_cycles, int extra_arrivals, float* ordered, cudaStream_t s) {
   StArgs a = {};
+  a.ordered = ordered;
   a.x = static_cast<const __nv_bfloat16*>(x);
   a.w_gate = static_cast<const __nv_bfloat16*>(w_gate);
   a.w_up = static_cast<const __nv_bfloat16*>(w_up);

@@ -365,7 +365,8 @@ k_select(const float* __restrict__ logits, StepPtrs st, Workspace ws, RoutePtrs 
     } else if (e < EN) {
       c = n_rows_active;
     }
-    tiles = (c + item_tile - 1) / item_tile;      // work items: ceil(c / item_tile) per expert
+    tiles = (c + item_tile - 1) / item_tile;      // work items: ceil(c / item_tile) per expert ...
+    if (e < E && (e < d.elo || e >= d.ehi)) tiles = 0;      // ... of this rank's own (expert parallelism)
     incl_c = c;
     incl_t = tiles;
 #pragma unroll

@@ -84,6 +84,7 @@ extern "C" int team_route_static(const team_config* cfg, const void* x, const vo
   team::Dims d;
   d.T = st->n_rows; d.H = cfg->hidden; d.E = cfg->n_experts; d.k = cfg->top_k; d.I = cfg->inter; d.ns = cfg->n_shared;
   d.G = cfg->max_groups;
+  d.elo = 0; d.ehi = cfg->n_experts;
   team::Policy p;
   p.flags = (cfg->refresh_every > 0 && st->step_index % cfg->refresh_every == 0) ? (cfg->flags & ~TEAM_F_DCD) : cfg->flags; p.tau_hot = cfg->tau_hot; p.L_hot = cfg->L_hot; p.inclusive = cfg->hot_dist_inclusive;
   p.prefix_decoded = cfg->prefix_decoded; p.norm_topk = cfg->norm_topk;

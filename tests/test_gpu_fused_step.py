@@ -107,3 +107,50 @@ def test_barrier_wait_runs_out_and_reports_a_timeout_without_hanging():
         assert err <= P.TOL_BF16 * np.abs(y_ref[comp]).max()
     finally:
         layer.close()
+
+
+def _ys_of_a_schedule(shape, steps, knobs, host_entry=False):
+    """y after every step of a schedule on a fresh context (no exports: the one-kernel step)."""
+    layer = P.Layer(shape, _weights(shape), TEAM)
+    for knob, value in knobs:
+        B.team_debug_knob(layer.ctx, knob, value)
+    T, H = shape.rows, shape.hidden
+    y = torch.zeros((T, H), dtype=torch.float32, device="cuda")
+    y_host = torch.zeros((T, H), dtype=torch.float32)
+    out = []
+    try:
+        for step in steps:
+            if host_entry:
+                st_host = {"tok_state": torch.as_tensor(step["tok_state"].astype(np.uint8)),
+                           "conf": torch.as_tensor(step["conf"].astype(np.float32)),
+                           "pos": torch.as_tensor(step["pos"].astype(np.int32)),
+                           "group": torch.as_tensor(step["group"].astype(np.int32)),
+                           "branch": torch.as_tensor(step["branch"].astype(np.int32))}
+                B.team_moe_forward_host(layer.ctx, torch.as_tensor(step["x"]).to(torch.bfloat16), st_host, None, y_host)
+                out.append(y_host.clone())
+            else:
+                B.team_moe_forward(layer.ctx, B.to_device(step["x"], B.TEAM_DTYPE_BF16), B.state_to_device(step), None, y)
+                assert B.team_last_launch_count(layer.ctx) == 1
+                out.append(y.cpu())
+        assert B.team_read_status(layer.ctx)[0] == B.TEAM_OK
+    finally:
+        layer.close()
+    return out
+
+
+@pytest.mark.parametrize("shape", [W.C2, W.STREAM_MULTI], ids=lambda s: s.name)
+def test_ordered_combine_is_reproducible_bit_for_bit(shape):
+    """With the ordered combine the contributions to y are summed in a fixed order: two runs, and the host-buffer
+    entry point against the device one, give identical bits; the default mode (fp32 reductions in arrival order)
+    agrees with it to rounding of the sums; and the ordered result matches the oracle like any other."""
+    steps = W.make_schedule(shape) * 2
+    ordered = [(B.TEAM_KNOB_ORDERED_COMBINE, 1)]
+    a = _ys_of_a_schedule(shape, steps, ordered)
+    b = _ys_of_a_schedule(shape, steps, ordered)
+    c = _ys_of_a_schedule(shape, steps, ordered, host_entry=True)
+    d = _ys_of_a_schedule(shape, steps, [])
+    for ya, yb, yc, yd in zip(a, b, c, d):
+        assert torch.equal(ya, yb) and torch.equal(ya, yc)
+        assert torch.allclose(ya, yd, rtol=0, atol=1e-5 * float(ya.abs().max()))
+    stats = P.run_schedule(shape, _weights(shape), W.make_schedule(shape), TEAM, tables=False, knobs=ordered)
+    assert all(s["launches"] == 1 for s in stats)

@@ -109,3 +109,41 @@ def test_bench_hands_gpus_n_to_the_launcher(monkeypatch):
         assert e.code == 17
     assert seen["n"] == 2 and seen["argv"] == ["--gpus", "2", "--steps", "20", "--warmup", "5"]
     assert os.path.basename(seen["script"]) == "bench.py"
+
+
+def _ep_worker(rank, world, port, out):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    sys.path.insert(0, ROOT)
+    from paper_2602_08404_b200 import ep as EP
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        T, H = 5, 8
+        tok_class = torch.tensor([1, 0, 2, 1, 0], dtype=torch.uint8)           # rows 1 and 4 were not computed
+        y = torch.full((T, H), 100.0 + rank)                                    # what the rank's y held before the step
+        y[tok_class != 0] = torch.arange(T * H, dtype=torch.float32).view(T, H)[tok_class != 0] * (rank + 1)
+        got = EP.combine_partial_outputs(y, tok_class)
+        out.put((rank, got.numpy().copy(), EP.expert_range(128, rank, world)))
+    finally:
+        dist.destroy_process_group()
+
+
+def test_expert_parallel_outputs_are_summed_on_the_computed_rows_only():
+    """The exchange step of expert-parallel sharding (two gloo ranks on CPU): computed rows become the sum of the
+    ranks' partial sums, rows that were not computed keep each rank's own previous values."""
+    ctx = mp.get_context("spawn")
+    out = ctx.Queue()
+    port = 29500 + (os.getpid() + 313) % 2000
+    procs = [ctx.Process(target=_ep_worker, args=(r, 2, port, out)) for r in range(2)]
+    for p in procs:
+        p.start()
+    got = sorted((out.get(timeout=120) for _ in procs), key=lambda g: g[0])
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    base = torch.arange(40, dtype=torch.float32).view(5, 8).numpy()
+    for rank, y, rng in got:
+        for t in (0, 2, 3):
+            assert (y[t] == base[t] * 3).all()                   # 1x + 2x
+        for t in (1, 4):
+            assert (y[t] == 100.0 + rank).all()
+        assert rng == (64 * rank, 64 * rank + 64)
