@@ -332,6 +332,30 @@ typedef struct { uint8_t *tok_state; float *conf; int32_t *pos; int32_t *group; 
 int team_seh_step(const team_seh_config *cfg, const team_seh_state *state, const int32_t *pred, const float *conf,
                   const team_seh_rows *rows, int32_t *adopted_out, void *stream);
 
+/* The attention half of delayed caching (Sec. 4.1; block diffusion, Sec. 2): one attention layer of one denoising
+ * step over the block being decoded.  Attention is bidirectional inside the block and runs over the cached keys /
+ * values of earlier blocks (the prefix).  Rows of cached tokens are not computed (flags & TEAM_F_DCD): they have no
+ * query, their output rows are left untouched, and the other rows see their keys / values from the in-block cache;
+ * after the pass the keys / values of the decoded rows computed in the base branch (branch 0) -- the tokens newly
+ * accepted in the previous step -- are inserted into that cache at their positions (delayed insertion).  A token
+ * that only a speculative branch treats as accepted is not inserted: the cache is shared by a sequence's branches.
+ *
+ * Rows are ordered [sequence][branch][position] and every (sequence, branch) presents its whole block:
+ * st->n_rows = n_seqs * n_branches * block, pos = 0 .. block-1 inside each run, group = sequence (a row that breaks
+ * this sets TEAM_ERR_STATE in `status`; conf is not read).  All pointers are device memory owned by the caller, 16-byte
+ * aligned; bf16 unless stated:
+ *   q [T, n_heads, head_dim]; k_new, v_new [T, n_kv_heads, head_dim] (this pass's projections of the rows);
+ *   k_prefix, v_prefix [n_seqs, max_prefix, n_kv_heads, head_dim] with prefix_len [n_seqs] int32 valid entries;
+ *   k_block, v_block [n_seqs, block, n_kv_heads, head_dim]: the in-block cache, read and then updated;
+ *   out fp32 [T, n_heads, head_dim]: softmax(q k^T / sqrt(head_dim)) v over prefix + block, computed rows only;
+ *   status int32 [2] (optional): first device-detected problem (code, detail), to be zeroed by the caller.
+ * Query head h uses key / value head h / (n_heads / n_kv_heads).  head_dim is 64 or 128, block <= TEAM_MAX_BLOCK.
+ * Asynchronous on `stream`; needs no context.  Errors: TEAM_ERR_ARG, TEAM_ERR_SHAPE, TEAM_ERR_CUDA. */
+typedef struct { int32_t n_heads, n_kv_heads, head_dim, block, n_seqs, n_branches, max_prefix, flags; } team_attn_config;
+int team_block_attention(const team_attn_config *cfg, const team_step_state *st, const void *q, const void *k_new,
+                         const void *v_new, const void *k_prefix, const void *v_prefix, const int32_t *prefix_len,
+                         void *k_block, void *v_block, float *out, int32_t *status, void *stream);
+
 /* Diagnostic knobs of a context (not for production use).
  *   TEAM_KNOB_NO_FUSE (value 0/1): with at most 8 rows and no dispatch table asked for, team_moe_forward runs the
  *     whole step as one kernel; 1 keeps the three-kernel sequence (router, selection, experts) instead.

@@ -23,7 +23,7 @@ TEAM_F_DCD, TEAM_F_LAC = 1, 2
 TEAM_DTYPE_F32, TEAM_DTYPE_BF16 = 0, 1
 
 EXPORTS = ["team_create", "team_destroy", "team_set_weights", "team_set_policy", "team_route",
-           "team_route_static", "team_pack_w_down", "team_pack_w_tiles", "team_seh_step", "team_select_experts", "team_moe_forward", "team_moe_forward_host", "team_residual_add", "team_read_status",
+           "team_route_static", "team_pack_w_down", "team_pack_w_tiles", "team_seh_step", "team_block_attention", "team_select_experts", "team_moe_forward", "team_moe_forward_host", "team_residual_add", "team_read_status",
            "team_last_launch_count", "team_expert_kernel_name", "team_expert_timing", "team_debug_force_simt", "team_debug_knob", "team_strerror",
            "team_last_cuda_error", "team_version"]
 
@@ -61,6 +61,11 @@ class team_seh_rows(ctypes.Structure):
     _fields_ = [(n, ctypes.c_void_p) for n in ("tok_state", "conf", "pos", "group", "branch")]
 
 
+class team_attn_config(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int32) for n in ("n_heads", "n_kv_heads", "head_dim", "block", "n_seqs", "n_branches",
+                                               "max_prefix", "flags")]
+
+
 class team_routing(ctypes.Structure):
     _fields_ = [(n, ctypes.c_void_p) for n in
                 ("probs", "topk_idx", "topk_w", "margin", "tok_class", "group_mask", "expert_count",
@@ -87,6 +92,7 @@ def lib():
         L.team_pack_w_tiles.argtypes = [vp, vp, vp, vp, vp, ctypes.c_int, ctypes.c_int, ctypes.c_int, vp]
         L.team_seh_step.argtypes = [ctypes.POINTER(team_seh_config), ctypes.POINTER(team_seh_state), vp, vp,
                                     ctypes.POINTER(team_seh_rows), vp, vp]
+        L.team_block_attention.argtypes = [ctypes.POINTER(team_attn_config), ctypes.POINTER(team_step_state)] + [vp] * 11
         L.team_route_static.argtypes = [ctypes.POINTER(team_config), vp, vp, ctypes.POINTER(team_step_state),
                                         ctypes.POINTER(team_routing), vp]
         L.team_select_experts.argtypes = [vp, ctypes.POINTER(team_step_state), ctypes.POINTER(team_routing), vp]
@@ -226,6 +232,15 @@ def team_seh_step(n_seqs, block, n_branches, tau, state, pred, conf, rows, adopt
     rw = team_seh_rows(*[_ptr(rows[n]) for n, _ in team_seh_rows._fields_])
     _check(lib().team_seh_step(ctypes.byref(cfg), ctypes.byref(st), _ptr(pred), _ptr(conf), ctypes.byref(rw), _ptr(adopted),
                                _stream()))
+
+
+def team_block_attention(cfg, st, q, k_new, v_new, k_prefix, v_prefix, prefix_len, k_block, v_block, out, status=None):
+    """cfg: team_attn_config; st: dict of device tensors (tok_state, pos, group, branch; conf is not read)."""
+    T = int(st["tok_state"].shape[0])
+    s = team_step_state(T, _ptr(st["tok_state"]), _ptr(st.get("conf")), _ptr(st["pos"]), _ptr(st["group"]), _ptr(st["branch"]), 0)
+    return lib().team_block_attention(ctypes.byref(cfg), ctypes.byref(s), _ptr(q), _ptr(k_new), _ptr(v_new), _ptr(k_prefix),
+                                      _ptr(v_prefix), _ptr(prefix_len), _ptr(k_block), _ptr(v_block), _ptr(out), _ptr(status),
+                                      _stream())
 
 
 def team_select_experts(ctx, st, out):
