@@ -77,7 +77,7 @@ def sm_max_hz():
 
 
 def measured_peaks():
-    """(HBM GB/s, bf16 TFLOP/s burst, sustained, kind) from the measured-peaks file, else the pool's earlier figures."""
+    """(HBM GB/s, bf16 TFLOP/s burst, sustained, kind) from the measured-peaks file, else earlier measurements of the same GPU model."""
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
         with open(path) as f:
@@ -794,8 +794,10 @@ def run_attn(args):
             us = e0.elapsed_time(e1) * 1e3 / (reps * n)
             comp = np.mean([(s["tok_state"] != 2).sum() if flags else T for s in steps])
             bytes_ = 2 * (P + L) * Hkv * d * 2 + comp * Hq * d * (2 + 4) + 2 * T * Hkv * d * 2
+            flops = 4.0 * comp * Hq * (P + L) * d          # q k^T and p v, 2 flops per multiply-add
             res[name] = {"us_per_call": us, "rows_computed_mean": float(comp), "algorithmic_bytes": float(bytes_),
-                         "hbm_frac": bytes_ / (us * 1e-6) / 1e9 / measured_peaks()[0]}
+                         "hbm_frac": bytes_ / (us * 1e-6) / 1e9 / measured_peaks()[0],
+                         "algorithmic_flops": flops, "tensor_tflops": flops / (us * 1e-6) / 1e12}
     t = res["delayed_caching"]
     line = {"metric": METRIC, "value": T / (t["us_per_call"] * 1e-6), "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": 3, "ms_per_step": t["us_per_call"] * 1e-3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -804,8 +806,10 @@ def run_attn(args):
                                    f"prefix {P}", "flags": 1, "rows_presented": T,
                        "l2": f"inputs larger than L2: KV caches rotate over {R} layers", "parallelism": "replicas"},
             "clocks": sampler.summary(), "delayed_caching": t, "recompute_all": res["recompute_all"],
-            "roofline": {"bound": "hbm", "kernel": "k_block_attention", "achieved": t["algorithmic_bytes"] / (t["us_per_call"] * 1e-6) / 1e9,
-                         "peak": measured_peaks()[0], "peak_kind": "of " + measured_peaks()[3], "unit": "GB/s", "frac": t["hbm_frac"],
+            # a contraction: at this shape the flops take longer on the tensor roof than the bytes on the HBM roof
+            "roofline": {"bound": "tensor", "kernel": "k_block_attention", "achieved": t["tensor_tflops"],
+                         "peak": measured_peaks()[2], "peak_kind": "of " + measured_peaks()[3] + " (bf16 sustained)",
+                         "unit": "TFLOP/s", "frac": t["tensor_tflops"] / measured_peaks()[2], "hbm_frac": t["hbm_frac"],
                          "traffic": None},
             "gpu_launches": 2 * args.steps}
     if rank == 0:
