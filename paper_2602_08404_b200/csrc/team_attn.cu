@@ -20,7 +20,7 @@
 
 #include <mutex>
 
-#include "team_common.cuh"
+#include "team_attn.cuh"
 #include "team_topk.cuh"
 
 namespace cg = cooperative_groups;
@@ -30,29 +30,7 @@ namespace team {
 constexpr int kAttnThreads = 256;
 constexpr int kAttnWarps = 8;
 constexpr int kAttnKeys = 64;          // keys per tile
-constexpr int kAttnPairs = 128;        // (row, head) pairs per CTA
 constexpr int kAttnStages = 3;
-constexpr int kAttnMaxSplits = 8;      // portable cluster size
-
-struct AttnArgs {
-  const __nv_bfloat16* q;        // [T, Hq, d]
-  const __nv_bfloat16* k_new;    // [T, Hkv, d]
-  const __nv_bfloat16* v_new;
-  const __nv_bfloat16* k_prefix; // [S, P, Hkv, d]
-  const __nv_bfloat16* v_prefix;
-  const int32_t* prefix_len;     // [S]
-  __nv_bfloat16* k_block;        // [S, L, Hkv, d]
-  __nv_bfloat16* v_block;
-  const uint8_t* tok_state;      // [T]
-  const int32_t* pos;
-  const int32_t* group;
-  const int32_t* branch;
-  float* out;                    // [T, Hq, d]
-  int32_t* status;               // [2] optional
-  int S, B, L, Hq, Hkv, d, P, flags;
-};
-
-__device__ __forceinline__ bool attn_computed(int state, int flags) { return !((flags & TEAM_F_DCD) && state == TEAM_TOK_CACHED); }
 
 __device__ __forceinline__ void at_cp16(uint32_t dst, const void* src, int bytes) {   // bytes 0: zero fill
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(bytes) : "memory");
@@ -427,8 +405,14 @@ extern "C" int team_block_attention(const team_attn_config* cfg, const team_step
   at[0].val.clusterDim.x = 1; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = n_splits;
   lc.attrs = at;
   lc.numAttrs = 1;
-  cudaError_t e = a.d == 128 ? cudaLaunchKernelEx(&lc, team::k_block_attention<128>, a, n_splits)
-                             : cudaLaunchKernelEx(&lc, team::k_block_attention<64>, a, n_splits);
+  // head size 128: the tensor-memory kernel; head size 64: the fragment kernel
+  cudaError_t e;
+  if (a.d == 128) {
+    e = team::configure_attention_tc();
+    if (e == cudaSuccess) e = team::launch_attention_tc(a, m_tiles, n_splits, s);
+  } else {
+    e = cudaLaunchKernelEx(&lc, team::k_block_attention<64>, a, n_splits);
+  }
   if (e != cudaSuccess) {
     cudaGetLastError();
     return TEAM_ERR_CUDA;

@@ -61,6 +61,44 @@ def test_block_attention_over_a_schedule(shape, flags, d, Hq, Hkv, P):
         assert (kb != 0).any()          # something was inserted along the way
 
 
+@pytest.mark.parametrize("flags", [0, B.TEAM_F_DCD], ids=["recompute_all", "delayed_caching"])
+@pytest.mark.parametrize("d,Hq,Hkv", [(128, 16, 2), (64, 8, 1)], ids=["d128", "d64"])
+def test_block_attention_long_prefix(flags, d, Hq, Hkv):
+    """A prefix of many key tiles with a ragged end, eight query heads per key/value head (more (row, head) pairs than
+    one CTA holds) and few enough CTAs that the keys are split over a cluster; queries scaled up so that the running
+    maximum keeps moving (the rescaling of the output accumulator is exercised, not only its first tile)."""
+    shape = W.paper_point()
+    rng = np.random.default_rng(977 + d)
+    steps = W.make_schedule(shape)[:2]
+    S, Bn, L, T = shape.seqs, shape.branches, shape.block, shape.rows
+    P = 1000
+    cfg = B.team_attn_config(Hq, Hkv, d, L, S, Bn, P, flags)
+    kp, vp = _bf16(rng, S, P, Hkv, d), _bf16(rng, S, P, Hkv, d)
+    plen = np.full(S, 937, np.int32)
+    kb, vb = _bf16(rng, S, L, Hkv, d), _bf16(rng, S, L, Hkv, d)
+    kb_dev, vb_dev = _dev(kb), _dev(vb)
+    out_dev = torch.full((T, Hq, d), 3.0, dtype=torch.float32, device="cuda")
+    out_ref = np.full((T, Hq, d), 3.0)
+    status = torch.zeros(2, dtype=torch.int32, device="cuda")
+    for si, step in enumerate(steps):
+        q = W.round_to_bf16((6.0 * rng.standard_normal((T, Hq, d))).astype(np.float32))
+        k, v = _bf16(rng, T, Hkv, d), _bf16(rng, T, Hkv, d)
+        rc = B.team_block_attention(cfg, B.state_to_device(step), _dev(q), _dev(k), _dev(v), _dev(kp), _dev(vp),
+                                    torch.as_tensor(plen).cuda(), kb_dev, vb_dev, out_dev, status)
+        assert rc == B.TEAM_OK
+        torch.cuda.synchronize()
+        assert status.cpu().tolist() == [0, 0]
+        out_ref, kb, vb = A.block_attention(q, k, v, kp, vp, plen, kb, vb, step["tok_state"], step["pos"], step["group"],
+                                            step["branch"], L, flags, out_prev=out_ref)
+        got = out_dev.cpu().numpy()
+        comp = A.computed_rows(step["tok_state"], flags)
+        err = np.abs(got[comp] - out_ref[comp]).max()
+        assert err <= TOL * np.abs(out_ref[comp]).max(), f"step {si}: {err}"
+        out_ref[~comp] = got[~comp]
+        np.testing.assert_array_equal(kb_dev.float().cpu().numpy(), kb.astype(np.float32))
+        np.testing.assert_array_equal(vb_dev.float().cpu().numpy(), vb.astype(np.float32))
+
+
 def test_block_attention_rejects_what_it_cannot_run():
     z = torch.zeros(16, dtype=torch.bfloat16, device="cuda")
     st = dict(tok_state=torch.zeros(4, dtype=torch.uint8, device="cuda"), pos=torch.arange(4, dtype=torch.int32, device="cuda"),
