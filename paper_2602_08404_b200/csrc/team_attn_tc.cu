@@ -155,15 +155,17 @@ __global__ void __launch_bounds__(kAtThreads, 1) k_block_attention_tc(AttnArgs a
   const int ltid = tid - 160, lw = warp - 5;
   constexpr int RPI = kAtLoadThreads / 16;                  // key rows covered per step of the copy loop
   const int c = ltid & 15, jr = ltid >> 4;                  // a loader thread's 16-byte piece and key row (jr + RPI i)
-  auto issue_tile = [&](int i) {                            // tile t_begin + i into key stage i % 3 and staging i % 3
-    const uint32_t kst = sm0 + kAtOffK + (i % kAtKStages) * kAtKBytes, vst = sm0 + kAtOffV + (i % kAtVStages) * kAtVBytes;
+  // Keys and values travel through registers (16-byte loads, two tiles ahead, then 16-byte shared-memory stores):
+  // cp.async tops out near 20 B per clock and SM here, a third of what one tile per microsecond needs.
+  constexpr int NR = kAtKeys / RPI;                         // key rows per loader thread and tile
+  uint4 kr0[NR], vr0[NR], kr1[NR], vr1[NR];                 // tiles of even / odd index
+  auto load_tile = [&](int i, uint4 (&kk)[NR], uint4 (&vv)[NR]) {
 #pragma unroll
-    for (int r8 = 0; r8 < kAtKeys / RPI; ++r8) {
-      const int j = r8 * RPI + jr, key = (t_begin + i) * kAtKeys + j;
-      const __nv_bfloat16 *ks = a.k_prefix, *vs = a.v_prefix;
-      int bytes = 0;
+    for (int r8 = 0; r8 < NR; ++r8) {
+      const int key = (t_begin + i) * kAtKeys + r8 * RPI + jr;
+      kk[r8] = vv[r8] = make_uint4(0u, 0u, 0u, 0u);          // keys past the end: zero rows
       if (key < n_keys) {
-        bytes = 16;
+        const __nv_bfloat16 *ks = a.k_prefix, *vs = a.v_prefix;
         size_t o;
         if (key < plen) {
           o = (((size_t)s * a.P + key) * a.Hkv + g) * kAtD;
@@ -177,17 +179,24 @@ __global__ void __launch_bounds__(kAtThreads, 1) k_block_attention_tc(AttnArgs a
             ks = a.k_block; vs = a.v_block;
           }
         }
-        ks += o + c * 8; vs += o + c * 8;
+        kk[r8] = __ldg(reinterpret_cast<const uint4*>(ks + o + c * 8));
+        vv[r8] = __ldg(reinterpret_cast<const uint4*>(vs + o + c * 8));
       }
-      at_cp16z(kst + (c >> 3) * (kAtKeys * 128) + sw128(j, c & 7), ks, bytes);
-      at_cp16z(vst + j * 256 + ((c ^ (j & 7)) << 4), vs, bytes);
+    }
+  };
+  auto store_tile = [&](int i, const uint4 (&kk)[NR], const uint4 (&vv)[NR]) {   // key stage i % 3, staging i % 3
+    unsigned char* kst = smem + kAtOffK + (i % kAtKStages) * kAtKBytes;
+    unsigned char* vst = smem + kAtOffV + (i % kAtVStages) * kAtVBytes;
+#pragma unroll
+    for (int r8 = 0; r8 < NR; ++r8) {
+      const int j = r8 * RPI + jr;
+      *reinterpret_cast<uint4*>(kst + (c >> 3) * (kAtKeys * 128) + sw128(j, c & 7)) = kk[r8];
+      *reinterpret_cast<uint4*>(vst + j * 256 + ((c ^ (j & 7)) << 4)) = vv[r8];
     }
   };
   if (warp >= 5) {
-    if (n_tiles > 0) issue_tile(0);
-    cp_async_commit();
-    if (n_tiles > 1) issue_tile(1);
-    cp_async_commit();
+    if (n_tiles > 0) load_tile(0, kr0, vr0);
+    if (n_tiles > 1) load_tile(1, kr1, vr1);
   }
   // ---- the queries of this CTA's pairs: A operand of S = Q K^T, two k-blocks of [128 rows][128 B], swizzled ----
   for (int i = tid; i < kAttnPairs * 16 && warp < 5; i += 160) {
@@ -210,17 +219,22 @@ __global__ void __launch_bounds__(kAtThreads, 1) k_block_attention_tc(AttnArgs a
     // ------------------------------ loaders ------------------------------
     bool ok = true;
     for (int i = 0; i < n_tiles; ++i) {
-      at_cp_wait<1>();                                      // this thread's pieces of tile i have landed
-      fence_async_smem();
-      if (ok) mbar_arrive(smem_u32(k_full + i % kAtKStages));
-      bar_loaders();                                        // ... and everybody else's: the staged values are complete,
-                                                            // and every warp is done transposing tile i - 1
-      if (ok && i + 2 < n_tiles) {
-        // tile i + 2 takes the stages of tile i - 1: its keys were read by S(i - 1)
-        ok = mbar_wait_warp(smem_u32(k_empty + (i + 2) % kAtKStages), (((i + 2) / kAtKStages) & 1) ^ 1, abort_flag, status, 51);
-        if (ok) issue_tile(i + 2);
+      // the key stage of tile i was read by S(i - 3)
+      if (ok && i >= kAtKStages)
+        ok = mbar_wait_warp(smem_u32(k_empty + i % kAtKStages), ((i / kAtKStages) & 1) ^ 1, abort_flag, status, 51);
+      if (ok) {
+        if (i & 1) {
+          store_tile(i, kr1, vr1);
+          if (i + 2 < n_tiles) load_tile(i + 2, kr1, vr1);
+        } else {
+          store_tile(i, kr0, vr0);
+          if (i + 2 < n_tiles) load_tile(i + 2, kr0, vr0);
+        }
       }
-      cp_async_commit();
+      fence_async_smem();                                   // generic-proxy writes, read by the tensor core
+      if (ok) mbar_arrive(smem_u32(k_full + i % kAtKStages));
+      bar_loaders();                                        // the staged values are complete, and every warp is done
+                                                            // transposing tile i - 1
       if (ok) ok = mbar_wait_warp(smem_u32(vt_empty + (i & 1)), ((i >> 1) & 1) ^ 1, abort_flag, status, 52);
       if (ok) {
         // V^T: 8 x 8 blocks transposed on the way; the warps share the 16 head-dimension pieces
@@ -242,7 +256,6 @@ __global__ void __launch_bounds__(kAtThreads, 1) k_block_attention_tc(AttnArgs a
         if (lane == 0) mbar_arrive(smem_u32(vt_full + (i & 1)));
       }
     }
-    at_cp_wait<0>();
   } else if (warp == 4) {
     // ------------------------------ MMA issuer ------------------------------
     const uint32_t idesc_s = make_idesc_bf16(kAtKeys), idesc_o = make_idesc_bf16(kAtD);
@@ -322,11 +335,10 @@ __global__ void __launch_bounds__(kAtThreads, 1) k_block_attention_tc(AttnArgs a
       float mx = kNegInf;
 #pragma unroll
       for (int e = 0; e < kAtKeys; ++e) {
-        float v = sc[e] * sl2;
-        if (ragged && key0 + e >= n_keys) v = kNegInf;
-        sc[e] = v;
-        mx = fmaxf(mx, v);
+        if (ragged && key0 + e >= n_keys) sc[e] = kNegInf;
+        mx = fmaxf(mx, sc[e]);
       }
+      mx *= sl2;                                             // sl2 > 0: the maximum of the scaled scores
       // the maximum in use moves only when it has to: P stays below 2^8, far inside fp32 and the bf16 pair
       const bool move = mx > m_used + kAtRescale;            // always on the first tile (m_used = -inf)
       float corr = 1.f;
@@ -336,9 +348,10 @@ __global__ void __launch_bounds__(kAtThreads, 1) k_block_attention_tc(AttnArgs a
         l_run *= corr;
       }
       float sum = 0.f;
+      const float neg_m = -m_used;
 #pragma unroll
       for (int e = 0; e < kAtKeys; ++e) {
-        sc[e] = at_ex2(sc[e] - m_used);
+        sc[e] = at_ex2(fmaf(sc[e], sl2, neg_m));             // scale and shift in one operation
         sum += sc[e];
       }
       l_run += sum;
