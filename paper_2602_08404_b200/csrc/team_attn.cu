@@ -3,6 +3,8 @@
 // of cached tokens are not computed and their keys / values come from an in-block cache, followed by the delayed
 // insertion of the newly accepted tokens' keys / values into that cache.
 //
+// team_block_attention runs head size 128 on the tensor-memory kernel of team_attn_tc.cu and head size 64 on
+// k_block_attention below.
 // k_block_attention: a contraction, so it runs on the tensor cores.  The (computed row, query head) pairs that share
 // one (sequence, branch) and one key / value head are the M side: a CTA owns 128 of them (8 warps x 16), their
 // queries live in registers as A fragments.  Keys and values are walked in tiles of 64 (prefix first, then the
@@ -338,9 +340,7 @@ static cudaError_t configure_attn(int* n_sms) {
     *n_sms = sms[dev];
     return cudaSuccess;
   }
-  e = cudaFuncSetAttribute(k_block_attention<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attn_smem_bytes(128));
-  if (e == cudaSuccess)
-    e = cudaFuncSetAttribute(k_block_attention<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attn_smem_bytes(64));
+  e = cudaFuncSetAttribute(k_block_attention<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attn_smem_bytes(64));
   int n = 0;
   if (e == cudaSuccess) e = cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
   if (e != cudaSuccess) return e;
