@@ -38,6 +38,7 @@ struct SelSmem {
   uint8_t* state;      // [T]
   uint8_t* cls;        // [T]
   uint8_t* has_first;  // [G]
+  int32_t* own;        // [T + 1] kSelRounds: the rows this CTA routes, own[T] = how many
 };
 
 __host__ __device__ inline size_t sel_smem_layout(Dims d, SelSmem* s, unsigned char* base) {
@@ -61,6 +62,7 @@ __host__ __device__ inline size_t sel_smem_layout(Dims d, SelSmem* s, unsigned c
   size_t a_state = take((size_t)d.T);
   size_t a_cls = take((size_t)d.T);
   size_t a_hf = take((size_t)d.G);
+  size_t a_own = take((size_t)(d.T + 1) * 4);
   if (s != nullptr) {
     s->mask = reinterpret_cast<uint32_t*>(base + a_mask);
     s->mask2 = reinterpret_cast<uint32_t*>(base + a_mask2);
@@ -74,6 +76,7 @@ __host__ __device__ inline size_t sel_smem_layout(Dims d, SelSmem* s, unsigned c
     s->state = base + a_state;
     s->cls = base + a_cls;
     s->has_first = base + a_hf;
+    s->own = reinterpret_cast<int32_t*>(base + a_own);
   }
   return o;
 }
@@ -116,6 +119,7 @@ k_select(const float* __restrict__ logits, StepPtrs st, Workspace ws, RoutePtrs 
   // ---- stage the step state (inputs of the call, not produced by the preceding kernel) ---------
   for (int i = tid; i < d.G * n_words32; i += kSelThreads) s.mask[i] = 0u;
   for (int i = tid; i < d.G; i += kSelThreads) s.has_first[i] = 0;
+  if (tid == 0) s.own[T] = 0;
   for (int i = tid; i < nw * EN; i += kSelThreads) s.hist[i] = 0;
   float conf_r[TEAM_MAX_ROWS / kSelThreads];     // confidences of the rows this thread classifies, fetched with the rest
 #pragma unroll
@@ -168,6 +172,19 @@ k_select(const float* __restrict__ logits, StepPtrs st, Workspace ws, RoutePtrs 
   for (int t = tid; t < T && mode != kSelDispatch; t += kSelThreads)
     if (s.cls[t] == TEAM_CLS_COLD && !s.has_first[s.key[t] >> 8]) s.cls[t] = TEAM_CLS_FIRST;
 
+  // kSelRounds: the rows of this CTA's groups, listed once (in any order: rows are routed independently and E_A
+  // is a union), so that the routing rounds walk 1/grid of the rows instead of testing every row in every warp
+  if (mode == kSelRounds) {
+    for (int t0r = 0; t0r < T; t0r += kSelThreads) {
+      const int t = t0r + tid;
+      const bool mine = t < T && (s.key[t] >> 8) % nb == cta;
+      const unsigned bal = __ballot_sync(0xffffffffu, mine);
+      int base = 0;
+      if (lane == 0 && bal) base = atomicAdd(&s.own[T], __popc(bal));
+      base = __shfl_sync(0xffffffffu, base, 0);
+      if (mine) s.own[base + __popc(bal & ((1u << lane) - 1u))] = t;
+    }
+  }
   // Everything above depends on the step state only (inputs of the call) and overlaps the preceding
   // kernel of the stream; the logits come from that kernel.
   if (wait_prior) asm volatile("griddepcontrol.wait;" ::: "memory");
@@ -186,8 +203,9 @@ k_select(const float* __restrict__ logits, StepPtrs st, Workspace ws, RoutePtrs 
 
   // ---- Algorithm 1, round 1 (free top-k) then round 2 (top-k inside E_A) -------------------
   for (int round = 1; round <= 2 && mode != kSelDispatch; ++round) {
-    for (int t = t0 + warp; t < t1; t += kSelWarps) {
-      if (!own_row(t)) continue;
+    const int n_mine = mode == kSelRounds ? s.own[T] : t1 - t0;
+    for (int i = warp; i < n_mine; i += kSelWarps) {
+      const int t = mode == kSelRounds ? s.own[i] : t0 + i;
       const uint8_t c = s.cls[t];
       if (round == 1 && c == TEAM_CLS_SKIP) {
         if (lane < k) {
