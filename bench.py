@@ -290,8 +290,9 @@ def run_layer(args):
     launches_per_step = B.team_last_launch_count(ctxs[0])
     bytes_per_expert = 3 * H * I * 2
 
-    # CUDA graphs: one full cycle (period steps), and the remainder of the timed region (steps % period), so that
-    # the timed region consists of graph replays only, whatever --steps is
+    # CUDA graphs: one graph of whole cycles (up to 64 steps, no more than the timed region holds), and the remainder
+    # of the timed region (steps % that), so that the timed region consists of graph replays only, whatever --steps
+    # is, and a replay's launch gap is spread over many steps
     def capture(n):
         g = torch.cuda.CUDAGraph()
         with torch.cuda.graph(g):
@@ -300,7 +301,8 @@ def run_layer(args):
         return g
 
     graph = tail_graph = None
-    n_tail = args.steps % period
+    chunk = period * max(1, min(64 // period, args.steps // period))
+    n_tail = args.steps % chunk
     if not args.no_graph:
         try:
             side = torch.cuda.Stream(device=dev)
@@ -310,26 +312,26 @@ def run_layer(args):
                     one_step(i)
             torch.cuda.current_stream().wait_stream(side)
             torch.cuda.synchronize()
-            graph = capture(period)
+            graph = capture(chunk)
             tail_graph = capture(n_tail) if n_tail else None
         except Exception as e:                                   # report, and time plain launches instead
             print(f"[bench] CUDA graph capture failed ({e}); timing plain launches", file=sys.stderr)
             graph = tail_graph = None
 
     def run_steps(n):
-        """Issues exactly n steps: whole cycles as graph replays, the remainder as one more replay (n % period ==
-        steps % period) or as plain calls."""
+        """Issues exactly n steps: whole graphs of `chunk` steps as replays, the remainder as one more replay (n %
+        chunk == steps % chunk) or as plain calls."""
         if graph is None:
             for i in range(n):
                 one_step(i)
             return n
-        for _ in range(n // period):
+        for _ in range(n // chunk):
             graph.replay()
-        if n % period:
-            if tail_graph is not None and n % period == n_tail:
+        if n % chunk:
+            if tail_graph is not None and n % chunk == n_tail:
                 tail_graph.replay()
             else:
-                for i in range(n % period):
+                for i in range(n % chunk):
                     one_step(i)
         return n
 
@@ -342,12 +344,12 @@ def run_layer(args):
     with sampler:
         # ---- device-resident timing -----------------------------------------------------------------
         # Untimed, whatever --warmup says: every graph replayed at least twice, every context called, and at least
-        # ~20 ms of the workload so that the clocks have settled.  Then the caller's warm-up steps.
+        # ~90 ms of the workload so that the clocks have settled (a first process on a cold GPU needs it).  Then the caller's warm-up steps.
         warm = 0
         for _ in range(2):
-            warm += run_steps(period + n_tail)
+            warm += run_steps(chunk + n_tail)
         warm += run_steps(max(args.warmup, 3))
-        warm += run_steps(period * max(0, (600 - warm + period - 1) // period))
+        warm += run_steps(chunk * max(0, (3000 - warm + chunk - 1) // chunk))
         barrier()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record()
@@ -439,7 +441,7 @@ def run_layer(args):
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16", "data": "synthetic",
         "config": config_of(args, shape, workload),
-        "run": {"layers_cycled": R, "weights_gb": R * (E + ns) * bytes_per_expert / 1e9, "cuda_graph": graph is not None,
+        "run": {"layers_cycled": R, "weights_gb": R * (E + ns) * bytes_per_expert / 1e9, "cuda_graph": graph is not None, "graph_steps": chunk if graph is not None else 0,
                 "steps_issued": issued, "warmup_issued": warm, "e2e_warmup_issued": e2e_warm,
                 "rows_computed_mean": mean_rows, "activated_experts_mean": mean_act},
         "clocks": clocks,
