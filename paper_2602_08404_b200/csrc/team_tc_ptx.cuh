@@ -164,7 +164,7 @@ __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
 // One-dimensional bulk copy global -> shared (both 16-byte aligned, size a multiple of 16 bytes); the barrier
-// receives the bytes as they land.  No multicast: every CTA fetches its own tiles.
+// receives the bytes as they land.  Every CTA fetches its own tiles (no copy is shared between the CTAs of a cluster).
 __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
   asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                ::"r"(dst), "l"(src), "r"(bytes), "r"(bar)
