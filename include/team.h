@@ -41,7 +41,11 @@
  * Row layout.  A call presents T = n_rows rows.  Rows that share (group,
  * branch) must be contiguous and form one decoding block (at most
  * TEAM_MAX_BLOCK rows); `pos` is the position inside that block.  `group` is
- * the scope of E_A (normally the sequence), 0 <= group < max_groups.
+ * the scope of E_A (normally the sequence), 0 <= group < max_groups.  A run
+ * longer than TEAM_MAX_BLOCK, or a group / branch index out of range, is
+ * reported as TEAM_ERR_STATE in the device status; rows of one (group,
+ * branch) that are NOT contiguous are not detected: each run then counts as a
+ * block of its own for the distance test of Eq. 4.
  *
  * Slot ids.  Row t's j-th routed choice is slot t*top_k + j.  Shared expert s
  * (expert id n_experts + s) applied to row t is slot T*top_k + s*T + t and has
